@@ -1,0 +1,339 @@
+"""Benchmark of the Step-Ahead Error Feedback hot path (one Algorithm-1 iteration = one step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--avg-period p] [--impl reference]
+
+Prints ONE JSON line.  `value` = steps/s over all N GPUs with the gradients already resident in HBM
+(a ring of pre-generated gradient sets, each far larger than L2, cycled step by step); `e2e` = the
+same step driven through the host-buffer entry points (pinned host gradients copied in, parameters
+copied out, inside the timed region); `roofline` = the dominant kernel (the worker pass) against the
+measured HBM copy bandwidth; `cpu_baseline` = the CPU oracle timed on a bounded sample of the same
+workload.  The path does not shard (the workers are a batch axis on one GPU), so N > 1 runs N
+independent replicas: no data-path collective, "scaling": "weak".
+
+`--impl reference` times the CPU oracle alone (there is no reference implementation of this paper).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "step-ahead EF steps/sec at W workers x d params"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one worker-pass launch per worker-element, from the committed ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case of the same kernel, which grows in
+# proportion to the elements processed).  None until a capture exists for the variant.
+WORKER_PASS_DRAM_BYTES_PER_ELEM = {"sign_p1": None, "sign_general": None, "topk": None}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, stream copy)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.splitlines():
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def sample_tensors(sizes, budget):
+    """A bounded sample of whole tensors (largest that fits, smallest, median, then a seeded shuffle)."""
+    import numpy as np
+    order = np.argsort(sizes)
+    pick = [int(j) for j in order[::-1] if sizes[j] <= budget][:1] + [int(order[0]), int(order[len(order) // 2])]
+    pick += [int(j) for j in np.random.default_rng(0).permutation(len(sizes))]
+    out, total = [], 0
+    for j in dict.fromkeys(pick):
+        if total + sizes[j] <= budget or not out:
+            out.append(j)
+            total += sizes[j]
+    return sorted(out)
+
+
+def cpu_baseline(w, avg_period, seed, steps, warmup, target_elems=40_000_000):
+    """The oracle, as it stands, on a sample of whole tensors of the workload (all K workers)."""
+    import numpy as np
+    from oracle import sae_oracle as so
+    from paper_2008_05823_b200 import synth
+    K, sizes = w.num_workers, w.tensor_sizes
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    js = sample_tensors(sizes, max(1, target_elems // K))
+    sub = [sizes[j] for j in js]
+    n_sub = int(sum(sub))
+    scales = synth.workload_scales(w, seed)
+    threads = max(1, min(so.max_threads(), len(os.sched_getaffinity(0))))
+    x0 = np.concatenate([synth.x0_numpy_range(seed, int(offs[j]), sizes[j]) for j in js])
+    orc = so.Oracle(K, sub, x0, compressor=w.compressor, avg_period=avg_period, momentum=w.momentum,
+                    weight_decay=w.weight_decay, topk_num=w.topk_num, topk_den=w.topk_den, threads=threads)
+    grads = [np.stack([np.concatenate([synth.grads_numpy_range(seed, t, k, int(offs[j]), sizes[j], scales[j],
+                                                               w.outlier_per_65536, w.outlier_mult) for j in js])
+                       for k in range(K)]) for t in range(2)]
+    for t in range(warmup):
+        t0 = time.perf_counter()
+        orc.step(grads[t % 2], w.lr)
+        warm_dt = time.perf_counter() - t0
+    if steps <= 0:                      # aim at ~15 s of CPU work
+        steps = int(max(2, min(200, 15.0 / max(warm_dt, 1e-3))))
+    t0 = time.perf_counter()
+    for t in range(steps):
+        orc.step(grads[t % 2], w.lr)
+    dt = time.perf_counter() - t0
+    frac = n_sub / w.d
+    return {"value": steps / dt * frac, "unit": "steps/s", "cores": threads, "kind": "oracle",
+            "sample": f"{len(js)} of {len(sizes)} whole tensors ({n_sub} of {w.d} params = {100 * frac:.2f}%), all "
+                      f"{K} workers, {steps} steps in {dt:.2f} s; value = sample steps/s x sampled fraction",
+            "sample_seconds": dt, "ms_per_sample_step": 1e3 * dt / steps}
+
+
+def run_reference(args, w, avg_period, rank):
+    if rank != 0:
+        return
+    steps, warmup = max(1, args.steps), max(1, args.warmup)
+    cb = cpu_baseline(w, avg_period, args.seed, steps, warmup, target_elems=30_000_000)
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": 1e3 / cb["value"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "num_workers": w.num_workers, "d": w.d, "avg_period": avg_period,
+                       "note": "no reference implementation exists for this paper: this arm is the CPU oracle"},
+            "cpu_baseline": cb,
+            "e2e": {"value": cb["value"], "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def algorithmic_bytes(w, avg_period):
+    """Bytes the method itself must move per step (each gradient read once, each persistent state word
+    read and written once) and per launch of the worker pass."""
+    Wd, d = w.num_workers * w.d, w.d
+    if avg_period == 1:
+        step = 12 * Wd + 24 * d              # g R, m RW | x RW, e_srv RW, ebar RW
+        worker = 12 * Wd + 4 * d             # g R, m RW | ebar R once
+        variant = "sign_p1" if w.compressor == 1 else "topk"
+    else:
+        step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW
+        worker = 20 * Wd                     # g R, m RW, Delta(e) RW
+        variant = "sign_general" if w.compressor == 1 else "topk"
+    return step, worker, variant
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=4, help="index into BASELINE.json configs (default: the largest)")
+    ap.add_argument("--avg-period", type=int, default=1,
+                    help="error-averaging period p (1 = average inside every step; 0 = never)")
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--ring", type=int, default=0, help="gradient sets kept in HBM (0 = auto)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
+
+    from paper_2008_05823_b200 import configs
+    w = configs.workload(args.workload)
+    p = args.avg_period
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, w, p, rank)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2008_05823_b200 import binding as sb
+    from paper_2008_05823_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, d = w.num_workers, w.d
+    scales = synth.workload_scales(w, args.seed)
+    gen = synth.DeviceGenerator(w.tensor_sizes, scales, device=dev)
+    x0 = torch.empty(d, device=dev)
+    gen.x0(x0, args.seed)
+    grad_bytes = 4 * K * d
+    ring = args.ring or int(max(2, min(4, (40 << 30) // grad_bytes, args.steps + args.warmup)))
+    grads = []
+    for t in range(ring):
+        g = torch.empty(K, d, device=dev)
+        gen.grads(g, K, args.seed, t, w.outlier_per_65536, w.outlier_mult)
+        grads.append(g)
+
+    def make():
+        return sb.Sae(K, w.tensor_sizes, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
+                      avg_period=p, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
+                      topk_den=w.topk_den)
+
+    # ---- device-resident throughput ------------------------------------------------------------------
+    sae = make()
+    for t in range(args.warmup):
+        sae.step(grads[t % ring], w.lr)
+    sae.sync()
+    sampler = ClockSampler(local_rank)
+    launches0 = sae.kernel_launches
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    ev0.record()
+    for t in range(args.steps):
+        sae.step(grads[(args.warmup + t) % ring], w.lr)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    gpu_launches = sae.kernel_launches - launches0
+    sae.sync()                                    # raises if the device flagged a range error
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)
+
+    # ---- per-kernel times (same steps again, every launch bracketed by events on the library's stream) ----
+    sae.set_profiling(True)
+    for t in range(args.steps):
+        sae.step(grads[(args.warmup + t) % ring], w.lr)
+    ktimes = sae.get_kernel_times()
+    sae.set_profiling(False)
+    total_k = sum(ms for ms, _ in ktimes.values())
+    kernels = {name: {"launches": cnt, "ms_per_launch": ms / cnt, "share": ms / total_k}
+               for name, (ms, cnt) in ktimes.items()}
+    step_bytes, worker_bytes, variant = algorithmic_bytes(w, p)
+    peak, peak_source = measured_peak()
+    wk_ms = kernels["worker_pass"]["ms_per_launch"]
+    achieved = worker_bytes / (wk_ms * 1e-3) / 1e9
+    per_elem = WORKER_PASS_DRAM_BYTES_PER_ELEM.get(variant)
+    roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": (per_elem * K * d) if per_elem else None,
+                "algorithmic_bytes_per_launch": worker_bytes, "ms_per_launch": wk_ms, "peak_source": peak_source,
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "step": {"algorithmic_bytes": step_bytes, "achieved_GBs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+                         "frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
+                "kernels": kernels}
+    sae.close()
+    del sae
+
+    # ---- end to end through the host-buffer entry points --------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        import psutil
+        if psutil.virtual_memory().available > 3 * grad_bytes + (8 << 30):
+            host_g = torch.empty(K, d, dtype=torch.float32, pin_memory=True)
+            host_g.copy_(grads[0])
+            host_x = torch.empty(d, dtype=torch.float32, pin_memory=True)
+            sae = make()
+            e2e_steps = max(2, min(args.steps, int(4e9 // grad_bytes) + 2))
+            for _ in range(2):
+                sae.step_host(host_g, w.lr)
+                sae.get_params_host(host_x)
+            barrier()
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                sae.step_host(host_g, w.lr)          # H2D of this step's gradients + the step
+                sae.get_params_host(host_x)          # D2H of the step's result, synchronises
+            torch.cuda.synchronize()
+            dt = time.perf_counter() - t0
+            if world > 1:
+                tt = torch.tensor([dt], device=dev)
+                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+                dt = float(tt.item())
+            sae.sync()
+            sae.close()
+            e2e = {"value": world * e2e_steps / dt, "unit": "steps/s", "h2d_bytes_per_step": grad_bytes,
+                   "d2h_bytes_per_step": 4 * d, "steps": e2e_steps, "ms_per_step": 1e3 * dt / e2e_steps,
+                   "api": "sae_step_host + sae_get_params_host (pinned host buffers)"}
+            del host_g, host_x
+        else:
+            e2e = {"value": None, "unit": "steps/s", "skipped": "not enough host memory to pin one gradient set"}
+
+    cb = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cb = cpu_baseline(w, p, args.seed, steps=0, warmup=1)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name, "num_workers": K, "d": d, "num_tensors": w.num_tensors,
+                           "compressor": {0: "identity", 1: "scaled_sign", 2: "topk"}[w.compressor],
+                           "avg_period": p, "momentum": w.momentum, "lr": w.lr, "weight_decay": w.weight_decay,
+                           "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
+                           "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient set "
+                                 f"(ring of {ring})"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cb}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,166 @@
+/*
+ * sae.h -- C ABI of the Step-Ahead Error Feedback hot path (sm_100a CUDA library, libsae.so).
+ *
+ * One handle holds the whole state of Algorithm 1 ("Distributed Momentum SGD with Double-Way
+ * Compression") for K data-parallel workers simulated as a batch axis on ONE GPU: parameters x,
+ * server error e, per-worker momentum m^(k) and per-worker error e^(k).  The caller supplies the
+ * stochastic gradients; the library performs every other line of the algorithm in CUDA kernels.
+ *
+ * Conventions
+ *  - All pointers are DEVICE pointers unless the name ends in _host.  The library never takes
+ *    ownership of a caller buffer; it owns its state and scratch (allocated in sae_init only).
+ *  - "Caller layout" of a parameter-shaped vector: the T tensors concatenated in list order with no
+ *    padding, d = sum_j n_j floats.  Gradients are [K][d] row-major in that layout.
+ *  - All work is enqueued on the stream given in the configuration and is asynchronous with respect
+ *    to the host unless stated otherwise.  A handle must not be used from two host threads at once.
+ *  - Arithmetic is IEEE fp32, round-to-nearest, denormals kept, with the fused operations fixed:
+ *    m = fma(mu, m, g'), Delta = fma(eta, m, e), g' = fma(lambda, xh, g); everything else is one
+ *    separately rounded operation; worker-axis sums run k = 0..K-1 from 0 and are divided by (float)K.
+ *  - Every function returns SAE_OK (0) or a negative sae_status.  No exceptions, no global state.
+ *    Errors detected on the device (non-finite or out-of-range values) are sticky and are reported
+ *    by the next sae_sync call.
+ */
+#ifndef SAE_H_
+#define SAE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SAE_ABI_VERSION 1u
+
+typedef enum {
+  SAE_OK = 0,
+  SAE_ERR_INVALID_ARG = -1, /* null pointer, K < 1, n_j <= 0, mu outside [0,1), lr <= 0, bad enum, ... */
+  SAE_ERR_NOMEM = -2,       /* device or host allocation failed                                          */
+  SAE_ERR_CUDA = -3,        /* a CUDA runtime call failed; sae_last_cuda_error gives the code            */
+  SAE_ERR_RANGE = -4,       /* a model difference was non-finite or had magnitude >= 2^32 (device check) */
+  SAE_ERR_TIMEOUT = -5,     /* reserved: a bounded device-side wait expired                               */
+  SAE_ERR_ABI = -6          /* abi_version mismatch                                                      */
+} sae_status;
+
+/* Compressor C(.) of Algorithm 1, applied per tensor (Section 5: "layer-wise"). */
+#define SAE_COMPRESSOR_IDENTITY 0 /* C(v) = v: full-precision distributed momentum SGD (Section 2)       */
+#define SAE_COMPRESSOR_SIGN 1     /* Eq. 2: C(v) = (||v||_1 / n) sign(v), sent as 1 scale + 1 bit/element */
+#define SAE_COMPRESSOR_TOPK 2     /* Section 3.1: keep the k largest magnitudes, zero the rest           */
+
+#define SAE_MODE_EF 0   /* Algorithm 1, "Local Error Feedback" branch: gradient evaluated at x_t          */
+#define SAE_MODE_SAEF 1 /* Algorithm 1, "Step Ahead Error Feedback" branch: at x_t - e_t^(k)              */
+
+typedef struct sae_handle sae_handle; /* opaque, library-owned */
+
+typedef struct {
+  uint32_t abi_version;        /* must be SAE_ABI_VERSION                                               */
+  int32_t num_workers;         /* K of Algorithm 1, 1..1024                                             */
+  int32_t num_tensors;         /* T >= 1 compression segments                                           */
+  const int64_t *tensor_sizes; /* HOST pointer, T entries, 0 < n_j < 2^31; copied by sae_init           */
+  int32_t compressor;          /* SAE_COMPRESSOR_*                                                      */
+  int32_t server_compress;     /* 1: double-way compression (server applies C, keeps its error e);
+                                  0: single-way (server sends Delta uncompressed, e stays 0) (Section 5) */
+  int32_t mode;                /* SAE_MODE_*                                                            */
+  int32_t avg_period;          /* p >= 1: worker errors are averaged in the pre-step of every iteration
+                                  t with (t+1) mod p = 0 (Algorithm 1, Section 3.2); 0 = never (p = inf) */
+  float momentum;              /* mu in [0,1)                                                           */
+  float weight_decay;          /* lambda >= 0: coupled L2, lambda * (point where the gradient is
+                                  evaluated) is added to the gradient                                    */
+  uint32_t topk_num, topk_den; /* Top-K keeps k_j = max(1, floor(n_j*num/den)) entries per tensor; all
+                                  entries tying the k_j-th magnitude are kept, exact zeros never are     */
+  int32_t device;              /* CUDA device ordinal                                                   */
+  void *stream;                /* cudaStream_t (NULL = default stream)                                  */
+} sae_config;
+
+/*
+ * Algorithm 1, "Initialize": x = x0, m^(k) = 0, e^(k) = 0, e = 0, t = 0, then the pre-step of
+ * iteration 0.  x0: device, d floats, caller layout, copied.  Allocates all state and scratch.
+ * *out receives the handle.  Host-synchronous.
+ */
+int sae_init(const sae_config *cfg, const float *x0, sae_handle **out);
+
+/*
+ * One iteration t of Algorithm 1 (worker lines, server lines, re-update) followed by the pre-step
+ * (error averaging when due) of iteration t+1:
+ *   xh = x - e^(k) (SAEF) or x (EF);  m^(k) = mu m^(k) + (g^(k) + lambda xh);  Delta^(k) = e^(k) + lr m^(k);
+ *   e^(k) = Delta^(k) - C(Delta^(k));  Delta = e + (1/K) sum_k C(Delta^(k));  e = Delta - C(Delta);
+ *   x = x - C(Delta).
+ * grads: device, [K][d] floats, caller layout, read-only, must stay valid until the step has run.
+ * lr: eta_t > 0.  Enqueues kernels only; allocates nothing.
+ */
+int sae_step(sae_handle *h, const float *grads, float lr);
+
+/*
+ * Same step with the gradients in HOST memory (pinned memory gives an asynchronous copy): copies
+ * them to a library-owned device staging buffer on the handle's stream, then runs the step.  The
+ * staging buffer (K*d floats) is allocated by the first call.
+ */
+int sae_step_host(sae_handle *h, const float *grads_host, float lr);
+
+/* Algorithm 1, "Output": x_t into out (device, d floats, caller layout). */
+int sae_get_params(sae_handle *h, float *out);
+/* Same into HOST memory (through a library-owned device buffer allocated by the first call);
+ * synchronises the stream before returning. */
+int sae_get_params_host(sae_handle *h, float *out_host);
+
+/*
+ * The point where worker k must evaluate its next gradient: x_t - e_t^(k) in SAEF mode ("One step
+ * ahead"), x_t in EF mode.  out: device, d floats, caller layout.
+ */
+int sae_get_step_ahead(sae_handle *h, int32_t worker, float *out);
+
+/* State and last-message getters (parity checks, checkpointing). `out` is a DEVICE buffer of at least
+ * `bytes` bytes; the call fails with SAE_ERR_INVALID_ARG if that is too small.  Parameter-shaped
+ * results are in caller layout. */
+#define SAE_STATE_MOMENTUM 0      /* m^(k): d floats                                                    */
+#define SAE_STATE_WORKER_ERROR 1  /* e^(k) after the last pre-step: d floats                            */
+#define SAE_STATE_SERVER_ERROR 2  /* e: d floats (worker ignored)                                       */
+#define SAE_STATE_WORKER_SCALES 3 /* scaled sign: ||Delta^(k)||_1/n_j of the last step, T floats        */
+#define SAE_STATE_SERVER_SCALES 4 /* same for the server's Delta, T floats                              */
+#define SAE_STATE_WORKER_WORDS 5  /* sign words of C(Delta^(k)) of the last step (format below)         */
+#define SAE_STATE_SERVER_WORDS 6  /* sign words of C(Delta) of the last step                            */
+#define SAE_STATE_WORKER_TAU 7    /* Top-K: bit pattern of the k_j-th largest |Delta^(k)|, T uint32     */
+#define SAE_STATE_SERVER_TAU 8    /* same for the server, T uint32                                      */
+#define SAE_STATE_WORKER_MASK 9   /* Top-K: selected set of the last step as bit words (format below)   */
+#define SAE_STATE_SERVER_MASK 10  /* same for the server                                                */
+int sae_get_state(sae_handle *h, int32_t which, int32_t worker, void *out, size_t bytes);
+/*
+ * Bit-word format (sign message and Top-K mask): per tensor ceil(n_j/32) little-endian uint32 words,
+ * bit i of word w <-> element 32w+i of that tensor; sign: 1 <-> Delta_i >= 0 (code +scale), mask:
+ * 1 <-> selected; padding bits 0; the tensors' word arrays concatenated in list order.
+ */
+
+/* Number of iterations performed so far (t). */
+int64_t sae_iteration(const sae_handle *h);
+/* d = sum n_j, and the number of bit words per worker, sum_j ceil(n_j/32). */
+int64_t sae_num_params(const sae_handle *h);
+int64_t sae_num_words(const sae_handle *h);
+
+/* Waits for the stream; returns and clears the sticky device status (SAE_OK or SAE_ERR_RANGE...). */
+int sae_sync(sae_handle *h);
+
+/*
+ * Per-kernel timing.  With profiling enabled every kernel launch of sae_step is bracketed by CUDA
+ * events on the handle's stream.  sae_get_kernel_times synchronises, then writes for each of the
+ * SAE_NUM_KERNELS kernel slots the accumulated milliseconds and launch count since the last reset
+ * and resets them.  Slot names: sae_kernel_name(slot).
+ */
+#define SAE_NUM_KERNELS 12
+int sae_set_profiling(sae_handle *h, int32_t enabled);
+int sae_get_kernel_times(sae_handle *h, float *ms_host, int64_t *launches_host);
+const char *sae_kernel_name(int32_t slot);
+/* Total kernels launched by this handle so far. */
+int64_t sae_kernel_launches(const sae_handle *h);
+
+/* Frees everything the handle owns (synchronises first). NULL is allowed. */
+void sae_destroy(sae_handle *h);
+
+const char *sae_strerror(int status);
+/* cudaError_t of the most recent failed CUDA call made on behalf of this handle (0 if none);
+ * with h == NULL, of the most recent failed sae_init. */
+int sae_last_cuda_error(const sae_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAE_H_ */

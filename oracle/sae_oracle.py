@@ -64,6 +64,7 @@ class Oracle:
         self.dtype = np.dtype(dtype)
         self.suf = "f32" if self.dtype == np.float32 else "f64"
         self.K = int(num_workers)
+        self.mode = mode
         self.sizes = np.ascontiguousarray(tensor_sizes, dtype=np.int64)
         self.T = len(self.sizes)
         self.d = int(self.sizes.sum())
@@ -76,9 +77,12 @@ class Oracle:
             raise ValueError("oracle rejected the configuration")
 
     def __del__(self):
-        if getattr(self, "h", None):
-            getattr(lib(), f"sao_destroy_{self.suf}")(self.h)
-            self.h = None
+        try:
+            if getattr(self, "h", None):
+                getattr(lib(), f"sao_destroy_{self.suf}")(self.h)
+                self.h = None
+        except Exception:      # interpreter shutdown
+            pass
 
     def step(self, grads, lr):
         g = np.ascontiguousarray(grads, dtype=self.dtype)
@@ -111,7 +115,10 @@ class Oracle:
         return bool(getattr(lib(), f"sao_range_flag_{self.suf}")(self.h))
 
     def step_ahead(self, worker):
-        """x_{t+1/2}^(k) = x_t - e_t^(k): one subtraction in the run's precision."""
+        """The point where worker k evaluates its next gradient: x_t - e_t^(k) in the SAEF branch (one
+        subtraction in the run's precision), x_t in the EF branch."""
+        if self.mode == EF:
+            return self.get(self.X)
         return self.get(self.X) - self.get(self.E, worker)
 
 

@@ -1,0 +1,468 @@
+// Host side of libsae: configuration checks, the segment/tile planner, state allocation and the
+// per-iteration launch sequence of Algorithm 1.  Declarations and argument contracts: include/sae.h.
+#include "../../include/sae.h"
+#include "sae_kernels.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace sae;
+
+namespace {
+
+thread_local int g_init_cuda_error = 0;
+
+enum Slot { S_WORKER = 0, S_SERVER, S_APPLY, S_TOPK_HIST, S_TOPK_SELECT, S_EXPORT, S_IMPORT, S_MASK, S_COUNT };
+const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregate", "apply_update", "topk_hist",
+                                                 "topk_select", "export", "import", "mask_words",
+                                                 "", "", "", ""};
+
+struct EventPair { int slot; cudaEvent_t a, b; };
+
+}  // namespace
+
+struct sae_handle {
+  sae_config cfg;
+  std::vector<int64_t> sizes;
+  Plan P;
+  int device;
+  cudaStream_t stream;
+  // tables
+  int *d_tile_tensor, *d_first_tile, *d_n;
+  long long *d_off, *d_poff;
+  // state
+  float *x, *e_srv, *ebar, *m, *D;
+  u32 *words, *words_srv, *mask_srv;
+  float *scale[2], *scale_srv;
+  u32 *tau[2], *tau_srv;
+  L1Record *recs, *recs_srv;
+  u32 *hist;
+  SelectState* sel;
+  u32* status;
+  u32* status_host;      // pinned
+  float* staging;        // sae_step_host
+  float* out_stage;      // sae_get_params_host
+  int64_t t;
+  int esrc;              // how e^(k) is held now (ESRC_*)
+  int last;              // which of scale[2]/tau[2] holds the last step's values
+  int last_cuda_error;
+  int64_t launches;
+  // profiling
+  int profiling;
+  std::vector<EventPair> pending;
+  std::vector<cudaEvent_t> pool;
+  double ms[SAE_NUM_KERNELS];
+  int64_t cnt[SAE_NUM_KERNELS];
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev;
+  bool ok;
+  explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    ok = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define SAE_CUDA(h, call)                                  \
+  do {                                                     \
+    cudaError_t e_ = (call);                               \
+    if (e_ != cudaSuccess) {                               \
+      (h)->last_cuda_error = (int)e_;                      \
+      cudaGetLastError();                                  \
+      return e_ == cudaErrorMemoryAllocation ? SAE_ERR_NOMEM : SAE_ERR_CUDA; \
+    }                                                      \
+  } while (0)
+
+cudaEvent_t take_event(sae_handle* h) {
+  if (!h->pool.empty()) { cudaEvent_t e = h->pool.back(); h->pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+struct LaunchScope {
+  sae_handle* h; int slot; cudaEvent_t a, b;
+  LaunchScope(sae_handle* h_, int slot_) : h(h_), slot(slot_), a(nullptr), b(nullptr) {
+    if (h->profiling) { a = take_event(h); b = take_event(h); cudaEventRecord(a, h->stream); }
+  }
+  ~LaunchScope() {
+    h->launches++;
+    if (h->profiling) { cudaEventRecord(b, h->stream); h->pending.push_back({slot, a, b}); }
+  }
+};
+
+#define LAUNCH(h, slot, kern, grid, ...)                                   \
+  do {                                                                     \
+    LaunchScope ls_(h, slot);                                              \
+    kern<<<(unsigned)(grid), THREADS, 0, (h)->stream>>>(__VA_ARGS__);      \
+  } while (0)
+
+int check_launch(sae_handle* h) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { h->last_cuda_error = (int)e; return SAE_ERR_CUDA; }
+  return SAE_OK;
+}
+
+template <class T>
+cudaError_t dalloc(T** p, size_t count) {
+  *p = nullptr;
+  if (count == 0) count = 1;
+  return cudaMalloc((void**)p, count * sizeof(T));
+}
+
+void free_all(sae_handle* h) {
+  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D,
+                  h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
+                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage};
+  for (void* p : ptrs) if (p) cudaFree(p);
+  if (h->status_host) cudaFreeHost(h->status_host);
+  for (auto& ep : h->pending) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+  for (auto e : h->pool) cudaEventDestroy(e);
+}
+
+// ---- Top-K threshold of every (row, tensor) of buf[rows][dpad] ---------------------------------------
+void topk_thresholds(sae_handle* h, const float* buf, int rows, u32* tau_out) {
+  const Plan& P = h->P;
+  for (int level = 0; level < 3; ++level) {
+    LAUNCH(h, S_TOPK_HIST, k_topk_hist, (long long)P.ntiles * rows, P, rows, level, buf, h->sel, h->hist);
+    LAUNCH(h, S_TOPK_SELECT, k_topk_select, rows * P.T, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, h->hist,
+           h->sel, tau_out);
+  }
+}
+
+template <int ESRC, bool SIGN, bool WRITE_D>
+void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
+  LAUNCH(h, S_WORKER, (k_worker<ESRC, SIGN, WRITE_D>), (long long)h->P.ntiles * h->P.K, h->P, sp, wa);
+}
+
+template <int COMP, int SRV>
+void launch_apply(sae_handle* h, int avg, const ApplyArgs& aa) {
+  if (avg == AVG_NONE) LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_NONE>), h->P.ntiles, h->P, aa);
+  else if (avg == AVG_FROM_D) LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_FROM_D>), h->P.ntiles, h->P, aa);
+  else LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_RECOMPUTE>), h->P.ntiles, h->P, aa);
+}
+
+int do_step(sae_handle* h, const float* grads, float lr) {
+  const sae_config& c = h->cfg;
+  const Plan& P = h->P;
+  const bool avg_after = c.avg_period > 0 && ((h->t + 2) % c.avg_period == 0);
+  const int cur = 1 - h->last;
+  const bool dc = c.server_compress != 0;
+  StepParams sp;
+  sp.mu = c.momentum; sp.eta = lr; sp.lambda = c.weight_decay;
+  sp.saef = (c.mode == SAE_MODE_SAEF); sp.wd = (c.weight_decay != 0.0f);
+  WorkerArgs wa;
+  wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = h->ebar; wa.x = h->x;
+  wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
+  wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
+  ServerArgs sa;
+  sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
+  sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
+  ApplyArgs aa;
+  aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.m = h->m; aa.D = h->D;
+  aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.tau_cur = h->tau[cur]; aa.tau_srv = h->tau_srv;
+  aa.mask_srv = h->mask_srv; aa.eta = lr;
+
+  if (c.compressor == SAE_COMPRESSOR_SIGN) {
+    // The model differences need not be stored when the previous error was uniform and the next
+    // pre-step averages: the averaging pass recomputes them from m and ebar with the same fused op.
+    const bool write_d = !(h->esrc == ESRC_UNIFORM && avg_after);
+    if (write_d && !h->D) return SAE_ERR_INVALID_ARG;
+    if (h->esrc == ESRC_UNIFORM) {
+      if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
+      else launch_worker<ESRC_UNIFORM, true, false>(h, sp, wa);
+    } else {
+      launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
+    }
+    if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, P.ntiles, P, sa);
+    else LAUNCH(h, S_SERVER, k_server_sign<false>, P.ntiles, P, sa);
+    const int avg = avg_after ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
+    if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
+    h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
+  } else if (c.compressor == SAE_COMPRESSOR_TOPK) {
+    if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
+    else launch_worker<ESRC_LAZY_TOPK, false, true>(h, sp, wa);
+    topk_thresholds(h, h->D, P.K, h->tau[cur]);
+    LAUNCH(h, S_SERVER, k_server_dense<2>, P.ntiles, P, sa);
+    if (dc) topk_thresholds(h, h->e_srv, 1, h->tau_srv);
+    const int avg = avg_after ? AVG_FROM_D : AVG_NONE;
+    if (dc) launch_apply<2, 2>(h, avg, aa); else launch_apply<2, 0>(h, avg, aa);
+    h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
+  } else {
+    // identity: every error stays exactly zero, so e^(k) is the (all-zero) uniform vector forever
+    launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
+    LAUNCH(h, S_SERVER, k_server_dense<0>, P.ntiles, P, sa);
+    launch_apply<0, 0>(h, AVG_NONE, aa);
+    h->esrc = ESRC_UNIFORM;
+  }
+  h->last = cur;
+  h->t += 1;
+  return check_launch(h);
+}
+
+int export_vec(sae_handle* h, int what, int k, float* out) {
+  ExportArgs ea;
+  ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = h->ebar;
+  ea.scale_last = h->scale[h->last]; ea.tau_last = h->tau[h->last];
+  ea.esrc = h->esrc; ea.what = what; ea.k = k; ea.saef = (h->cfg.mode == SAE_MODE_SAEF);
+  LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
+  return check_launch(h);
+}
+
+}  // namespace
+
+extern "C" {
+
+int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
+  if (out) *out = nullptr;
+  if (!cfg || !x0 || !out) return SAE_ERR_INVALID_ARG;
+  if (cfg->abi_version != SAE_ABI_VERSION) return SAE_ERR_ABI;
+  if (cfg->num_workers < 1 || cfg->num_workers > MAX_WORKERS || cfg->num_tensors < 1 || !cfg->tensor_sizes)
+    return SAE_ERR_INVALID_ARG;
+  if (cfg->compressor < 0 || cfg->compressor > 2 || (cfg->mode != 0 && cfg->mode != 1) ||
+      (cfg->server_compress != 0 && cfg->server_compress != 1) || cfg->avg_period < 0)
+    return SAE_ERR_INVALID_ARG;
+  if (!(cfg->momentum >= 0.0f && cfg->momentum < 1.0f) || !(cfg->weight_decay >= 0.0f)) return SAE_ERR_INVALID_ARG;
+  if (cfg->compressor == SAE_COMPRESSOR_TOPK && (cfg->topk_den == 0 || cfg->topk_num > cfg->topk_den))
+    return SAE_ERR_INVALID_ARG;
+  if (cfg->device < 0) return SAE_ERR_INVALID_ARG;
+  const int T = cfg->num_tensors, K = cfg->num_workers;
+  long long d = 0, dpad = 0, ntiles = 0;
+  for (int j = 0; j < T; ++j) {
+    const int64_t n = cfg->tensor_sizes[j];
+    if (n <= 0 || n >= (1ll << 31)) return SAE_ERR_INVALID_ARG;
+    d += n; dpad += (n + 31) / 32 * 32; ntiles += (n + TILE - 1) / TILE;
+  }
+  if (ntiles * K >= (1ll << 31) || ntiles >= (1ll << 31)) return SAE_ERR_INVALID_ARG;
+
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) { g_init_cuda_error = (int)cudaGetLastError(); return SAE_ERR_CUDA; }
+
+  sae_handle* h = new (std::nothrow) sae_handle();
+  if (!h) return SAE_ERR_NOMEM;
+  h->cfg = *cfg;
+  h->sizes.assign(cfg->tensor_sizes, cfg->tensor_sizes + T);
+  h->cfg.tensor_sizes = h->sizes.data();
+  h->device = cfg->device;
+  h->stream = (cudaStream_t)cfg->stream;
+  h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
+  for (int i = 0; i < SAE_NUM_KERNELS; ++i) { h->ms[i] = 0; h->cnt[i] = 0; }
+
+  std::vector<int> tile_tensor((size_t)ntiles), first_tile(T), n32(T);
+  std::vector<long long> off(T), poff(T);
+  {
+    long long o = 0, po = 0; int tl = 0;
+    for (int j = 0; j < T; ++j) {
+      const long long n = h->sizes[j];
+      off[j] = o; poff[j] = po; first_tile[j] = tl; n32[j] = (int)n;
+      const int tj = (int)((n + TILE - 1) / TILE);
+      for (int q = 0; q < tj; ++q) tile_tensor[tl + q] = j;
+      tl += tj; o += n; po += (n + 31) / 32 * 32;
+    }
+  }
+  const bool sign = cfg->compressor == SAE_COMPRESSOR_SIGN, topk = cfg->compressor == SAE_COMPRESSOR_TOPK;
+  const bool need_D = !(sign && cfg->avg_period == 1);
+  const long long nwords = dpad / 32;
+  const size_t KT = (size_t)K * T;
+
+  int rc = SAE_OK;
+  auto fail = [&](cudaError_t e) {
+    h->last_cuda_error = (int)e; g_init_cuda_error = (int)e; cudaGetLastError();
+    rc = (e == cudaErrorMemoryAllocation) ? SAE_ERR_NOMEM : SAE_ERR_CUDA;
+  };
+#define TRY(call) do { if (rc == SAE_OK) { cudaError_t e_ = (call); if (e_ != cudaSuccess) fail(e_); } } while (0)
+#define ALLOC0(ptr, count) do { TRY(dalloc(&(ptr), (count))); \
+    if (rc == SAE_OK) TRY(cudaMemsetAsync((ptr), 0, (size_t)((count) ? (count) : 1) * sizeof(*(ptr)), h->stream)); } while (0)
+  ALLOC0(h->d_tile_tensor, (size_t)ntiles); ALLOC0(h->d_first_tile, T); ALLOC0(h->d_n, T);
+  ALLOC0(h->d_off, T); ALLOC0(h->d_poff, T);
+  ALLOC0(h->x, dpad); ALLOC0(h->e_srv, dpad); ALLOC0(h->ebar, dpad);
+  ALLOC0(h->m, (size_t)K * dpad);
+  if (need_D) ALLOC0(h->D, (size_t)K * dpad);
+  ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
+  ALLOC0(h->words_srv, sign ? nwords : 0);
+  ALLOC0(h->mask_srv, topk ? nwords : 0);
+  ALLOC0(h->scale[0], KT); ALLOC0(h->scale[1], KT); ALLOC0(h->scale_srv, T);
+  ALLOC0(h->tau[0], KT); ALLOC0(h->tau[1], KT); ALLOC0(h->tau_srv, T);
+  ALLOC0(h->recs, sign ? KT : 0); ALLOC0(h->recs_srv, sign ? T : 0);
+  ALLOC0(h->hist, topk ? KT * HIST_BINS : 0);
+  ALLOC0(h->sel, topk ? KT : 0);
+  ALLOC0(h->status, 1);
+  TRY(cudaMallocHost((void**)&h->status_host, sizeof(u32)));
+  TRY(cudaMemcpyAsync(h->d_tile_tensor, tile_tensor.data(), sizeof(int) * ntiles, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_first_tile, first_tile.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_n, n32.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_off, off.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_poff, poff.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
+#undef ALLOC0
+  if (rc == SAE_OK) {
+    Plan& P = h->P;
+    P.K = K; P.T = T; P.ntiles = (int)ntiles; P.d = d; P.dpad = dpad; P.nwords = nwords;
+    P.tile_tensor = h->d_tile_tensor; P.first_tile = h->d_first_tile; P.n = h->d_n; P.off = h->d_off; P.poff = h->d_poff;
+    LAUNCH(h, S_IMPORT, k_import, P.ntiles, P, x0, h->x);
+    TRY(cudaGetLastError());
+    TRY(cudaStreamSynchronize(h->stream));     // host tables above go out of scope
+  }
+#undef TRY
+  if (rc != SAE_OK) { free_all(h); delete h; return rc; }
+  // Pre-step of iteration 0: all errors are zero, so averaging (if (0+1) mod p = 0) changes nothing.
+  *out = h;
+  return SAE_OK;
+}
+
+int sae_step(sae_handle* h, const float* grads, float lr) {
+  if (!h || !grads || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  return do_step(h, grads, lr);
+}
+
+int sae_step_host(sae_handle* h, const float* grads_host, float lr) {
+  if (!h || !grads_host || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  const size_t count = (size_t)h->P.K * (size_t)h->P.d;
+  if (!h->staging) SAE_CUDA(h, dalloc(&h->staging, count));
+  SAE_CUDA(h, cudaMemcpyAsync(h->staging, grads_host, count * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+  return do_step(h, h->staging, lr);
+}
+
+int sae_get_params(sae_handle* h, float* out) {
+  if (!h || !out) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  return export_vec(h, EXP_X, 0, out);
+}
+
+int sae_get_params_host(sae_handle* h, float* out_host) {
+  if (!h || !out_host) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  // Export into a library-owned caller-layout buffer (allocated by the first call), then one
+  // contiguous device-to-host copy.
+  if (!h->out_stage) SAE_CUDA(h, dalloc(&h->out_stage, (size_t)h->P.d));
+  int rc = export_vec(h, EXP_X, 0, h->out_stage);
+  if (rc != SAE_OK) return rc;
+  SAE_CUDA(h, cudaMemcpyAsync(out_host, h->out_stage, sizeof(float) * h->P.d, cudaMemcpyDeviceToHost, h->stream));
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  return SAE_OK;
+}
+
+int sae_get_step_ahead(sae_handle* h, int32_t worker, float* out) {
+  if (!h || !out || worker < 0 || worker >= h->P.K) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  return export_vec(h, EXP_STEP_AHEAD, worker, out);
+}
+
+int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_t bytes) {
+  if (!h || !out) return SAE_ERR_INVALID_ARG;
+  const Plan& P = h->P;
+  const bool per_worker = which == SAE_STATE_MOMENTUM || which == SAE_STATE_WORKER_ERROR ||
+                          which == SAE_STATE_WORKER_SCALES || which == SAE_STATE_WORKER_WORDS ||
+                          which == SAE_STATE_WORKER_TAU || which == SAE_STATE_WORKER_MASK;
+  if (per_worker && (worker < 0 || worker >= P.K)) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  const bool sign = h->cfg.compressor == SAE_COMPRESSOR_SIGN, topk = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
+  const size_t vec = sizeof(float) * (size_t)P.d, tb = sizeof(float) * (size_t)P.T, wb = sizeof(u32) * (size_t)P.nwords;
+  const void* src = nullptr; size_t need = 0;
+  switch (which) {
+    case SAE_STATE_MOMENTUM: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_M, worker, (float*)out);
+    case SAE_STATE_WORKER_ERROR: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_WERR, worker, (float*)out);
+    case SAE_STATE_SERVER_ERROR: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_ESRV, 0, (float*)out);
+    case SAE_STATE_WORKER_SCALES: if (!sign) return SAE_ERR_INVALID_ARG; src = h->scale[h->last] + (size_t)worker * P.T; need = tb; break;
+    case SAE_STATE_SERVER_SCALES: if (!sign) return SAE_ERR_INVALID_ARG; src = h->scale_srv; need = tb; break;
+    case SAE_STATE_WORKER_WORDS: if (!sign) return SAE_ERR_INVALID_ARG; src = h->words + (size_t)worker * P.nwords; need = wb; break;
+    case SAE_STATE_SERVER_WORDS: if (!sign) return SAE_ERR_INVALID_ARG; src = h->words_srv; need = wb; break;
+    case SAE_STATE_WORKER_TAU: if (!topk) return SAE_ERR_INVALID_ARG; src = h->tau[h->last] + (size_t)worker * P.T; need = tb; break;
+    case SAE_STATE_SERVER_TAU: if (!topk) return SAE_ERR_INVALID_ARG; src = h->tau_srv; need = tb; break;
+    case SAE_STATE_SERVER_MASK: if (!topk) return SAE_ERR_INVALID_ARG; src = h->mask_srv; need = wb; break;
+    case SAE_STATE_WORKER_MASK:
+      if (!topk || bytes < wb) return SAE_ERR_INVALID_ARG;
+      LAUNCH(h, S_MASK, k_mask_words, P.ntiles, P, h->D + (size_t)worker * P.dpad, h->tau[h->last] + (size_t)worker * P.T,
+             (u32*)out);
+      return check_launch(h);
+    default: return SAE_ERR_INVALID_ARG;
+  }
+  if (bytes < need) return SAE_ERR_INVALID_ARG;
+  SAE_CUDA(h, cudaMemcpyAsync(out, src, need, cudaMemcpyDeviceToDevice, h->stream));
+  return SAE_OK;
+}
+
+int64_t sae_iteration(const sae_handle* h) { return h ? h->t : -1; }
+int64_t sae_num_params(const sae_handle* h) { return h ? h->P.d : -1; }
+int64_t sae_num_words(const sae_handle* h) { return h ? h->P.nwords : -1; }
+
+int sae_sync(sae_handle* h) {
+  if (!h) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  SAE_CUDA(h, cudaMemcpyAsync(h->status_host, h->status, sizeof(u32), cudaMemcpyDeviceToHost, h->stream));
+  SAE_CUDA(h, cudaMemsetAsync(h->status, 0, sizeof(u32), h->stream));
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  const u32 st = *h->status_host;
+  if (st & STATUS_RANGE) return SAE_ERR_RANGE;
+  return SAE_OK;
+}
+
+int sae_set_profiling(sae_handle* h, int32_t enabled) {
+  if (!h) return SAE_ERR_INVALID_ARG;
+  h->profiling = enabled ? 1 : 0;
+  return SAE_OK;
+}
+
+int sae_get_kernel_times(sae_handle* h, float* ms_host, int64_t* launches_host) {
+  if (!h || !ms_host || !launches_host) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  for (auto& ep : h->pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ep.a, ep.b) == cudaSuccess) { h->ms[ep.slot] += ms; h->cnt[ep.slot] += 1; }
+    h->pool.push_back(ep.a); h->pool.push_back(ep.b);
+  }
+  h->pending.clear();
+  for (int i = 0; i < SAE_NUM_KERNELS; ++i) {
+    ms_host[i] = (float)h->ms[i]; launches_host[i] = h->cnt[i];
+    h->ms[i] = 0; h->cnt[i] = 0;
+  }
+  return SAE_OK;
+}
+
+const char* sae_kernel_name(int32_t slot) {
+  if (slot < 0 || slot >= SAE_NUM_KERNELS) return "";
+  return kSlotNames[slot];
+}
+
+int64_t sae_kernel_launches(const sae_handle* h) { return h ? h->launches : -1; }
+
+void sae_destroy(sae_handle* h) {
+  if (!h) return;
+  DeviceGuard guard(h->device);
+  if (guard.ok) cudaStreamSynchronize(h->stream);
+  free_all(h);
+  delete h;
+}
+
+const char* sae_strerror(int status) {
+  switch (status) {
+    case SAE_OK: return "ok";
+    case SAE_ERR_INVALID_ARG: return "invalid argument";
+    case SAE_ERR_NOMEM: return "out of memory";
+    case SAE_ERR_CUDA: return "CUDA runtime error";
+    case SAE_ERR_RANGE: return "model difference non-finite or out of range (|v| >= 2^32)";
+    case SAE_ERR_TIMEOUT: return "device wait timed out";
+    case SAE_ERR_ABI: return "ABI version mismatch";
+    default: return "unknown status";
+  }
+}
+
+int sae_last_cuda_error(const sae_handle* h) { return h ? h->last_cuda_error : g_init_cuda_error; }
+
+}  // extern "C"

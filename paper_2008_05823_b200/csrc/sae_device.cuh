@@ -1,0 +1,197 @@
+// Device-side helpers shared by the kernels of libsae: tile plan, pinned fp32 arithmetic, the exact
+// fixed-point L1 accumulator of the scaled-sign compressor (Eq. 2) and Top-K magnitude keys.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sae {
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+
+constexpr int TILE = 4096;       // elements of one tensor handled by one thread block
+constexpr int THREADS = 256;     // threads per block: 8 warps
+constexpr int VEC_ITERS = TILE / (THREADS * 4);   // float4 iterations per thread (4)
+constexpr int ROWS = TILE / THREADS;              // scalar elements per thread (16)
+constexpr int MAX_WORKERS = 1024;
+
+constexpr u32 STATUS_RANGE = 1u;  // a model difference was non-finite or >= 2^32 in magnitude
+
+// Segment / tile tables (device memory), passed to kernels by value.
+// Internal ("padded") layout: tensor j starts at poff[j], a multiple of 32 elements, so that every
+// tensor start is 128-byte aligned and owns whole bit words; padding elements stay zero.
+struct Plan {
+  int K, T;
+  int ntiles;            // tiles over all tensors
+  long long d;           // sum n_j (caller layout length)
+  long long dpad;        // padded length, multiple of 32
+  long long nwords;      // dpad / 32 = sum ceil(n_j/32)
+  const int* tile_tensor;     // [ntiles] tensor of each tile
+  const int* first_tile;      // [T] first tile of each tensor
+  const int* n;               // [T] tensor sizes
+  const long long* off;       // [T] caller-layout offsets
+  const long long* poff;      // [T] padded offsets
+};
+
+struct TileInfo {
+  int j;            // tensor
+  int t0;           // first element of the tile inside the tensor
+  int n;            // tensor size
+  int cnt;          // valid elements in this tile (1..TILE)
+  int tiles_j;      // number of tiles of this tensor
+  long long off, poff;
+};
+
+__device__ __forceinline__ TileInfo tile_info(const Plan& P, int tile) {
+  TileInfo ti;
+  ti.j = P.tile_tensor[tile];
+  ti.n = P.n[ti.j];
+  ti.t0 = (tile - P.first_tile[ti.j]) * TILE;
+  ti.cnt = min(TILE, ti.n - ti.t0);
+  ti.tiles_j = (ti.n + TILE - 1) / TILE;
+  ti.off = P.off[ti.j];
+  ti.poff = P.poff[ti.j];
+  return ti;
+}
+
+// ---- streaming loads/stores ------------------------------------------------------------------------
+__device__ __forceinline__ float4 ld4_stream(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+
+// ---- the scaled-sign code of one element -------------------------------------------------------------
+__device__ __forceinline__ float sign_code(float v, float s) { return (v >= 0.0f) ? s : -s; }
+
+// ---- Top-K ---------------------------------------------------------------------------------------
+__device__ __forceinline__ u32 mag_key(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+__device__ __forceinline__ bool topk_selected(float v, u32 tau) {
+  u32 key = mag_key(v);
+  return key >= tau && key != 0u;
+}
+
+// ---- exact L1: S = sum floor(|v| 2^64) as a 128-bit integer ----------------------------------------
+struct Acc128 {
+  u64 lo, hi;
+  u32 bad;
+};
+
+__device__ __forceinline__ void acc_init(Acc128& a) { a.lo = 0; a.hi = 0; a.bad = 0; }
+
+__device__ __forceinline__ void acc_add_u(Acc128& a, u64 lo, u64 hi) {
+  a.lo += lo;
+  a.hi += hi + (a.lo < lo ? 1ull : 0ull);
+}
+
+// |v| < 1: |v| * 2^64 is exact in fp32 (a power-of-two scaling that can neither overflow nor lose
+// bits; denormals become normal) and the round-down conversion is the floor.  1 <= |v| < 2^32: integer
+// part and fraction are split exactly first.  Anything else (including NaN/Inf) flags RANGE.
+__device__ __forceinline__ void acc_add(Acc128& a, float v) {
+  float m = fabsf(v);
+  if (m < 1.0f) {
+    u64 f = __float2ull_rd(__fmul_rn(m, 18446744073709551616.0f));
+    a.lo += f;
+    a.hi += (a.lo < f ? 1ull : 0ull);
+  } else if (m < 4294967296.0f) {
+    float ip = floorf(m);
+    float fr = __fsub_rn(m, ip);
+    acc_add_u(a, __float2ull_rd(__fmul_rn(fr, 18446744073709551616.0f)), __float2ull_rd(ip));
+  } else {
+    a.bad = 1u;
+  }
+}
+
+__device__ __forceinline__ void acc_warp_reduce(Acc128& a) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    u64 lo = __shfl_xor_sync(0xffffffffu, a.lo, o);
+    u64 hi = __shfl_xor_sync(0xffffffffu, a.hi, o);
+    u32 bad = __shfl_xor_sync(0xffffffffu, a.bad, o);
+    acc_add_u(a, lo, hi);
+    a.bad |= bad;
+  }
+}
+
+// Block reduction; the result is valid in thread 0.  `sh` must hold 3 * (THREADS/32) u64.
+__device__ __forceinline__ void acc_block_reduce(Acc128& a, u64* sh) {
+  acc_warp_reduce(a);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int NW = THREADS / 32;
+  if (lane == 0) { sh[warp] = a.lo; sh[NW + warp] = a.hi; sh[2 * NW + warp] = a.bad; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    Acc128 r; acc_init(r);
+    for (int w = 0; w < NW; ++w) { acc_add_u(r, sh[w], sh[NW + w]); r.bad |= (u32)sh[2 * NW + w]; }
+    a = r;
+  }
+}
+
+// The per-(row, tensor) accumulator in global memory: three 43-bit limbs in 64-bit words (21 bits of
+// headroom each, so integer atomicAdd from up to 2^21 tiles cannot overflow and the total does not
+// depend on the order of arrival) and an arrival counter.  The block that arrives last finalises the
+// scale and resets the record for the next step.
+struct L1Record {
+  u64 limb[3];
+  u32 count;
+  u32 pad;
+};
+
+constexpr u64 M43 = (1ull << 43) - 1;
+
+// scale = (float)((double)(S truncated to its top 53 bits) / n * 2^-64)
+__device__ __forceinline__ float scale_from_limbs(u64 l0, u64 l1, u64 l2, int n) {
+  Acc128 s; acc_init(s);
+  s.lo = l0;
+  acc_add_u(s, l1 << 43, l1 >> 21);
+  acc_add_u(s, 0ull, l2 << 22);
+  if (s.lo == 0 && s.hi == 0) return 0.0f;
+  int p = s.hi ? 127 - __clzll((long long)s.hi) : 63 - __clzll((long long)s.lo);
+  u64 mant; int sh = 0;
+  if (p > 52) {
+    sh = p - 52;
+    mant = (sh >= 64) ? (s.hi >> (sh - 64)) : ((s.lo >> sh) | (s.hi << (64 - sh)));   // sh in 1..75
+  } else {
+    mant = s.lo;
+  }
+  double Dd = ldexp((double)mant, sh);                  // exact: mant < 2^53
+  double q = __ddiv_rn(Dd, (double)n);
+  return __double2float_rn(q * 5.421010862427522e-20);  // 2^-64, exact scaling
+}
+
+// Called by thread 0 of a block with that block's partial sum.  Returns true in the block that arrived
+// last for this record and then writes the finished scale.
+__device__ __forceinline__ void l1_commit(const Acc128& a, L1Record* rec, int tiles, int n, float* scale_out,
+                                          u32* status) {
+  if (a.bad) atomicOr(status, STATUS_RANGE);
+  u64 l0 = a.lo & M43;
+  u64 l1 = ((a.lo >> 43) | (a.hi << 21)) & M43;
+  u64 l2 = a.hi >> 22;
+  if (l0) atomicAdd(&rec->limb[0], l0);
+  if (l1) atomicAdd(&rec->limb[1], l1);
+  if (l2) atomicAdd(&rec->limb[2], l2);
+  __threadfence();
+  u32 ticket = atomicAdd(&rec->count, 1u);
+  if (ticket == (u32)tiles - 1u) {
+    __threadfence();
+    u64 r0 = atomicExch(&rec->limb[0], 0ull);
+    u64 r1 = atomicExch(&rec->limb[1], 0ull);
+    u64 r2 = atomicExch(&rec->limb[2], 0ull);
+    atomicExch(&rec->count, 0u);
+    *scale_out = scale_from_limbs(r0, r1, r2, n);
+  }
+}
+
+// ---- sign bits -----------------------------------------------------------------------------------
+// Four consecutive elements per lane (lane l holds elements 4l..4l+3 of a 128-element row): the four
+// words of the row are assembled by OR-ing nibbles across each group of 8 lanes.  Every lane of group
+// g ends up holding word g.
+__device__ __forceinline__ u32 pack_row4(bool p0, bool p1, bool p2, bool p3) {
+  int lane = threadIdx.x & 31;
+  u32 nib = (p0 ? 1u : 0u) | (p1 ? 2u : 0u) | (p2 ? 4u : 0u) | (p3 ? 8u : 0u);
+  u32 w = nib << (4 * (lane & 7));
+  w |= __shfl_xor_sync(0xffffffffu, w, 1);
+  w |= __shfl_xor_sync(0xffffffffu, w, 2);
+  w |= __shfl_xor_sync(0xffffffffu, w, 4);
+  return w;
+}
+
+}  // namespace sae

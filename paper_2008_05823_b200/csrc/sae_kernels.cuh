@@ -1,0 +1,563 @@
+// Kernels of one iteration of Algorithm 1.  One thread block handles one tile (TILE consecutive
+// elements of one tensor), for one worker in the worker pass, for all workers in the server passes.
+// Full tiles whose gradient pointer is 16-byte aligned take a 128-bit vector path; ragged tails and
+// misaligned gradient rows take a lane-strided scalar path.  Both produce identical bits.
+#pragma once
+#include "sae_device.cuh"
+
+namespace sae {
+
+struct StepParams {
+  float mu, eta, lambda;
+  int saef;   // 1: gradient point is x - e^(k), 0: x
+  int wd;     // lambda != 0
+};
+
+// where the previous local error e_t^(k) comes from
+constexpr int ESRC_UNIFORM = 0;    // e^(k) = ebar for all k (after an averaging pre-step, or at t = 0)
+constexpr int ESRC_LAZY_SIGN = 1;  // e^(k) = D^(k) - C(D^(k)) with last step's scales, D^(k) = last Delta^(k)
+constexpr int ESRC_LAZY_TOPK = 2;  // same with last step's Top-K thresholds
+
+template <int ESRC>
+__device__ __forceinline__ float prev_error(float v, float sprev, u32 tprev) {
+  if (ESRC == ESRC_UNIFORM) return v;
+  if (ESRC == ESRC_LAZY_SIGN) return __fsub_rn(v, sign_code(v, sprev));
+  return __fsub_rn(v, topk_selected(v, tprev) ? v : 0.0f);
+}
+
+// Algorithm 1, worker lines: step-ahead point, local momentum, local model difference.
+__device__ __forceinline__ float worker_update(float g, float mo, float e, float x, const StepParams& sp,
+                                               float& mn) {
+  float ge = g;
+  if (sp.wd) {
+    float xh = sp.saef ? __fsub_rn(x, e) : x;
+    ge = __fmaf_rn(sp.lambda, xh, g);
+  }
+  mn = __fmaf_rn(sp.mu, mo, ge);
+  return __fmaf_rn(sp.eta, mn, e);
+}
+
+struct WorkerArgs {
+  const float* g;         // [K][d] caller layout
+  float* m;               // [K][dpad]
+  float* D;               // [K][dpad] last model difference (read when lazy, written when WRITE_D)
+  const float* ebar;      // [dpad]
+  const float* x;         // [dpad]
+  const float* scale_prev;  // [K][T]
+  const u32* tau_prev;      // [K][T]
+  u32* words;             // [K][nwords]
+  float* scale_cur;       // [K][T]
+  L1Record* recs;         // [K][T]
+  u32* status;
+};
+
+// K1: worker pass.  grid = ntiles * K, block (tile, k) with k fastest so that the K blocks sharing one
+// tile of ebar / x run close together.
+template <int ESRC, bool SIGN, bool WRITE_D>
+__global__ void __launch_bounds__(THREADS) k_worker(Plan P, StepParams sp, WorkerArgs A) {
+  __shared__ u64 sh_red[3 * (THREADS / 32)];
+  const int tile = blockIdx.x / P.K;
+  const int k = blockIdx.x - tile * P.K;
+  const TileInfo ti = tile_info(P, tile);
+  const float* __restrict__ gp = A.g + (long long)k * P.d + ti.off + ti.t0;
+  const long long pbase = ti.poff + ti.t0;
+  const long long wbase = (long long)k * P.dpad + pbase;
+  float* __restrict__ mp = A.m + wbase;
+  float* dp = A.D + wbase;
+  const float* __restrict__ ebp = A.ebar + pbase;
+  const float* __restrict__ xp = A.x + pbase;
+  u32* wp = A.words + (long long)k * P.nwords + (pbase >> 5);
+  const float sprev = (ESRC == ESRC_LAZY_SIGN) ? A.scale_prev[(long long)k * P.T + ti.j] : 0.0f;
+  const u32 tprev = (ESRC == ESRC_LAZY_TOPK) ? A.tau_prev[(long long)k * P.T + ti.j] : 0u;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  Acc128 acc; acc_init(acc);
+
+  const bool vec = (ti.cnt == TILE) && ((reinterpret_cast<uintptr_t>(gp) & 15) == 0);
+  if (vec) {
+    float4 G[VEC_ITERS], M[VEC_ITERS], E[VEC_ITERS], X[VEC_ITERS];
+#pragma unroll
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      G[it] = ld4_stream(gp + i);
+      M[it] = ld4(mp + i);
+      E[it] = (ESRC == ESRC_UNIFORM) ? ld4(ebp + i) : ld4(dp + i);
+      if (sp.wd) X[it] = ld4(xp + i); else X[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      float4 mn, dl;
+      dl.x = worker_update(G[it].x, M[it].x, prev_error<ESRC>(E[it].x, sprev, tprev), X[it].x, sp, mn.x);
+      dl.y = worker_update(G[it].y, M[it].y, prev_error<ESRC>(E[it].y, sprev, tprev), X[it].y, sp, mn.y);
+      dl.z = worker_update(G[it].z, M[it].z, prev_error<ESRC>(E[it].z, sprev, tprev), X[it].z, sp, mn.z);
+      dl.w = worker_update(G[it].w, M[it].w, prev_error<ESRC>(E[it].w, sprev, tprev), X[it].w, sp, mn.w);
+      st4(mp + i, mn);
+      if (WRITE_D) st4(dp + i, dl);
+      if (SIGN) {
+        acc_add(acc, dl.x); acc_add(acc, dl.y); acc_add(acc, dl.z); acc_add(acc, dl.w);
+        u32 w = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
+        if ((lane & 7) == 0) wp[(i >> 5)] = w;
+      }
+    }
+  } else {
+#pragma unroll 4
+    for (int r = 0; r < ROWS; ++r) {
+      const int i = r * THREADS + tid;
+      const bool valid = i < ti.cnt;
+      float dl = 0.0f;
+      if (valid) {
+        float e = prev_error<ESRC>((ESRC == ESRC_UNIFORM) ? ebp[i] : dp[i], sprev, tprev);
+        float xv = sp.wd ? xp[i] : 0.0f;
+        float mn;
+        dl = worker_update(__ldcs(gp + i), mp[i], e, xv, sp, mn);
+        mp[i] = mn;
+        if (WRITE_D) dp[i] = dl;
+        if (SIGN) acc_add(acc, dl);
+      }
+      if (SIGN) {
+        u32 w = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
+        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wp[(r * THREADS + warp * 32) >> 5] = w;
+      }
+    }
+  }
+  if (SIGN) {
+    acc_block_reduce(acc, sh_red);
+    if (tid == 0)
+      l1_commit(acc, A.recs + (long long)k * P.T + ti.j, ti.tiles_j, ti.n,
+                A.scale_cur + (long long)k * P.T + ti.j, A.status);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+struct ServerArgs {
+  float* e_srv;            // [dpad]: in: server error e_t, out: server model difference Delta_{t+1}
+  const u32* words;        // [K][nwords] worker sign words
+  const float* scale_cur;  // [K][T] worker scales of this step
+  const float* D;          // [K][dpad] (dense variants)
+  const u32* tau_cur;      // [K][T] (Top-K)
+  u32* words_srv;          // [nwords]
+  float* scale_srv;        // [T]
+  L1Record* recs_srv;      // [T]
+  u32* status;
+};
+
+// K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
+// compression also the server's L1 partials and sign words.  grid = ntiles.
+template <bool DC>
+__global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
+  __shared__ u64 sh_red[3 * (THREADS / 32)];
+  __shared__ float s_k[MAX_WORKERS];
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int k = tid; k < P.K; k += THREADS) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
+  __syncthreads();
+  const long long pbase = ti.poff + ti.t0;
+  float* ep = A.e_srv + pbase;
+  const u32* __restrict__ wp = A.words + (pbase >> 5);
+  u32* wsp = A.words_srv + (pbase >> 5);
+  const float Kf = (float)P.K;
+  Acc128 acc; acc_init(acc);
+
+  if (ti.cnt == TILE) {
+#pragma unroll 2
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      const float4 e = ld4(ep + i);
+      const int wi = i >> 5, sh = i & 31;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 8
+      for (int k = 0; k < P.K; ++k) {
+        const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> sh;
+        const float s = s_k[k];
+        a0 = __fadd_rn(a0, (w & 1u) ? s : -s);
+        a1 = __fadd_rn(a1, (w & 2u) ? s : -s);
+        a2 = __fadd_rn(a2, (w & 4u) ? s : -s);
+        a3 = __fadd_rn(a3, (w & 8u) ? s : -s);
+      }
+      float4 ds;
+      ds.x = __fadd_rn(e.x, __fdiv_rn(a0, Kf));
+      ds.y = __fadd_rn(e.y, __fdiv_rn(a1, Kf));
+      ds.z = __fadd_rn(e.z, __fdiv_rn(a2, Kf));
+      ds.w = __fadd_rn(e.w, __fdiv_rn(a3, Kf));
+      st4(ep + i, ds);
+      if (DC) {
+        acc_add(acc, ds.x); acc_add(acc, ds.y); acc_add(acc, ds.z); acc_add(acc, ds.w);
+        u32 w = pack_row4(ds.x >= 0.0f, ds.y >= 0.0f, ds.z >= 0.0f, ds.w >= 0.0f);
+        if ((lane & 7) == 0) wsp[wi] = w;
+      }
+    }
+  } else {
+    for (int r = 0; r < ROWS; ++r) {
+      const int i = r * THREADS + tid;
+      const bool valid = i < ti.cnt;
+      float ds = 0.0f;
+      if (valid) {
+        float a = 0.f;
+        const int wi = i >> 5;
+        for (int k = 0; k < P.K; ++k) {
+          const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> lane;
+          const float s = s_k[k];
+          a = __fadd_rn(a, (w & 1u) ? s : -s);
+        }
+        ds = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+        ep[i] = ds;
+        if (DC) acc_add(acc, ds);
+      }
+      if (DC) {
+        u32 w = __ballot_sync(0xffffffffu, valid && ds >= 0.0f);
+        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wsp[(r * THREADS + warp * 32) >> 5] = w;
+      }
+    }
+  }
+  if (DC) {
+    acc_block_reduce(acc, sh_red);
+    if (tid == 0) l1_commit(acc, A.recs_srv + ti.j, ti.tiles_j, ti.n, A.scale_srv + ti.j, A.status);
+  }
+}
+
+// K3 (identity / Top-K): the same aggregation from the dense model differences.
+// COMP 0: C = identity, 2: Top-K with this step's thresholds.
+template <int COMP>
+__global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
+  __shared__ u32 t_k[MAX_WORKERS];
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const int tid = threadIdx.x;
+  if (COMP == 2) {
+    for (int k = tid; k < P.K; k += THREADS) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
+    __syncthreads();
+  }
+  const long long pbase = ti.poff + ti.t0;
+  float* ep = A.e_srv + pbase;
+  const float* __restrict__ dp = A.D + pbase;
+  const float Kf = (float)P.K;
+  if (ti.cnt == TILE) {
+#pragma unroll 2
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      const float4 e = ld4(ep + i);
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+      for (int k = 0; k < P.K; ++k) {
+        const float4 v = ld4(dp + (long long)k * P.dpad + i);
+        const u32 t = (COMP == 2) ? t_k[k] : 0u;
+        a0 = __fadd_rn(a0, (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f);
+        a1 = __fadd_rn(a1, (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f);
+        a2 = __fadd_rn(a2, (COMP == 0 || topk_selected(v.z, t)) ? v.z : 0.0f);
+        a3 = __fadd_rn(a3, (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f);
+      }
+      float4 ds;
+      ds.x = __fadd_rn(e.x, __fdiv_rn(a0, Kf));
+      ds.y = __fadd_rn(e.y, __fdiv_rn(a1, Kf));
+      ds.z = __fadd_rn(e.z, __fdiv_rn(a2, Kf));
+      ds.w = __fadd_rn(e.w, __fdiv_rn(a3, Kf));
+      st4(ep + i, ds);
+    }
+  } else {
+    for (int r = 0; r < ROWS; ++r) {
+      const int i = r * THREADS + tid;
+      if (i < ti.cnt) {
+        float a = 0.f;
+        for (int k = 0; k < P.K; ++k) {
+          const float v = dp[(long long)k * P.dpad + i];
+          a = __fadd_rn(a, (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f);
+        }
+        ep[i] = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+struct ApplyArgs {
+  float* e_srv;            // [dpad] in: Delta_{t+1}, out: e_{t+1}
+  float* x;                // [dpad]
+  float* ebar;             // [dpad] in: previous uniform error (recompute variant), out: averaged error
+  const float* m;          // [K][dpad]
+  const float* D;          // [K][dpad]
+  const float* scale_cur;  // [K][T]
+  const float* scale_srv;  // [T]
+  const u32* tau_cur;      // [K][T]
+  const u32* tau_srv;      // [T]
+  u32* mask_srv;           // [nwords] Top-K: server selection of this step
+  float eta;
+};
+
+constexpr int AVG_NONE = 0;
+constexpr int AVG_FROM_D = 1;        // e^(k) = D^(k) - C(D^(k)) from the stored model differences
+constexpr int AVG_RECOMPUTE = 2;     // D^(k) = fma(eta, m^(k), ebar) recomputed (previous error was uniform)
+
+// COMP: compressor of the workers; SRV: what the server applies (0 identity, 1 sign, 2 Top-K).
+template <int COMP, int SRV, int AVG>
+__device__ __forceinline__ void apply_elem(float ds, float& x, float& es, bool& sel_srv, float s_srv, u32 t_srv) {
+  float cs;
+  if (SRV == 1) cs = sign_code(ds, s_srv);
+  else if (SRV == 2) { sel_srv = topk_selected(ds, t_srv); cs = sel_srv ? ds : 0.0f; }
+  else cs = ds;
+  es = __fsub_rn(ds, cs);       // e_{t+1} = Delta - C(Delta)
+  x = __fsub_rn(x, cs);         // re-update x_{t+1} = x_t - C(Delta)
+}
+
+template <int COMP>
+__device__ __forceinline__ float worker_err(float dk, float s, u32 t) {
+  if (COMP == 1) return __fsub_rn(dk, sign_code(dk, s));
+  if (COMP == 2) return __fsub_rn(dk, topk_selected(dk, t) ? dk : 0.0f);
+  return __fsub_rn(dk, dk);
+}
+
+// K5: server error, re-update, and (when the next pre-step averages) the averaged worker error.
+template <int COMP, int SRV, int AVG>
+__global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
+  __shared__ float s_k[MAX_WORKERS];
+  __shared__ u32 t_k[MAX_WORKERS];
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (AVG != AVG_NONE) {
+    for (int k = tid; k < P.K; k += THREADS) {
+      if (COMP == 1) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
+      if (COMP == 2) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
+    }
+    __syncthreads();
+  }
+  const float s_srv = (SRV == 1) ? A.scale_srv[ti.j] : 0.0f;
+  const u32 t_srv = (SRV == 2) ? A.tau_srv[ti.j] : 0u;
+  const long long pbase = ti.poff + ti.t0;
+  float* ep = A.e_srv + pbase;
+  float* xp = A.x + pbase;
+  float* ebp = A.ebar + pbase;
+  const float* __restrict__ src = (AVG == AVG_RECOMPUTE) ? A.m + pbase : A.D + pbase;
+  u32* mwp = A.mask_srv + (pbase >> 5);
+  const float Kf = (float)P.K;
+
+  if (ti.cnt == TILE) {
+#pragma unroll 2
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      const float4 ds = ld4(ep + i);
+      float4 x = ld4(xp + i), es;
+      bool q0 = false, q1 = false, q2 = false, q3 = false;
+      apply_elem<COMP, SRV, AVG>(ds.x, x.x, es.x, q0, s_srv, t_srv);
+      apply_elem<COMP, SRV, AVG>(ds.y, x.y, es.y, q1, s_srv, t_srv);
+      apply_elem<COMP, SRV, AVG>(ds.z, x.z, es.z, q2, s_srv, t_srv);
+      apply_elem<COMP, SRV, AVG>(ds.w, x.w, es.w, q3, s_srv, t_srv);
+      st4(ep + i, es);
+      st4(xp + i, x);
+      if (SRV == 2) {
+        u32 w = pack_row4(q0, q1, q2, q3);
+        if ((lane & 7) == 0) mwp[i >> 5] = w;
+      }
+      if (AVG != AVG_NONE) {
+        float4 eb = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (AVG == AVG_RECOMPUTE) eb = ld4(ebp + i);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < P.K; ++k) {
+          float4 v = ld4_stream(src + (long long)k * P.dpad + i);
+          if (AVG == AVG_RECOMPUTE) {
+            v.x = __fmaf_rn(A.eta, v.x, eb.x); v.y = __fmaf_rn(A.eta, v.y, eb.y);
+            v.z = __fmaf_rn(A.eta, v.z, eb.z); v.w = __fmaf_rn(A.eta, v.w, eb.w);
+          }
+          const float s = (COMP == 1) ? s_k[k] : 0.0f;
+          const u32 t = (COMP == 2) ? t_k[k] : 0u;
+          a0 = __fadd_rn(a0, worker_err<COMP>(v.x, s, t));
+          a1 = __fadd_rn(a1, worker_err<COMP>(v.y, s, t));
+          a2 = __fadd_rn(a2, worker_err<COMP>(v.z, s, t));
+          a3 = __fadd_rn(a3, worker_err<COMP>(v.w, s, t));
+        }
+        st4(ebp + i, make_float4(__fdiv_rn(a0, Kf), __fdiv_rn(a1, Kf), __fdiv_rn(a2, Kf), __fdiv_rn(a3, Kf)));
+      }
+    }
+  } else {
+    for (int r = 0; r < ROWS; ++r) {
+      const int i = r * THREADS + tid;
+      const bool valid = i < ti.cnt;
+      bool q = false;
+      if (valid) {
+        float x = xp[i], es;
+        apply_elem<COMP, SRV, AVG>(ep[i], x, es, q, s_srv, t_srv);
+        ep[i] = es;
+        xp[i] = x;
+        if (AVG != AVG_NONE) {
+          const float eb = (AVG == AVG_RECOMPUTE) ? ebp[i] : 0.0f;
+          float a = 0.f;
+          for (int k = 0; k < P.K; ++k) {
+            float v = src[(long long)k * P.dpad + i];
+            if (AVG == AVG_RECOMPUTE) v = __fmaf_rn(A.eta, v, eb);
+            a = __fadd_rn(a, worker_err<COMP>(v, (COMP == 1) ? s_k[k] : 0.0f, (COMP == 2) ? t_k[k] : 0u));
+          }
+          ebp[i] = __fdiv_rn(a, Kf);
+        }
+      }
+      if (SRV == 2) {
+        u32 w = __ballot_sync(0xffffffffu, valid && q);
+        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) mwp[(r * THREADS + warp * 32) >> 5] = w;
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Top-K threshold: exact k-th largest 31-bit magnitude key per (row, tensor) by a three-level radix
+// select (11 + 10 + 10 bits).  Level L histograms the digit of every key whose higher digits equal the
+// prefix found so far; a select kernel then walks the histogram from the top.
+struct SelectState {     // per (row, tensor)
+  u32 prefix;            // digits found so far, right-aligned
+  u32 rank;              // rank (1-based, from the top) still to find inside the prefix bucket
+};
+
+constexpr int HIST_BINS = 2048;
+
+__device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* hist) {
+  if (level == 0) atomicAdd(hist + (key >> 20), 1u);
+  else if (level == 1) { if ((key >> 20) == prefix) atomicAdd(hist + ((key >> 10) & 1023u), 1u); }
+  else { if ((key >> 10) == prefix) atomicAdd(hist + (key & 1023u), 1u); }
+}
+
+// grid = ntiles * rows; buf is [rows][dpad]; hist is [rows][T][HIST_BINS]
+__global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, int rows, int level, const float* __restrict__ buf,
+                                                        const SelectState* __restrict__ st, u32* hist) {
+  __shared__ u32 sh[HIST_BINS];
+  const int tile = blockIdx.x / rows;
+  const int k = blockIdx.x - tile * rows;
+  const TileInfo ti = tile_info(P, tile);
+  const int tid = threadIdx.x;
+  const float* __restrict__ bp = buf + (long long)k * P.dpad + ti.poff + ti.t0;
+  u32* gh = hist + ((long long)k * P.T + ti.j) * HIST_BINS;
+  const u32 prefix = level ? st[(long long)k * P.T + ti.j].prefix : 0u;
+  if (level == 0) {
+    for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
+    __syncthreads();
+  }
+  u32* target = (level == 0) ? sh : gh;
+  if (ti.cnt == TILE) {
+#pragma unroll
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const float4 v = ld4(bp + it * (THREADS * 4) + tid * 4);
+      hist_elem(mag_key(v.x), level, prefix, target);
+      hist_elem(mag_key(v.y), level, prefix, target);
+      hist_elem(mag_key(v.z), level, prefix, target);
+      hist_elem(mag_key(v.w), level, prefix, target);
+    }
+  } else {
+    for (int i = tid; i < ti.cnt; i += THREADS) hist_elem(mag_key(bp[i]), level, prefix, target);
+  }
+  if (level == 0) {
+    __syncthreads();
+    for (int b = tid; b < HIST_BINS; b += THREADS) {
+      u32 c = sh[b];
+      if (c) atomicAdd(gh + b, c);
+    }
+  }
+}
+
+// One block per (row, tensor): find the bin holding the rank-th largest key, update prefix/rank, clear
+// the histogram.  After level 2 the prefix is the threshold key itself.
+__global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const int* __restrict__ n, u32 num, u32 den,
+                                                          u32* hist, SelectState* st, u32* tau) {
+  __shared__ u32 part[THREADS];
+  __shared__ u32 above[THREADS];
+  const int rj = blockIdx.x;              // row * T + j
+  const int j = rj % T;
+  const int tid = threadIdx.x;
+  const int bins = (level == 0) ? HIST_BINS : 1024;
+  const int per = bins / THREADS;         // 8 or 4
+  u32* gh = hist + (long long)rj * HIST_BINS;
+  u32 rank;
+  if (level == 0) {
+    unsigned long long kk = ((unsigned long long)n[j] * num) / den;
+    if (kk < 1) kk = 1;
+    if (kk > (unsigned long long)n[j]) kk = n[j];
+    rank = (u32)kk;
+  } else {
+    rank = st[rj].rank;
+  }
+  // thread t owns bins [hi - per*t - per + 1 .. hi - per*t] counted from the top
+  u32 c[8];
+  u32 sum = 0;
+  for (int q = 0; q < per; ++q) {
+    const int b = bins - 1 - (tid * per + q);
+    c[q] = gh[b];
+    gh[b] = 0u;
+    sum += c[q];
+  }
+  part[tid] = sum;
+  __syncthreads();
+  if (tid == 0) {
+    u32 run = 0;
+    for (int t = 0; t < THREADS; ++t) { above[t] = run; run += part[t]; }
+  }
+  __syncthreads();
+  u32 run = above[tid];
+  if (run < rank && rank <= run + sum) {
+    for (int q = 0; q < per; ++q) {
+      if (rank <= run + c[q]) {
+        const u32 b = (u32)(bins - 1 - (tid * per + q));
+        const u32 prefix = (level == 0) ? b : ((st[rj].prefix << 10) | b);
+        st[rj].prefix = prefix;
+        st[rj].rank = rank - run;
+        if (level == 2) tau[rj] = prefix;
+        break;
+      }
+      run += c[q];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Layout conversion and getters (not on the hot path).
+constexpr int EXP_X = 0, EXP_ESRV = 1, EXP_M = 2, EXP_WERR = 3, EXP_STEP_AHEAD = 4;
+
+struct ExportArgs {
+  const float* x; const float* e_srv; const float* m; const float* D; const float* ebar;
+  const float* scale_last; const u32* tau_last;
+  int esrc;      // ESRC_* describing how e^(k) is currently held
+  int what;      // EXP_*
+  int k;
+  int saef;
+};
+
+__device__ __forceinline__ float current_error(const ExportArgs& A, const Plan& P, int j, long long p) {
+  if (A.esrc == ESRC_UNIFORM) return A.ebar[p];
+  const float v = A.D[(long long)A.k * P.dpad + p];
+  if (A.esrc == ESRC_LAZY_SIGN) return prev_error<ESRC_LAZY_SIGN>(v, A.scale_last[(long long)A.k * P.T + j], 0u);
+  return prev_error<ESRC_LAZY_TOPK>(v, 0.0f, A.tau_last[(long long)A.k * P.T + j]);
+}
+
+__global__ void __launch_bounds__(THREADS) k_export(Plan P, ExportArgs A, float* __restrict__ out) {
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  for (int i = threadIdx.x; i < ti.cnt; i += THREADS) {
+    const long long p = ti.poff + ti.t0 + i;
+    float v;
+    switch (A.what) {
+      case EXP_X: v = A.x[p]; break;
+      case EXP_ESRV: v = A.e_srv[p]; break;
+      case EXP_M: v = A.m[(long long)A.k * P.dpad + p]; break;
+      case EXP_WERR: v = current_error(A, P, ti.j, p); break;
+      default: v = A.saef ? __fsub_rn(A.x[p], current_error(A, P, ti.j, p)) : A.x[p]; break;
+    }
+    out[ti.off + ti.t0 + i] = v;
+  }
+}
+
+// caller layout -> padded layout
+__global__ void __launch_bounds__(THREADS) k_import(Plan P, const float* __restrict__ in, float* __restrict__ out) {
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  for (int i = threadIdx.x; i < ti.cnt; i += THREADS) out[ti.poff + ti.t0 + i] = in[ti.off + ti.t0 + i];
+}
+
+// Top-K selection of row k of buf as bit words
+__global__ void __launch_bounds__(THREADS) k_mask_words(Plan P, const float* __restrict__ buf,
+                                                         const u32* __restrict__ tau, u32* __restrict__ out) {
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 t = tau[ti.j];
+  const long long pbase = ti.poff + ti.t0;
+  for (int r = 0; r < ROWS; ++r) {
+    const int i = r * THREADS + tid;
+    const bool valid = i < ti.cnt;
+    const bool q = valid && topk_selected(buf[pbase + i], t);
+    u32 w = __ballot_sync(0xffffffffu, q);
+    if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) out[(pbase + r * THREADS + warp * 32) >> 5] = w;
+  }
+}
+
+}  // namespace sae

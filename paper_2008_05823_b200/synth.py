@@ -169,3 +169,18 @@ class DeviceGenerator:
 
     def x0(self, out, seed):
         return self._fill(out, 1, seed, T_X0, self.ones, 0, 1.0, 0.05)
+
+
+def grads_numpy_range(seed, t, k, i0, count, scale, outlier_per_65536=0, outlier_mult=1.0):
+    """Gradient entries i0 .. i0+count-1 (flat caller-layout indices, all inside one tensor of scale
+    `scale`) of worker k at iteration t: lets a test reproduce single tensors of a large workload."""
+    z, lane12 = _unit_normal_and_lane12(stream_key(seed, t, k), i0, count)
+    g = np.float32(scale) * z
+    if outlier_per_65536 > 0:
+        g = np.where(lane12 < outlier_per_65536, g * np.float32(outlier_mult), g).astype(np.float32)
+    return g
+
+
+def x0_numpy_range(seed, i0, count):
+    z, _ = _unit_normal_and_lane12(stream_key(seed, T_X0, 0), i0, count)
+    return np.float32(0.05) * z

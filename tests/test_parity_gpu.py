@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle on the same seeded inputs,
+element by element, after every step.  Sign words, Top-K thresholds and index sets must be bit-exact;
+floats are held to the stated 1e-5 relative bar (and are expected to be bit-identical)."""
+import numpy as np
+import pytest
+
+from oracle import sae_oracle as so
+from paper_2008_05823_b200 import binding as sb
+from paper_2008_05823_b200 import configs, synth
+from parity_util import compare_state, compare_server_messages, assert_same
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [1, 2, 31, 32, 33, 1000, 4097, 4096, 5000, 8192 + 5, 3 * 4096]
+
+
+def run_pair(K, sizes, comp, steps, seed=0, p=0, dc=1, mode=so.SAEF, mu=0.9, lam=0.0, num=1, den=100, lrs=None,
+             scale=1e-2, outliers=(0, 1.0), every=1):
+    import torch
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(seed, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(seed, d)
+    orc = so.Oracle(K, sizes, x0, compressor=comp, server_compress=dc, mode=mode, avg_period=p, momentum=mu,
+                    weight_decay=lam, topk_num=num, topk_den=den, threads=4)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=comp, server_compress=dc, mode=mode, avg_period=p,
+                 momentum=mu, weight_decay=lam, topk_num=num, topk_den=den)
+    compare_state(gpu, orc, comp, tag="t=0")
+    for t in range(steps):
+        g = synth.grads_numpy(seed, t, K, sizes, scales, outliers[0], outliers[1])
+        lr = 0.1 if lrs is None else lrs[t % len(lrs)]
+        orc.step(g, lr)
+        gpu.step(torch.from_numpy(g).cuda(), lr)
+        if (t + 1) % every == 0 or t == steps - 1:
+            tag = f"K={K} comp={comp} p={p} dc={dc} mode={mode} t={t + 1}"
+            compare_state(gpu, orc, comp, tag=tag)
+            compare_server_messages(gpu, orc, comp, dc, tag=tag)
+    assert not orc.range_flag
+    gpu.close()
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4])
+@pytest.mark.parametrize("p", [0, 1, 3])
+def test_sign_ragged(K, p):
+    run_pair(K, RAGGED, so.SIGN, 7, p=p, lrs=[0.1, 0.05, 0.2])
+
+
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("mode", [so.EF, so.SAEF])
+@pytest.mark.parametrize("mu,lam", [(0.0, 0.0), (0.9, 1e-4), (0.5, 1e-2)])
+def test_sign_variants(dc, mode, mu, lam):
+    run_pair(3, RAGGED, so.SIGN, 6, p=2, dc=dc, mode=mode, mu=mu, lam=lam, seed=1)
+
+
+@pytest.mark.parametrize("K", [1, 3, 4])
+@pytest.mark.parametrize("p", [0, 1, 3])
+@pytest.mark.parametrize("num,den", [(1, 100), (1, 10)])
+def test_topk_ragged(K, p, num, den):
+    run_pair(K, RAGGED, so.TOPK, 6, p=p, num=num, den=den, outliers=(66, 100.0), seed=2)
+
+
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("mode", [so.EF, so.SAEF])
+def test_topk_variants(dc, mode):
+    run_pair(2, RAGGED, so.TOPK, 5, p=2, dc=dc, mode=mode, mu=0.9, lam=1e-3, num=1, den=20, seed=1)
+
+
+@pytest.mark.parametrize("K", [1, 3])
+def test_identity(K):
+    run_pair(K, RAGGED, so.IDENTITY, 5, p=2, lam=1e-3)
+
+
+def test_sign_aligned_rows_vector_path():
+    """d a multiple of 4 and tensors of whole tiles: every tile takes the 128-bit path."""
+    run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.SIGN, 6, p=1)
+    run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.SIGN, 6, p=3)
+    run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.TOPK, 6, p=3)
+
+
+def test_topk_ties_and_zeros():
+    """Gradients quantised to a few levels: many exact ties at the threshold and exact zeros."""
+    import torch
+    K, sizes = 2, [100, 4096, 5000]
+    d = sum(sizes)
+    rng = np.random.default_rng(7)
+    x0 = np.zeros(d, dtype=np.float32)
+    orc = so.Oracle(K, sizes, x0, compressor=so.TOPK, avg_period=2, momentum=0.5, topk_num=1, topk_den=10)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=sb.TOPK, avg_period=2, momentum=0.5, topk_num=1,
+                 topk_den=10)
+    for t in range(5):
+        g = (rng.integers(-3, 4, (K, d)) * 0.25).astype(np.float32)
+        g[:, :50] = 0
+        orc.step(g, 0.5)
+        gpu.step(torch.from_numpy(g).cuda(), 0.5)
+        compare_state(gpu, orc, so.TOPK, tag=f"ties t={t + 1}")
+        compare_server_messages(gpu, orc, so.TOPK, 1, tag=f"ties t={t + 1}")
+
+
+def test_all_zero_gradients_and_tiny_values():
+    """Degenerate inputs: zero gradients (scale 0, sign(0) = +), values below the 2^-64 fixed-point unit."""
+    import torch
+    K, sizes = 2, [33, 4096]
+    d = sum(sizes)
+    x0 = np.ones(d, dtype=np.float32)
+    for comp in (so.SIGN, so.TOPK):
+        orc = so.Oracle(K, sizes, x0, compressor=comp, avg_period=1)
+        gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=comp, avg_period=1)
+        for t, val in enumerate([0.0, 1e-30, 1e-42, 3.0]):
+            g = np.full((K, d), val, dtype=np.float32)
+            g[1] = -g[1]
+            orc.step(g, 0.1)
+            gpu.step(torch.from_numpy(g).cuda(), 0.1)
+            compare_state(gpu, orc, comp, tag=f"degenerate comp={comp} t={t + 1}")
+
+
+def test_large_values_take_the_integer_part_path():
+    import torch
+    K, sizes = 2, [1000, 4096]
+    d = sum(sizes)
+    rng = np.random.default_rng(3)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    orc = so.Oracle(K, sizes, x0, compressor=so.SIGN, avg_period=0)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=sb.SIGN, avg_period=0)
+    for t in range(3):
+        g = (rng.standard_normal((K, d)) * np.exp(rng.uniform(-10, 18, (K, d)))).astype(np.float32)
+        orc.step(g, 0.5)
+        gpu.step(torch.from_numpy(g).cuda(), 0.5)
+        compare_state(gpu, orc, so.SIGN, tag=f"large t={t + 1}")
+
+
+def test_range_error_is_reported_and_sticky_until_sync():
+    import torch
+    sizes = [64]
+    x0 = torch.zeros(64, device="cuda")
+    gpu = sb.Sae(1, sizes, x0, compressor=sb.SIGN)
+    g = torch.zeros(1, 64, device="cuda")
+    g[0, 5] = float("inf")
+    gpu.step(g, 0.1)
+    with pytest.raises(sb.SaeError) as ei:
+        gpu.sync()
+    assert ei.value.status == sb.ERR_RANGE
+    gpu.sync()          # cleared
+
+
+def test_invalid_arguments():
+    import torch
+    x0 = torch.zeros(10, device="cuda")
+    with pytest.raises(sb.SaeError):
+        sb.Sae(0, [10], x0)
+    with pytest.raises(sb.SaeError):
+        sb.Sae(1, [10], x0, momentum=1.0)
+    with pytest.raises(sb.SaeError):
+        sb.Sae(1, [10], x0, compressor=7)
+    gpu = sb.Sae(1, [10], x0)
+    with pytest.raises(sb.SaeError):
+        gpu.step(torch.zeros(1, 10, device="cuda"), 0.0)
+    with pytest.raises(sb.SaeError):
+        gpu.get_step_ahead(3)
+    with pytest.raises(sb.SaeError):
+        gpu.get_state(sb.STATE_WORKER_TAU)          # not a Top-K run
+
+
+def test_device_generator_matches_numpy():
+    import torch
+    for idx in (0, 1):
+        w = configs.workload(idx)
+        scales = synth.workload_scales(w, 0)
+        gen = synth.DeviceGenerator(w.tensor_sizes, scales)
+        out = torch.empty(w.num_workers, w.d, device="cuda")
+        for t in (0, 3):
+            gen.grads(out, w.num_workers, 0, t, w.outlier_per_65536, w.outlier_mult)
+            assert_same(f"grads cfg{idx} t={t}", out.cpu().numpy(), synth.workload_grads_numpy(w, 0, t, scales))
+        x = torch.empty(w.d, device="cuda")
+        gen.x0(x, 0)
+        assert_same("x0", x.cpu().numpy(), synth.x0_numpy(0, w.d))
+
+
+def test_step_host_and_get_params_host_match_device_path():
+    import torch
+    K, sizes = 3, RAGGED
+    d = sum(sizes)
+    x0 = torch.from_numpy(synth.x0_numpy(0, d)).cuda()
+    a = sb.Sae(K, sizes, x0, avg_period=2)
+    b = sb.Sae(K, sizes, x0, avg_period=2)
+    scales = synth.tensor_scales(0, len(sizes), -4.0, -1.0)
+    pinned = torch.empty(K, d).pin_memory()
+    out_host = torch.empty(d).pin_memory()
+    for t in range(4):
+        g = synth.grads_numpy(0, t, K, sizes, scales)
+        pinned.copy_(torch.from_numpy(g))
+        a.step(torch.from_numpy(g).cuda(), 0.1)
+        b.step_host(pinned, 0.1)
+        b.get_params_host(out_host)
+        assert_same("host path x", out_host.numpy(), a.get_params().cpu().numpy())
+
+
+def _trajectory(idx, p, steps, seed):
+    w = configs.workload(idx)
+    run_pair(w.num_workers, w.tensor_sizes, w.compressor, steps, seed=seed, p=p, mu=w.momentum, lam=w.weight_decay,
+             num=w.topk_num, den=w.topk_den, lrs=[w.lr], outliers=(w.outlier_per_65536, w.outlier_mult),
+             every=max(1, steps // 4))
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("p", [1, 5])
+def test_config0_full_trajectory(seed, p):
+    _trajectory(0, p, 10, seed)
+
+
+@pytest.mark.parametrize("p", [1, 20])
+def test_config1_trajectory(p):
+    _trajectory(1, p, 60, 0)
