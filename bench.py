@@ -179,6 +179,8 @@ def main():
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--ring", type=int, default=0, help="gradient sets kept in HBM (0 = auto)")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="override the workload's worker count (smaller cases of the same kernels for ncu captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -186,6 +188,9 @@ def main():
 
     from paper_2008_05823_b200 import configs
     w = configs.workload(args.workload)
+    if args.workers > 0:
+        w.num_workers = args.workers
+        w.name += f"_workers{args.workers}"
     p = args.avg_period
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -37,7 +37,8 @@ def build(force: bool = False, verbose: bool = False):
         src_paths = [os.path.join(CSRC, s) for s in srcs]
         dep_paths = src_paths + [h if os.path.isabs(h) else os.path.join(CSRC, h) for h in hdrs]
         if force or _stale(out, dep_paths):
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", out] + src_paths
+            extra = os.environ.get("SAE_NVCC_EXTRA", "").split()
+            cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", out] + src_paths
             subprocess.check_call(cmd)
         outs.append(out)
     return outs

@@ -9,7 +9,13 @@ namespace sae {
 typedef unsigned long long u64;
 typedef unsigned int u32;
 
-constexpr int TILE = 4096;       // elements of one tensor handled by one thread block
+#ifndef SAE_TILE
+#define SAE_TILE 4096
+#endif
+#ifndef SAE_WORKER_MINBLOCKS
+#define SAE_WORKER_MINBLOCKS 4
+#endif
+constexpr int TILE = SAE_TILE;   // elements of one tensor handled by one thread block
 constexpr int THREADS = 256;     // threads per block: 8 warps
 constexpr int VEC_ITERS = TILE / (THREADS * 4);   // float4 iterations per thread (4)
 constexpr int ROWS = TILE / THREADS;              // scalar elements per thread (16)

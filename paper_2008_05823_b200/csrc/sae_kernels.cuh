@@ -54,7 +54,7 @@ struct WorkerArgs {
 // K1: worker pass.  grid = ntiles * K, block (tile, k) with k fastest so that the K blocks sharing one
 // tile of ebar / x run close together.
 template <int ESRC, bool SIGN, bool WRITE_D>
-__global__ void __launch_bounds__(THREADS) k_worker(Plan P, StepParams sp, WorkerArgs A) {
+__global__ void __launch_bounds__(THREADS, SAE_WORKER_MINBLOCKS) k_worker(Plan P, StepParams sp, WorkerArgs A) {
   __shared__ u64 sh_red[3 * (THREADS / 32)];
   const int tile = blockIdx.x / P.K;
   const int k = blockIdx.x - tile * P.K;
