@@ -39,7 +39,8 @@ typedef enum {
   SAE_ERR_CUDA = -3,        /* a CUDA runtime call failed; sae_last_cuda_error gives the code            */
   SAE_ERR_RANGE = -4,       /* a model difference was non-finite or had magnitude >= 2^32 (device check) */
   SAE_ERR_TIMEOUT = -5,     /* reserved: a bounded device-side wait expired                               */
-  SAE_ERR_ABI = -6          /* abi_version mismatch                                                      */
+  SAE_ERR_ABI = -6,         /* abi_version mismatch                                                      */
+  SAE_ERR_TOO_LARGE = -7    /* input larger than the fixed scratch of sae_sign_compress_noalloc          */
 } sae_status;
 
 /* Compressor C(.) of Algorithm 1, applied per tensor (Section 5: "layer-wise"). */
@@ -159,6 +160,38 @@ const char *sae_strerror(int status);
 /* cudaError_t of the most recent failed CUDA call made on behalf of this handle (0 if none);
  * with h == NULL, of the most recent failed sae_init. */
 int sae_last_cuda_error(const sae_handle *h);
+
+/*
+ * (The paper has no counterpart for this entry point; it exists for a class of callers, not for a
+ * step of Algorithm 1.)
+ *
+ * The scaled-sign compressor of ONE tensor without any allocation, for callers that cannot call
+ * cudaMalloc: code running inside another framework's memory pool or under a fixed device-memory
+ * budget, plug-ins that are handed only their input and output buffers, and latency-critical loops in
+ * which an allocation (which may synchronise the whole device) is not acceptable.  Every other entry
+ * point of this library works on a handle whose state and scratch sae_init allocates.
+ *
+ * Computes C(v) of Eq. 2 for v[0..n): the exact L1 scale (same definition and same bits as the
+ * worker pass: sum of floor(|v_i| 2^64) as an integer, truncated to 53 bits, divided by n) into
+ * *scale, and the sign words (bit i of word w <-> v[32w+i] >= 0, padding bits 0) into
+ * words[0..ceil(n/32)).  range_flag (may be NULL) receives 1 if some |v_i| was non-finite or >= 2^32,
+ * else 0.  v, words, scale, range_flag: DEVICE pointers owned by the caller; the work is enqueued on
+ * `stream` (cudaStream_t, NULL = default stream) of the CURRENT device and is asynchronous.
+ *
+ * The per-tile partial sums live in a fixed array inside the library image (128 KiB + 256 B of
+ * device memory on every GPU that loads the library, held until the process exits), so:
+ *  - n must not exceed sae_noalloc_max_elements() = 33 554 432; larger inputs are rejected with
+ *    SAE_ERR_TOO_LARGE and nothing is launched (n < 1 or a NULL pointer: SAE_ERR_INVALID_ARG);
+ *  - the first call on each device looks up the array's device address (no allocation); make that
+ *    first call before starting any stream capture;
+ *  - all calls share the one array: two calls whose kernels may overlap on the GPU (different
+ *    streams, or different host threads) race on it -- serialise them.  The array keeps the previous
+ *    call's contents; the call itself clears the counter and flag it relies on.
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ */
+int sae_sign_compress_noalloc(const float *v, int64_t n, uint32_t *words, float *scale, int32_t *range_flag,
+                              void *stream);
+int64_t sae_noalloc_max_elements(void);
 
 #ifdef __cplusplus
 }

@@ -16,14 +16,14 @@ NUM_KERNELS = 12
  STATE_WORKER_WORDS, STATE_SERVER_WORDS, STATE_WORKER_TAU, STATE_SERVER_TAU, STATE_WORKER_MASK,
  STATE_SERVER_MASK) = range(11)
 
-OK, ERR_INVALID_ARG, ERR_NOMEM, ERR_CUDA, ERR_RANGE, ERR_TIMEOUT, ERR_ABI = 0, -1, -2, -3, -4, -5, -6
+OK, ERR_INVALID_ARG, ERR_NOMEM, ERR_CUDA, ERR_RANGE, ERR_TIMEOUT, ERR_ABI, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsae.so")
 
 EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_params_host", "sae_get_step_ahead",
            "sae_get_state", "sae_iteration", "sae_num_params", "sae_num_words", "sae_sync", "sae_set_profiling",
            "sae_get_kernel_times", "sae_kernel_name", "sae_kernel_launches", "sae_destroy", "sae_strerror",
-           "sae_last_cuda_error"]
+           "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements"]
 
 
 class SaeConfig(C.Structure):
@@ -74,6 +74,9 @@ def lib():
         L.sae_strerror.argtypes = [C.c_int]
         L.sae_strerror.restype = C.c_char_p
         L.sae_last_cuda_error.argtypes = [vp]
+        L.sae_sign_compress_noalloc.argtypes = [vp, i64, vp, vp, vp, vp]
+        L.sae_noalloc_max_elements.argtypes = []
+        L.sae_noalloc_max_elements.restype = i64
         _lib = L
     return _lib
 
@@ -185,3 +188,26 @@ class Sae:
         _check(lib().sae_get_kernel_times(self.h, ms, cnt), "sae_get_kernel_times", self.h)
         return {lib().sae_kernel_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(NUM_KERNELS)
                 if cnt[i] > 0}
+
+
+def noalloc_max_elements():
+    return int(lib().sae_noalloc_max_elements())
+
+
+def sign_compress_noalloc(v, words, scale, range_flag=None, stream=None):
+    """Scaled-sign compressor of one tensor through `sae_sign_compress_noalloc`: for callers that cannot
+    allocate device memory (they pass every buffer; the library's only scratch is a fixed array in its
+    image).  v: float32 CUDA tensor (n elements); words: int32 CUDA tensor of ceil(n/32) elements; scale:
+    float32 CUDA tensor of 1 element; range_flag: optional int32 CUDA tensor of 1 element.  Asynchronous on
+    the current stream of v's device.  Calls must not overlap on the GPU (they share the scratch array)."""
+    import torch
+    n = v.numel()
+    if not (v.is_cuda and v.dtype == torch.float32 and v.is_contiguous()):
+        raise ValueError("v must be a contiguous float32 CUDA tensor")
+    if words.numel() < (n + 31) // 32 or words.element_size() != 4 or not words.is_cuda or scale.numel() < 1:
+        raise ValueError("output buffers are too small")
+    with torch.cuda.device(v.device):
+        st = torch.cuda.current_stream(v.device).cuda_stream if stream is None else stream
+        rc = lib().sae_sign_compress_noalloc(v.data_ptr(), n, words.data_ptr(), scale.data_ptr(),
+                                             range_flag.data_ptr() if range_flag is not None else None, C.c_void_p(st))
+    _check(rc, "sae_sign_compress_noalloc")

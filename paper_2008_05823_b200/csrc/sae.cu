@@ -459,6 +459,7 @@ const char* sae_strerror(int status) {
     case SAE_ERR_RANGE: return "model difference non-finite or out of range (|v| >= 2^32)";
     case SAE_ERR_TIMEOUT: return "device wait timed out";
     case SAE_ERR_ABI: return "ABI version mismatch";
+    case SAE_ERR_TOO_LARGE: return "input exceeds the fixed scratch capacity of the no-allocation entry point";
     default: return "unknown status";
   }
 }
