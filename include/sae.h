@@ -38,7 +38,7 @@ typedef enum {
   SAE_ERR_NOMEM = -2,       /* device or host allocation failed                                          */
   SAE_ERR_CUDA = -3,        /* a CUDA runtime call failed; sae_last_cuda_error gives the code            */
   SAE_ERR_RANGE = -4,       /* a model difference was non-finite or had magnitude >= 2^32 (device check) */
-  SAE_ERR_TIMEOUT = -5,     /* reserved: a bounded device-side wait expired                               */
+  SAE_ERR_TIMEOUT = -5,     /* a bounded device-side wait (on a shared-memory barrier) expired           */
   SAE_ERR_ABI = -6,         /* abi_version mismatch                                                      */
   SAE_ERR_TOO_LARGE = -7    /* input larger than the fixed scratch of sae_sign_compress_noalloc          */
 } sae_status;
@@ -57,7 +57,7 @@ typedef struct {
   uint32_t abi_version;        /* must be SAE_ABI_VERSION                                               */
   int32_t num_workers;         /* K of Algorithm 1, 1..1024                                             */
   int32_t num_tensors;         /* T >= 1 compression segments                                           */
-  const int64_t *tensor_sizes; /* HOST pointer, T entries, 0 < n_j < 2^31; copied by sae_init           */
+  const int64_t *tensor_sizes; /* HOST pointer, T entries, 0 < n_j <= 2^30; copied by sae_init          */
   int32_t compressor;          /* SAE_COMPRESSOR_*                                                      */
   int32_t server_compress;     /* 1: double-way compression (server applies C, keeps its error e);
                                   0: single-way (server sends Delta uncompressed, e stays 0) (Section 5) */

@@ -2,6 +2,7 @@
 // per-iteration launch sequence of Algorithm 1.  Declarations and argument contracts: include/sae.h.
 #include "../../include/sae.h"
 #include "sae_kernels.cuh"
+#include "sae_worker_tma.cuh"
 
 #include <cstdio>
 #include <cstring>
@@ -14,10 +15,10 @@ namespace {
 
 thread_local int g_init_cuda_error = 0;
 
-enum Slot { S_WORKER = 0, S_SERVER, S_APPLY, S_TOPK_HIST, S_TOPK_SELECT, S_EXPORT, S_IMPORT, S_MASK, S_COUNT };
+enum Slot { S_WORKER = 0, S_SERVER, S_APPLY, S_TOPK_HIST, S_TOPK_SELECT, S_EXPORT, S_IMPORT, S_MASK, S_FINALIZE, S_COUNT };
 const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregate", "apply_update", "topk_hist",
                                                  "topk_select", "export", "import", "mask_words",
-                                                 "", "", "", ""};
+                                                 "finalize_scales", "", "", ""};
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
@@ -48,6 +49,7 @@ struct sae_handle {
   int esrc;              // how e^(k) is held now (ESRC_*)
   int last;              // which of scale[2]/tau[2] holds the last step's values
   int last_cuda_error;
+  int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
   int64_t launches;
   // profiling
   int profiling;
@@ -136,9 +138,24 @@ void topk_thresholds(sae_handle* h, const float* buf, int rows, u32* tau_out) {
   }
 }
 
+constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
+
 template <int ESRC, bool SIGN, bool WRITE_D>
 void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
-  LAUNCH(h, S_WORKER, (k_worker<ESRC, SIGN, WRITE_D>), (long long)h->P.ntiles * h->P.K, h->P, sp, wa);
+  static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
+  if (configured_device != h->device) {
+    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kWorkerSmem);
+    configured_device = h->device;
+  }
+  const long long nitems = (long long)h->P.ntiles * h->P.K;
+  // As many persistent blocks as the GPU holds, rounded down to a multiple of K when possible: block b
+  // then always works for worker b mod K, which lets its warps carry L1 partials across items.
+  long long grid = h->persistent_blocks;
+  if (h->P.K <= grid) grid -= grid % h->P.K;
+  if (nitems < grid) grid = nitems;
+  LaunchScope ls(h, S_WORKER);
+  k_worker_tma<ESRC, SIGN, WRITE_D><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
 }
 
 template <int COMP, int SRV>
@@ -166,7 +183,8 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
   ApplyArgs aa;
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.m = h->m; aa.D = h->D;
-  aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.tau_cur = h->tau[cur]; aa.tau_srv = h->tau_srv;
+  aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv; aa.tau_cur = h->tau[cur];
+  aa.tau_srv = h->tau_srv;
   aa.mask_srv = h->mask_srv; aa.eta = lr;
 
   if (c.compressor == SAE_COMPRESSOR_SIGN) {
@@ -180,6 +198,8 @@ int do_step(sae_handle* h, const float* grads, float lr) {
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
+    LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
+           h->scale[cur], h->recs_srv);
     if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, P.ntiles, P, sa);
     else LAUNCH(h, S_SERVER, k_server_sign<false>, P.ntiles, P, sa);
     const int avg = avg_after ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
@@ -236,7 +256,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   long long d = 0, dpad = 0, ntiles = 0;
   for (int j = 0; j < T; ++j) {
     const int64_t n = cfg->tensor_sizes[j];
-    if (n <= 0 || n >= (1ll << 31)) return SAE_ERR_INVALID_ARG;
+    if (n <= 0 || n > (1ll << 30)) return SAE_ERR_INVALID_ARG;
     d += n; dpad += (n + 31) / 32 * 32; ntiles += (n + TILE - 1) / TILE;
   }
   if (ntiles * K >= (1ll << 31) || ntiles >= (1ll << 31)) return SAE_ERR_INVALID_ARG;
@@ -253,6 +273,11 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
   for (int i = 0; i < SAE_NUM_KERNELS; ++i) { h->ms[i] = 0; h->cnt[i] = 0; }
+  {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms < 1) sms = 148;
+    h->persistent_blocks = sms * SAE_WT_BLOCKS_PER_SM;
+  }
 
   std::vector<int> tile_tensor((size_t)ntiles), first_tile(T), n32(T);
   std::vector<long long> off(T), poff(T);
@@ -407,6 +432,7 @@ int sae_sync(sae_handle* h) {
   SAE_CUDA(h, cudaMemsetAsync(h->status, 0, sizeof(u32), h->stream));
   SAE_CUDA(h, cudaStreamSynchronize(h->stream));
   const u32 st = *h->status_host;
+  if (st & STATUS_TIMEOUT) return SAE_ERR_TIMEOUT;
   if (st & STATUS_RANGE) return SAE_ERR_RANGE;
   return SAE_OK;
 }

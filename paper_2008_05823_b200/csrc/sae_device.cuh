@@ -133,12 +133,11 @@ __device__ __forceinline__ void acc_block_reduce(Acc128& a, u64* sh) {
 
 // The per-(row, tensor) accumulator in global memory: three 43-bit limbs in 64-bit words (21 bits of
 // headroom each, so integer atomicAdd from up to 2^21 tiles cannot overflow and the total does not
-// depend on the order of arrival) and an arrival counter.  The block that arrives last finalises the
-// scale and resets the record for the next step.
+// depend on the order of arrival).  A later kernel turns the finished sum into the scale and clears
+// the record for the next step.
 struct L1Record {
   u64 limb[3];
-  u32 count;
-  u32 pad;
+  u64 pad;
 };
 
 constexpr u64 M43 = (1ull << 43) - 1;
@@ -163,27 +162,16 @@ __device__ __forceinline__ float scale_from_limbs(u64 l0, u64 l1, u64 l2, int n)
   return __double2float_rn(q * 5.421010862427522e-20);  // 2^-64, exact scaling
 }
 
-// Called by thread 0 of a block with that block's partial sum.  Returns true in the block that arrived
-// last for this record and then writes the finished scale.
-__device__ __forceinline__ void l1_commit(const Acc128& a, L1Record* rec, int tiles, int n, float* scale_out,
-                                          u32* status) {
+// Adds one partial sum to a record: three fire-and-forget integer atomics (no ordering needed: the
+// record is only read by a later kernel of the same stream).
+__device__ __forceinline__ void l1_add_partial(const Acc128& a, L1Record* rec, u32* status) {
   if (a.bad) atomicOr(status, STATUS_RANGE);
-  u64 l0 = a.lo & M43;
-  u64 l1 = ((a.lo >> 43) | (a.hi << 21)) & M43;
-  u64 l2 = a.hi >> 22;
+  const u64 l0 = a.lo & M43;
+  const u64 l1 = ((a.lo >> 43) | (a.hi << 21)) & M43;
+  const u64 l2 = a.hi >> 22;
   if (l0) atomicAdd(&rec->limb[0], l0);
   if (l1) atomicAdd(&rec->limb[1], l1);
   if (l2) atomicAdd(&rec->limb[2], l2);
-  __threadfence();
-  u32 ticket = atomicAdd(&rec->count, 1u);
-  if (ticket == (u32)tiles - 1u) {
-    __threadfence();
-    u64 r0 = atomicExch(&rec->limb[0], 0ull);
-    u64 r1 = atomicExch(&rec->limb[1], 0ull);
-    u64 r2 = atomicExch(&rec->limb[2], 0ull);
-    atomicExch(&rec->count, 0u);
-    *scale_out = scale_from_limbs(r0, r1, r2, n);
-  }
 }
 
 // ---- sign bits -----------------------------------------------------------------------------------

@@ -51,83 +51,6 @@ struct WorkerArgs {
   u32* status;
 };
 
-// K1: worker pass.  grid = ntiles * K, block (tile, k) with k fastest so that the K blocks sharing one
-// tile of ebar / x run close together.
-template <int ESRC, bool SIGN, bool WRITE_D>
-__global__ void __launch_bounds__(THREADS, SAE_WORKER_MINBLOCKS) k_worker(Plan P, StepParams sp, WorkerArgs A) {
-  __shared__ u64 sh_red[3 * (THREADS / 32)];
-  const int tile = blockIdx.x / P.K;
-  const int k = blockIdx.x - tile * P.K;
-  const TileInfo ti = tile_info(P, tile);
-  const float* __restrict__ gp = A.g + (long long)k * P.d + ti.off + ti.t0;
-  const long long pbase = ti.poff + ti.t0;
-  const long long wbase = (long long)k * P.dpad + pbase;
-  float* __restrict__ mp = A.m + wbase;
-  float* dp = A.D + wbase;
-  const float* __restrict__ ebp = A.ebar + pbase;
-  const float* __restrict__ xp = A.x + pbase;
-  u32* wp = A.words + (long long)k * P.nwords + (pbase >> 5);
-  const float sprev = (ESRC == ESRC_LAZY_SIGN) ? A.scale_prev[(long long)k * P.T + ti.j] : 0.0f;
-  const u32 tprev = (ESRC == ESRC_LAZY_TOPK) ? A.tau_prev[(long long)k * P.T + ti.j] : 0u;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  Acc128 acc; acc_init(acc);
-
-  const bool vec = (ti.cnt == TILE) && ((reinterpret_cast<uintptr_t>(gp) & 15) == 0);
-  if (vec) {
-    float4 G[VEC_ITERS], M[VEC_ITERS], E[VEC_ITERS], X[VEC_ITERS];
-#pragma unroll
-    for (int it = 0; it < VEC_ITERS; ++it) {
-      const int i = it * (THREADS * 4) + tid * 4;
-      G[it] = ld4_stream(gp + i);
-      M[it] = ld4(mp + i);
-      E[it] = (ESRC == ESRC_UNIFORM) ? ld4(ebp + i) : ld4(dp + i);
-      if (sp.wd) X[it] = ld4(xp + i); else X[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int it = 0; it < VEC_ITERS; ++it) {
-      const int i = it * (THREADS * 4) + tid * 4;
-      float4 mn, dl;
-      dl.x = worker_update(G[it].x, M[it].x, prev_error<ESRC>(E[it].x, sprev, tprev), X[it].x, sp, mn.x);
-      dl.y = worker_update(G[it].y, M[it].y, prev_error<ESRC>(E[it].y, sprev, tprev), X[it].y, sp, mn.y);
-      dl.z = worker_update(G[it].z, M[it].z, prev_error<ESRC>(E[it].z, sprev, tprev), X[it].z, sp, mn.z);
-      dl.w = worker_update(G[it].w, M[it].w, prev_error<ESRC>(E[it].w, sprev, tprev), X[it].w, sp, mn.w);
-      st4(mp + i, mn);
-      if (WRITE_D) st4(dp + i, dl);
-      if (SIGN) {
-        acc_add(acc, dl.x); acc_add(acc, dl.y); acc_add(acc, dl.z); acc_add(acc, dl.w);
-        u32 w = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
-        if ((lane & 7) == 0) wp[(i >> 5)] = w;
-      }
-    }
-  } else {
-#pragma unroll 4
-    for (int r = 0; r < ROWS; ++r) {
-      const int i = r * THREADS + tid;
-      const bool valid = i < ti.cnt;
-      float dl = 0.0f;
-      if (valid) {
-        float e = prev_error<ESRC>((ESRC == ESRC_UNIFORM) ? ebp[i] : dp[i], sprev, tprev);
-        float xv = sp.wd ? xp[i] : 0.0f;
-        float mn;
-        dl = worker_update(__ldcs(gp + i), mp[i], e, xv, sp, mn);
-        mp[i] = mn;
-        if (WRITE_D) dp[i] = dl;
-        if (SIGN) acc_add(acc, dl);
-      }
-      if (SIGN) {
-        u32 w = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
-        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wp[(r * THREADS + warp * 32) >> 5] = w;
-      }
-    }
-  }
-  if (SIGN) {
-    acc_block_reduce(acc, sh_red);
-    if (tid == 0)
-      l1_commit(acc, A.recs + (long long)k * P.T + ti.j, ti.tiles_j, ti.n,
-                A.scale_cur + (long long)k * P.T + ti.j, A.status);
-  }
-}
-
 // ---------------------------------------------------------------------------------------------------
 struct ServerArgs {
   float* e_srv;            // [dpad]: in: server error e_t, out: server model difference Delta_{t+1}
@@ -211,7 +134,7 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
   }
   if (DC) {
     acc_block_reduce(acc, sh_red);
-    if (tid == 0) l1_commit(acc, A.recs_srv + ti.j, ti.tiles_j, ti.n, A.scale_srv + ti.j, A.status);
+    if (tid == 0) l1_add_partial(acc, A.recs_srv + ti.j, A.status);
   }
 }
 
@@ -267,6 +190,22 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   }
 }
 
+// Between the worker pass and the server pass: one thread per (worker, tensor) record turns the exact
+// L1 sum into the scale and clears the record; T more threads clear the server records, which the
+// previous step's apply kernel has finished reading.
+__global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const int* __restrict__ n, L1Record* recs,
+                                                              float* __restrict__ scale_cur, L1Record* recs_srv) {
+  const int q = blockIdx.x * THREADS + threadIdx.x;
+  if (q < K * T) {
+    L1Record r = recs[q];
+    recs[q].limb[0] = 0; recs[q].limb[1] = 0; recs[q].limb[2] = 0;
+    scale_cur[q] = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], n[q % T]);
+  } else if (q < K * T + T) {
+    L1Record* r = recs_srv + (q - K * T);
+    r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------
 struct ApplyArgs {
   float* e_srv;            // [dpad] in: Delta_{t+1}, out: e_{t+1}
@@ -275,7 +214,8 @@ struct ApplyArgs {
   const float* m;          // [K][dpad]
   const float* D;          // [K][dpad]
   const float* scale_cur;  // [K][T]
-  const float* scale_srv;  // [T]
+  float* scale_srv;        // [T] written here (scaled sign) from the server's L1 records
+  const L1Record* recs_srv;  // [T]
   const u32* tau_cur;      // [K][T]
   const u32* tau_srv;      // [T]
   u32* mask_srv;           // [nwords] Top-K: server selection of this step
@@ -318,7 +258,17 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
     }
     __syncthreads();
   }
-  const float s_srv = (SRV == 1) ? A.scale_srv[ti.j] : 0.0f;
+  __shared__ float sh_s_srv;
+  if (SRV == 1) {
+    // the server's scale of this tensor, from the exact sum the server pass accumulated
+    if (tid == 0) {
+      const L1Record r = A.recs_srv[ti.j];
+      sh_s_srv = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
+      if (ti.t0 == 0) A.scale_srv[ti.j] = sh_s_srv;
+    }
+    __syncthreads();
+  }
+  const float s_srv = (SRV == 1) ? sh_s_srv : 0.0f;
   const u32 t_srv = (SRV == 2) ? A.tau_srv[ti.j] : 0u;
   const long long pbase = ti.poff + ti.t0;
   float* ep = A.e_srv + pbase;
