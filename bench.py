@@ -30,7 +30,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one worker-pass launch per worker-element, from the committed ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case of the same kernel, which grows in
 # proportion to the elements processed).  None until a capture exists for the variant.
-WORKER_PASS_DRAM_BYTES_PER_ELEM = {"sign_p1": None, "sign_general": None, "topk": None}
+WORKER_PASS_DRAM_BYTES_PER_ELEM = {"sign_p1": 12.76, "sign_general": 19.63, "topk": None}   # profiles/worker_pass_sign_cfg2shapes_4workers.md
 
 
 def measured_peak():
@@ -153,6 +153,23 @@ def run_reference(args, w, avg_period, rank):
     print(json.dumps(line), flush=True)
 
 
+def max_over_ranks(value, device=None):
+    """Max of a per-rank scalar over the process group (a no-op without one).  Works on CPU tensors
+    (gloo) and CUDA tensors (nccl)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(steps, ms_total_max, world):
+    """steps/s of all replicas together: every rank runs `steps` steps in at most ms_total_max."""
+    return world * steps / (ms_total_max * 1e-3)
+
+
 def algorithmic_bytes(w, avg_period):
     """Bytes the method itself must move per step (each gradient read once, each persistent state word
     read and written once) and per launch of the worker pass."""
@@ -256,12 +273,9 @@ def main():
     ms_total = ev0.elapsed_time(ev1)
     gpu_launches = sae.kernel_launches - launches0
     sae.sync()                                    # raises if the device flagged a range error
-    if world > 1:
-        tt = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)
+    value = whole_job_value(args.steps, ms_total, world)
 
     # ---- per-kernel times (same steps again, every launch bracketed by events on the library's stream) ----
     sae.set_profiling(True)
@@ -307,10 +321,7 @@ def main():
                 sae.get_params_host(host_x)          # D2H of the step's result, synchronises
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
-            if world > 1:
-                tt = torch.tensor([dt], device=dev)
-                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-                dt = float(tt.item())
+            dt = max_over_ranks(dt, dev)
             sae.sync()
             sae.close()
             e2e = {"value": world * e2e_steps / dt, "unit": "steps/s", "h2d_bytes_per_step": grad_bytes,
