@@ -140,11 +140,11 @@ void topk_thresholds(sae_handle* h, const float* buf, int rows, u32* tau_out) {
 
 constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
 
-template <int ESRC, bool SIGN, bool WRITE_D>
-void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD>
+void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
   static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
   if (configured_device != h->device) {
-    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)kWorkerSmem);
     configured_device = h->device;
   }
@@ -155,7 +155,13 @@ void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
   if (h->P.K <= grid) grid -= grid % h->P.K;
   if (nitems < grid) grid = nitems;
   LaunchScope ls(h, S_WORKER);
-  k_worker_tma<ESRC, SIGN, WRITE_D><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
+  k_worker_tma<ESRC, SIGN, WRITE_D, WD><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
+}
+
+template <int ESRC, bool SIGN, bool WRITE_D>
+void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
+  if (sp.wd) launch_worker_wd<ESRC, SIGN, WRITE_D, true>(h, sp, wa);
+  else launch_worker_wd<ESRC, SIGN, WRITE_D, false>(h, sp, wa);
 }
 
 template <int COMP, int SRV>

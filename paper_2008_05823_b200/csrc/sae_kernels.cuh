@@ -26,10 +26,11 @@ __device__ __forceinline__ float prev_error(float v, float sprev, u32 tprev) {
 }
 
 // Algorithm 1, worker lines: step-ahead point, local momentum, local model difference.
+template <bool WD>
 __device__ __forceinline__ float worker_update(float g, float mo, float e, float x, const StepParams& sp,
                                                float& mn) {
   float ge = g;
-  if (sp.wd) {
+  if (WD) {
     float xh = sp.saef ? __fsub_rn(x, e) : x;
     ge = __fmaf_rn(sp.lambda, xh, g);
   }

@@ -94,26 +94,49 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes,
                : "memory");
 }
 
-// Per-lane L1 accumulator of the worker pass: 64-bit low word plus a carry / high count.  A lane adds
-// at most WT_SLICE/32 values per item, each < 2^96, so `hi` cannot overflow.
+// Per-lane L1 accumulator of the worker pass: a 96-bit sum (lo0, lo1, carry) fed by a three-instruction
+// carry chain, plus a 64-bit word for the integer parts of the rare values >= 1.
 struct LaneAcc {
-  u64 lo, hi;
+  u32 lo0, lo1, carry;
+  u64 hi;
   u32 bad;
 };
 
+__device__ __forceinline__ void lane_acc_init(LaneAcc& a) { a.lo0 = 0; a.lo1 = 0; a.carry = 0; a.hi = 0; a.bad = 0; }
+
+// += floor(m 2^64) for 0 <= m < 1 (exact: power-of-two scaling, then a round-down conversion)
+__device__ __forceinline__ void lane_add_small(LaneAcc& a, float m) {
+  const u64 f = __float2ull_rd(__fmul_rn(m, 18446744073709551616.0f));
+  const u32 f0 = (u32)f, f1 = (u32)(f >> 32);
+  asm("add.cc.u32 %0, %0, %3;\n\taddc.cc.u32 %1, %1, %4;\n\taddc.u32 %2, %2, 0;"
+      : "+r"(a.lo0), "+r"(a.lo1), "+r"(a.carry)
+      : "r"(f0), "r"(f1));
+}
+
+// any magnitude: the general (rare) path splits off the integer part, non-finite / >= 2^32 flags RANGE
 __device__ __forceinline__ void lane_add(LaneAcc& a, float v) {
   const float m = fabsf(v);
   if (m < 1.0f) {
-    const u64 f = __float2ull_rd(__fmul_rn(m, 18446744073709551616.0f));
-    a.lo += f;
-    a.hi += (a.lo < f ? 1ull : 0ull);
+    lane_add_small(a, m);
   } else if (m < 4294967296.0f) {
     const float ip = floorf(m);
-    const u64 f = __float2ull_rd(__fmul_rn(__fsub_rn(m, ip), 18446744073709551616.0f));
-    a.lo += f;
-    a.hi += __float2ull_rd(ip) + (a.lo < f ? 1ull : 0ull);
+    lane_add_small(a, __fsub_rn(m, ip));
+    a.hi += __float2ull_rd(ip);
   } else {
     a.bad = 1u;
+  }
+}
+
+// Four values at once: one test decides whether all of them are below 1 (the bit pattern of |v| orders
+// magnitudes and puts NaN / Inf above every finite value), so the common case has no per-element branch.
+__device__ __forceinline__ void lane_add4(LaneAcc& a, float4 v) {
+  const u32 k0 = __float_as_uint(v.x) & 0x7fffffffu, k1 = __float_as_uint(v.y) & 0x7fffffffu;
+  const u32 k2 = __float_as_uint(v.z) & 0x7fffffffu, k3 = __float_as_uint(v.w) & 0x7fffffffu;
+  if (max(max(k0, k1), max(k2, k3)) < 0x3f800000u) {
+    lane_add_small(a, __uint_as_float(k0)); lane_add_small(a, __uint_as_float(k1));
+    lane_add_small(a, __uint_as_float(k2)); lane_add_small(a, __uint_as_float(k3));
+  } else {
+    lane_add(a, v.x); lane_add(a, v.y); lane_add(a, v.z); lane_add(a, v.w);
   }
 }
 
@@ -122,16 +145,16 @@ __device__ __forceinline__ void lane_add(LaneAcc& a, float v) {
 // high word (almost always a small carry count) takes one more redux, or a shuffle tree if large.
 __device__ __forceinline__ void warp_commit(const LaneAcc& a, L1Record* rec, u32* status) {
   const u32 full = 0xffffffffu;
-  const u32 r0 = __reduce_add_sync(full, (u32)(a.lo & 0x3fffffu));
-  const u32 r1 = __reduce_add_sync(full, (u32)((a.lo >> 22) & 0x3fffffu));
-  const u32 r2 = __reduce_add_sync(full, (u32)(a.lo >> 44));                 // 20 bits
-  u64 hi;
-  if (__any_sync(full, a.hi >> 24)) {
-    hi = a.hi;
+  const u64 lo = ((u64)a.lo1 << 32) | a.lo0;
+  const u32 r0 = __reduce_add_sync(full, (u32)(lo & 0x3fffffu));
+  const u32 r1 = __reduce_add_sync(full, (u32)((lo >> 22) & 0x3fffffu));
+  const u32 r2 = __reduce_add_sync(full, (u32)(lo >> 44));                   // 20 bits
+  u64 hi = a.hi + a.carry;
+  if (__any_sync(full, hi >> 24)) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) hi += __shfl_xor_sync(full, hi, o);
   } else {
-    hi = __reduce_add_sync(full, (u32)a.hi);
+    hi = __reduce_add_sync(full, (u32)hi);
   }
   const u32 bad = __any_sync(full, a.bad);
   if ((threadIdx.x & 31) == 0) {
@@ -164,7 +187,7 @@ __device__ __forceinline__ WtItem wt_lookup(const Plan& P, const WorkerArgs& A, 
   return it;
 }
 
-template <int ESRC, bool SIGN, bool WRITE_D>
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD>
 __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma(Plan P, StepParams sp, WorkerArgs A,
                                                                                   long long nitems) {
   extern __shared__ unsigned char smem_raw[];
@@ -220,7 +243,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
   // A warp keeps adding to its L1 partial while consecutive items belong to the same (worker, tensor)
   // -- with a grid that is a multiple of K every item of a block has the same worker -- and commits
   // when that changes: the commit (atomics plus a fence) is then off the per-item path.
-  LaneAcc acc; acc.lo = 0; acc.hi = 0; acc.bad = 0;
+  LaneAcc acc; lane_acc_init(acc);
   int acc_k = 0, acc_j = 0;
   u32 acc_items = 0;
   long long w = blockIdx.x;
@@ -237,7 +260,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
     if (SIGN) {
       if (acc_items && (it.k != acc_k || it.j != acc_j)) {
         warp_commit(acc, A.recs + (long long)acc_k * P.T + acc_j, A.status);
-        acc.lo = 0; acc.hi = 0; acc.bad = 0; acc_items = 0;
+        lane_acc_init(acc); acc_items = 0;
       }
       acc_k = it.k; acc_j = it.j; acc_items += 1;
     }
@@ -254,16 +277,16 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
         const float4 M = *reinterpret_cast<const float4*>(sm + e0);
         const float4 E = *reinterpret_cast<const float4*>(se + e0);
         float4 X = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (sp.wd) X = ld4(xp + e0);
+        if (WD) X = ld4(xp + e0);
         float4 mn, dl;
-        dl.x = worker_update(G.x, M.x, prev_error<ESRC>(E.x, it.sprev, it.tprev), X.x, sp, mn.x);
-        dl.y = worker_update(G.y, M.y, prev_error<ESRC>(E.y, it.sprev, it.tprev), X.y, sp, mn.y);
-        dl.z = worker_update(G.z, M.z, prev_error<ESRC>(E.z, it.sprev, it.tprev), X.z, sp, mn.z);
-        dl.w = worker_update(G.w, M.w, prev_error<ESRC>(E.w, it.sprev, it.tprev), X.w, sp, mn.w);
+        dl.x = worker_update<WD>(G.x, M.x, prev_error<ESRC>(E.x, it.sprev, it.tprev), X.x, sp, mn.x);
+        dl.y = worker_update<WD>(G.y, M.y, prev_error<ESRC>(E.y, it.sprev, it.tprev), X.y, sp, mn.y);
+        dl.z = worker_update<WD>(G.z, M.z, prev_error<ESRC>(E.z, it.sprev, it.tprev), X.z, sp, mn.z);
+        dl.w = worker_update<WD>(G.w, M.w, prev_error<ESRC>(E.w, it.sprev, it.tprev), X.w, sp, mn.w);
         st4(mp + e0, mn);
         if (WRITE_D) st4(dp + e0, dl);
         if (SIGN) {
-          lane_add(acc, dl.x); lane_add(acc, dl.y); lane_add(acc, dl.z); lane_add(acc, dl.w);
+          lane_add4(acc, dl);
           const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
           if ((lane & 7) == 0) wp[e0 >> 5] = wd;
         }
@@ -284,9 +307,9 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
         float dl = 0.0f;
         if (valid) {
           const float e = prev_error<ESRC>((ESRC == ESRC_UNIFORM) ? ebp[e0] : dp[e0], it.sprev, it.tprev);
-          const float xv = sp.wd ? xp[e0] : 0.0f;
+          const float xv = WD ? xp[e0] : 0.0f;
           float mn;
-          dl = worker_update(__ldcs(gp + e0), mp[e0], e, xv, sp, mn);
+          dl = worker_update<WD>(__ldcs(gp + e0), mp[e0], e, xv, sp, mn);
           mp[e0] = mn;
           if (WRITE_D) dp[e0] = dl;
           if (SIGN) lane_add(acc, dl);
