@@ -3,6 +3,7 @@
 #include "../../include/sae.h"
 #include "sae_kernels.cuh"
 #include "sae_worker_tma.cuh"
+#include "sae_worker_fused.cuh"
 
 #include <cstdio>
 #include <cstring>
@@ -35,6 +36,7 @@ struct sae_handle {
   long long *d_off, *d_poff;
   // state
   float *x, *e_srv, *ebar, *m, *D;
+  float* etmp;           // [dpad] the pending average, materialised for getters only
   u32 *words, *words_srv, *mask_srv;
   float *scale[2], *scale_srv;
   u32 *tau[2], *tau_srv;
@@ -47,6 +49,8 @@ struct sae_handle {
   float* out_stage;      // sae_get_params_host
   int64_t t;
   int esrc;              // how e^(k) is held now (ESRC_*)
+  int fused_ok;          // p = 1, scaled sign, K a power of two <= 32: averaging is folded into the next worker pass
+  float eta_prev;        // learning rate of the last step (needed while the average is pending)
   int last;              // which of scale[2]/tau[2] holds the last step's values
   int last_cuda_error;
   int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
@@ -119,7 +123,7 @@ cudaError_t dalloc(T** p, size_t count) {
 }
 
 void free_all(sae_handle* h) {
-  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D,
+  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
                   h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -171,6 +175,38 @@ void launch_apply(sae_handle* h, int avg, const ApplyArgs& aa) {
   else LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_RECOMPUTE>), h->P.ntiles, h->P, aa);
 }
 
+constexpr size_t kFusedSmem = sizeof(FwSmem) + 128;
+
+template <int K, bool WD>
+void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
+  static thread_local int configured_device = -1;
+  if (configured_device != h->device) {
+    cudaFuncSetAttribute(k_worker_fused<K, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
+    configured_device = h->device;
+  }
+  const long long nitems = (long long)h->P.ntiles * FwGeom<K>::SUB;
+  long long grid = h->persistent_blocks / SAE_WT_BLOCKS_PER_SM;      // one block per SM
+  if (nitems < grid) grid = nitems;
+  LaunchScope ls(h, S_WORKER);
+  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems);
+}
+
+template <int K>
+void launch_fused_k(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
+  if (sp.wd) launch_fused_kw<K, true>(h, sp, fa); else launch_fused_kw<K, false>(h, sp, fa);
+}
+
+void launch_fused(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
+  switch (h->P.K) {
+    case 1: launch_fused_k<1>(h, sp, fa); break;
+    case 2: launch_fused_k<2>(h, sp, fa); break;
+    case 4: launch_fused_k<4>(h, sp, fa); break;
+    case 8: launch_fused_k<8>(h, sp, fa); break;
+    case 16: launch_fused_k<16>(h, sp, fa); break;
+    default: launch_fused_k<32>(h, sp, fa); break;
+  }
+}
+
 int do_step(sae_handle* h, const float* grads, float lr) {
   const sae_config& c = h->cfg;
   const Plan& P = h->P;
@@ -196,9 +232,17 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   if (c.compressor == SAE_COMPRESSOR_SIGN) {
     // The model differences need not be stored when the previous error was uniform and the next
     // pre-step averages: the averaging pass recomputes them from m and ebar with the same fused op.
-    const bool write_d = !(h->esrc == ESRC_UNIFORM && avg_after);
+    const bool pending_in = h->esrc == ESRC_PENDING_AVG;
+    const bool write_d = !((h->esrc == ESRC_UNIFORM || pending_in) && avg_after);
     if (write_d && !h->D) return SAE_ERR_INVALID_ARG;
-    if (h->esrc == ESRC_UNIFORM) {
+    // p = 1: the average is not formed here but at the head of the next worker pass
+    const bool defer_avg = avg_after && !write_d && h->fused_ok;
+    if (pending_in) {
+      FusedArgs fa;
+      fa.g = grads; fa.m = h->m; fa.ebar = h->ebar; fa.x = h->x; fa.scale_prev = h->scale[h->last];
+      fa.words = h->words; fa.recs = h->recs; fa.status = h->status; fa.eta_prev = h->eta_prev;
+      launch_fused(h, sp, fa);
+    } else if (h->esrc == ESRC_UNIFORM) {
       if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
       else launch_worker<ESRC_UNIFORM, true, false>(h, sp, wa);
     } else {
@@ -208,9 +252,9 @@ int do_step(sae_handle* h, const float* grads, float lr) {
            h->scale[cur], h->recs_srv);
     if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, P.ntiles, P, sa);
     else LAUNCH(h, S_SERVER, k_server_sign<false>, P.ntiles, P, sa);
-    const int avg = avg_after ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
+    const int avg = (avg_after && !defer_avg) ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
     if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
-    h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
+    h->esrc = defer_avg ? ESRC_PENDING_AVG : (avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN);
   } else if (c.compressor == SAE_COMPRESSOR_TOPK) {
     if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
     else launch_worker<ESRC_LAZY_TOPK, false, true>(h, sp, wa);
@@ -228,6 +272,7 @@ int do_step(sae_handle* h, const float* grads, float lr) {
     h->esrc = ESRC_UNIFORM;
   }
   h->last = cur;
+  h->eta_prev = lr;
   h->t += 1;
   return check_launch(h);
 }
@@ -237,6 +282,13 @@ int export_vec(sae_handle* h, int what, int k, float* out) {
   ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = h->ebar;
   ea.scale_last = h->scale[h->last]; ea.tau_last = h->tau[h->last];
   ea.esrc = h->esrc; ea.what = what; ea.k = k; ea.saef = (h->cfg.mode == SAE_MODE_SAEF);
+  if (h->esrc == ESRC_PENDING_AVG) {
+    // the averaged error exists only implicitly: form it in a scratch vector, leave the state alone
+    if (what == EXP_WERR || what == EXP_STEP_AHEAD)
+      LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, h->ebar, h->scale[h->last], h->eta_prev, h->etmp);
+    ea.ebar = h->etmp;
+    ea.esrc = ESRC_UNIFORM;
+  }
   LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
   return check_launch(h);
 }
@@ -277,7 +329,9 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   h->cfg.tensor_sizes = h->sizes.data();
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
-  h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
+  h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f;
+  h->fused_ok = (cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
+                 (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
   for (int i = 0; i < SAE_NUM_KERNELS; ++i) { h->ms[i] = 0; h->cnt[i] = 0; }
   {
     int sms = 0;
@@ -314,6 +368,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   ALLOC0(h->d_off, T); ALLOC0(h->d_poff, T);
   ALLOC0(h->x, dpad); ALLOC0(h->e_srv, dpad); ALLOC0(h->ebar, dpad);
   ALLOC0(h->m, (size_t)K * dpad);
+  if (h->fused_ok) ALLOC0(h->etmp, dpad);
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);

@@ -17,6 +17,7 @@ struct StepParams {
 constexpr int ESRC_UNIFORM = 0;    // e^(k) = ebar for all k (after an averaging pre-step, or at t = 0)
 constexpr int ESRC_LAZY_SIGN = 1;  // e^(k) = D^(k) - C(D^(k)) with last step's scales, D^(k) = last Delta^(k)
 constexpr int ESRC_LAZY_TOPK = 2;  // same with last step's Top-K thresholds
+constexpr int ESRC_PENDING_AVG = 3;  // p = 1, scaled sign: e^(k) = mean_k(fma(eta_prev, m^(k), ebar) - C(.)), not yet formed
 
 template <int ESRC>
 __device__ __forceinline__ float prev_error(float v, float sprev, u32 tprev) {

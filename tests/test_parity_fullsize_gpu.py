@@ -83,9 +83,12 @@ def test_config3_fullsize(p):
     run_fullsize(3, p, 5, budget=4_000_000)
 
 
-def test_config4_fullsize():
-    """32 workers x 109.5 M parameters: element offsets beyond 2^31, byte offsets beyond 2^32."""
-    run_fullsize(4, 2, 4, budget=6_000_000)
+@pytest.mark.parametrize("p", [1, 2])
+def test_config4_fullsize(p):
+    """32 workers x 109.5 M parameters: element offsets beyond 2^31, byte offsets beyond 2^32.
+    p = 1 runs the worker pass with the folded-in averaging (from the second step on), p = 2 alternates
+    stored and recomputed model differences."""
+    run_fullsize(4, p, 4, budget=2_500_000)
 
 
 def test_config4_embedding_scale_first_step():
