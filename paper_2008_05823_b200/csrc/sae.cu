@@ -5,6 +5,8 @@
 #include "sae_worker_tma.cuh"
 #include "sae_worker_fused.cuh"
 
+#include <cuda.h>
+#include <cudaTypedefs.h>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -37,6 +39,7 @@ struct sae_handle {
   // state
   float *x, *e_srv, *ebar, *m, *D;
   float* etmp;           // [dpad] the pending average, materialised for getters only
+  CUtensorMap tm_m;      // momentum rows [K][dpad] as a tensor map (folded-averaging worker pass)
   u32 *words, *words_srv, *mask_srv;
   float *scale[2], *scale_srv;
   u32 *tau[2], *tau_srv;
@@ -177,8 +180,34 @@ void launch_apply(sae_handle* h, int avg, const ApplyArgs& aa) {
 
 constexpr size_t kFusedSmem = sizeof(FwSmem) + 128;
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time dependency on libcuda).
+PFN_cuTensorMapEncodeTiled tensor_map_encoder() {
+  static PFN_cuTensorMapEncodeTiled fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (PFN_cuTensorMapEncodeTiled)p;
+  }
+  return fn;
+}
+
+// Row-major fp32 matrix [rows][inner] with the given row pitch, fetched in boxes of 256 x rows.
+bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows, long long pitch_elems) {
+  PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
+  if (!enc || (reinterpret_cast<uintptr_t>(base) & 15) || ((pitch_elems * 4) & 15)) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 4};
+  cuuint32_t box[2] = {(cuuint32_t)FW_BOX, (cuuint32_t)rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int K, bool WD>
-void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
+void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, const CUtensorMap& tm_g) {
   static thread_local int configured_device = -1;
   if (configured_device != h->device) {
     cudaFuncSetAttribute(k_worker_fused<K, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
@@ -188,22 +217,26 @@ void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
   long long grid = h->persistent_blocks / SAE_WT_BLOCKS_PER_SM;      // one block per SM
   if (nitems < grid) grid = nitems;
   LaunchScope ls(h, S_WORKER);
-  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems);
+  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, h->tm_m, tm_g);
 }
 
 template <int K>
-void launch_fused_k(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
-  if (sp.wd) launch_fused_kw<K, true>(h, sp, fa); else launch_fused_kw<K, false>(h, sp, fa);
+void launch_fused_k(sae_handle* h, const StepParams& sp, const FusedArgs& fa, const CUtensorMap& tm_g) {
+  if (sp.wd) launch_fused_kw<K, true>(h, sp, fa, tm_g); else launch_fused_kw<K, false>(h, sp, fa, tm_g);
 }
 
-void launch_fused(sae_handle* h, const StepParams& sp, const FusedArgs& fa) {
+void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa) {
+  // the gradients live in the caller's buffer: encode their tensor map for this step (host-only work)
+  CUtensorMap tm_g;
+  memset(&tm_g, 0, sizeof(tm_g));
+  fa.g_tma_ok = make_row_map(&tm_g, fa.g, h->P.d, h->P.K, h->P.d) ? 1 : 0;
   switch (h->P.K) {
-    case 1: launch_fused_k<1>(h, sp, fa); break;
-    case 2: launch_fused_k<2>(h, sp, fa); break;
-    case 4: launch_fused_k<4>(h, sp, fa); break;
-    case 8: launch_fused_k<8>(h, sp, fa); break;
-    case 16: launch_fused_k<16>(h, sp, fa); break;
-    default: launch_fused_k<32>(h, sp, fa); break;
+    case 1: launch_fused_k<1>(h, sp, fa, tm_g); break;
+    case 2: launch_fused_k<2>(h, sp, fa, tm_g); break;
+    case 4: launch_fused_k<4>(h, sp, fa, tm_g); break;
+    case 8: launch_fused_k<8>(h, sp, fa, tm_g); break;
+    case 16: launch_fused_k<16>(h, sp, fa, tm_g); break;
+    default: launch_fused_k<32>(h, sp, fa, tm_g); break;
   }
 }
 
@@ -240,7 +273,7 @@ int do_step(sae_handle* h, const float* grads, float lr) {
     if (pending_in) {
       FusedArgs fa;
       fa.g = grads; fa.m = h->m; fa.ebar = h->ebar; fa.x = h->x; fa.scale_prev = h->scale[h->last];
-      fa.words = h->words; fa.recs = h->recs; fa.status = h->status; fa.eta_prev = h->eta_prev;
+      fa.words = h->words; fa.recs = h->recs; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
       launch_fused(h, sp, fa);
     } else if (h->esrc == ESRC_UNIFORM) {
       if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
@@ -395,6 +428,10 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
     TRY(cudaStreamSynchronize(h->stream));     // host tables above go out of scope
   }
 #undef TRY
+  if (rc == SAE_OK && h->fused_ok) {
+    // the folded-averaging pass needs a tensor map over the momentum rows and 32-bit TMA coordinates
+    if (dpad >= (1ll << 31) || d >= (1ll << 31) || !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_ok = 0;
+  }
   if (rc != SAE_OK) { free_all(h); delete h; return rc; }
   // Pre-step of iteration 0: all errors are zero, so averaging (if (0+1) mod p = 0) changes nothing.
   *out = h;

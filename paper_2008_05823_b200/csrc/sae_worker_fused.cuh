@@ -5,25 +5,38 @@
 // Doing that in the apply kernel costs a second read of all K momentum rows.  This kernel instead
 // leaves the average pending and computes it at the head of the NEXT step's worker pass, which has to
 // read the same momentum rows anyway:
-//   phase A (per tile, all K workers): ebar' from the rows of m in shared memory, k = 0..K-1 in order,
+//   averaging (per tile, all K workers): ebar' from the rows of m in shared memory, k = 0..K-1 in order,
 //            with last step's learning rate and scales (same fused op, same order: same bits);
-//   phase B: the usual worker lines with e^(k) = ebar' -- momentum, Delta, exact L1 partials, sign words.
-// One block handles a tile for ALL workers: the producer warp brings the K momentum tiles and the ebar
-// tile -- and the K gradient tiles when they are 16-byte aligned -- in with bulk asynchronous copies
-// (3-stage ring, full/empty mbarriers), so the consumers touch global memory only to store.
+//   worker lines with e^(k) = ebar': momentum, Delta, exact L1 partials, sign words.
+// The two are done by different warps: four "averager" warps run one tile ahead of sixteen "worker"
+// warps and hand each tile over through an mbarrier, so the averaging overlaps the worker lines.
+// One block handles a tile for ALL workers: the producer warp brings the tile of all K momentum rows in
+// with 2-D tensor-map TMA copies (one request per box of 256 elements x K rows -- per-row copies of
+// 1-2 KB each were limited by the per-request cost), likewise the K gradient rows when the caller's
+// layout allows a tensor map (16-byte aligned base and row pitch), and the ebar tile with a 1-D bulk
+// copy; 3-stage ring, full/empty mbarriers.  The consumers touch global memory only to store.
 // In phase B a consumer warp always works for the same worker(s), so it carries their L1 partials
 // across tiles and adds them to the (worker, tensor) records only when the tensor changes.
 // All waits are bounded (STATUS_TIMEOUT).
 #pragma once
 #include "sae_worker_tma.cuh"
+#include <cuda.h>
 
 namespace sae {
 
-constexpr int FW_WARPS = 16;                       // consumer warps
-constexpr int FW_THREADS = FW_WARPS * 32 + 32;     // + producer warp
-constexpr int FW_STAGES = 3;
+constexpr int FW_WARPS = 16;                       // worker warps (warps 0..15)
+constexpr int FW_AVG_WARPS = 4;                    // averager warps (warps 17..20); warp 16 is the producer
+constexpr int FW_THREADS = (FW_WARPS + 1 + FW_AVG_WARPS) * 32;
+#ifndef SAE_FW_STAGES
+#define SAE_FW_STAGES 3
+#endif
+constexpr int FW_STAGES = SAE_FW_STAGES;
 constexpr int FW_MAXTILE = 2048;
-constexpr int FW_MBUF = 8192;                      // floats of momentum (and of gradient) per stage (32 KB each)
+constexpr int FW_BOX = 256;                        // inner extent of a TMA box (the hardware limit)
+#ifndef SAE_FW_MBUF
+#define SAE_FW_MBUF 8192
+#endif
+constexpr int FW_MBUF = SAE_FW_MBUF;                      // floats of momentum (and of gradient) per stage (32 KB each)
 
 template <int K>
 struct FwGeom {
@@ -33,13 +46,25 @@ struct FwGeom {
   static constexpr int RPW = K * ROWS_PER_WORKER / FW_WARPS;  // 128-element rows per warp and item
   static constexpr int WPW = RPW > ROWS_PER_WORKER ? RPW / ROWS_PER_WORKER : 1;   // workers per warp
   static_assert(K >= 1 && K <= 32 && (K & (K - 1)) == 0, "power-of-two worker counts up to 32");
-  static_assert(RPW >= 1 && WPW <= 2, "geometry");
+  static constexpr int CHUNKS = TILEF / FW_BOX;               // TMA boxes per array and item
+  static_assert(RPW >= 1 && WPW <= 2 && CHUNKS >= 1, "geometry");
+  // position of element e of worker k inside a stage buffer: boxes of [K][256] one after the other
+  __device__ static __forceinline__ int idx(int k, int e) { return (e >> 8) * (K * FW_BOX) + k * FW_BOX + (e & 255); }
 };
+
+// 2-D tiled TMA load of one box at element coordinates (x, y), completing on `bar`.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, u64* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
 
 struct FwItem {
   long long pbase;   // first element in the [dpad] arrays
   long long goff;    // first element inside a gradient row (caller layout)
-  int j, cnt, gvec;  // tensor, valid elements (0 = empty item), gradients 16-byte aligned for every worker
+  int j, cnt, gvec;  // tensor, valid elements (0 = empty item), gradient tile fetched by TMA into the stage
 };
 
 struct FwSmem {
@@ -48,6 +73,7 @@ struct FwSmem {
   alignas(128) float e[FW_STAGES][FW_MAXTILE];
   alignas(8) u64 full[FW_STAGES];
   alignas(8) u64 empty[FW_STAGES];
+  alignas(8) u64 avgd[FW_STAGES];   // "ebar' of this stage is ready": one arrival per averager warp
   FwItem item[FW_STAGES];
   float sc[FW_STAGES][32];      // last step's scales of the item's tensor, one per worker
 };
@@ -62,10 +88,11 @@ struct FusedArgs {
   L1Record* recs;
   u32* status;
   float eta_prev;
+  int g_tma_ok;            // the gradient buffer admits a tensor map (16-byte aligned base and row pitch)
 };
 
 template <int K>
-__device__ __forceinline__ FwItem fw_lookup(const Plan& P, const float* g, long long w, long long nitems) {
+__device__ __forceinline__ FwItem fw_lookup(const Plan& P, int g_tma_ok, long long w, long long nitems) {
   typedef FwGeom<K> G;
   FwItem it;
   it.pbase = 0; it.goff = 0; it.j = 0; it.cnt = 0; it.gvec = 0;
@@ -79,18 +106,22 @@ __device__ __forceinline__ FwItem fw_lookup(const Plan& P, const float* g, long 
   it.j = ti.j; it.cnt = cnt;
   it.pbase = ti.poff + t0;
   it.goff = ti.off + t0;
-  it.gvec = ((reinterpret_cast<uintptr_t>(g + it.goff) & 15) == 0) && (K == 1 || (P.d & 3) == 0);
+  it.gvec = g_tma_ok && ((it.goff & 3) == 0);
   return it;
 }
 
 template <int K, bool WD>
-__global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepParams sp, FusedArgs A, long long nitems) {
+__global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepParams sp, FusedArgs A, long long nitems,
+                                                                 const __grid_constant__ CUtensorMap tm_m,
+                                                                 const __grid_constant__ CUtensorMap tm_g) {
   typedef FwGeom<K> G;
   extern __shared__ unsigned char smem_raw[];
   FwSmem& S = *reinterpret_cast<FwSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
-    for (int s = 0; s < FW_STAGES; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], FW_WARPS); }
+    for (int s = 0; s < FW_STAGES; ++s) {
+      mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], FW_WARPS); mbar_init(&S.avgd[s], FW_AVG_WARPS);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -99,10 +130,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     // ---------------- producer ----------------
     const long long GR = gridDim.x;
     long long wb = blockIdx.x;
-    FwItem nxt = fw_lookup<K>(P, A.g, wb + lane * GR, nitems);
+    FwItem nxt = fw_lookup<K>(P, A.g_tma_ok, wb + lane * GR, nitems);
     for (int i0 = 0; wb < nitems; i0 += 32, wb += 32 * GR) {
       const FwItem cur = nxt;
-      nxt = fw_lookup<K>(P, A.g, wb + (32 + lane) * GR, nitems);
+      nxt = fw_lookup<K>(P, A.g_tma_ok, wb + (32 + lane) * GR, nitems);
       for (int l = 0; l < 32; ++l) {
         // the item of lane l, broadcast so that the lanes can share the issue of its copies
         const int cnt = __shfl_sync(0xffffffffu, cur.cnt, l);
@@ -127,18 +158,18 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         if (cnt == 0) {
           if (lane == 0) mbar_arrive(&S.full[s]);
         } else {
-          const u32 bytes = (u32)((cnt + 31) & ~31) * 4u;     // rows are padded to 32 elements
-          const int gfast = __shfl_sync(0xffffffffu, cur.gvec, l) && cnt == G::TILEF;
+          const u32 ebytes = (u32)((cnt + 31) & ~31) * 4u;    // rows are padded to 32 elements
+          const int gtma = __shfl_sync(0xffffffffu, cur.gvec, l);
           const long long goff = __shfl_sync(0xffffffffu, cur.goff, l);
           if (lane == 0) {
-            mbar_arrive_expect_tx(&S.full[s], bytes * (K + 1) + (gfast ? (u32)(G::TILEF * 4 * K) : 0u));
-            bulk_load(S.e[s], A.ebar + pbase, bytes, &S.full[s]);
-          }
-          __syncwarp();
-          if (lane < K) {
-            bulk_load(&S.m[s][lane * G::TILEF], A.m + (long long)lane * P.dpad + pbase, bytes, &S.full[s]);
-            if (gfast)
-              bulk_load(&S.g[s][lane * G::TILEF], A.g + (long long)lane * P.d + goff, G::TILEF * 4, &S.full[s]);
+            const int chunks = (cnt + FW_BOX - 1) / FW_BOX;
+            constexpr u32 BOXB = (u32)(K * FW_BOX * 4);
+            mbar_arrive_expect_tx(&S.full[s], ebytes + (u32)chunks * BOXB * (gtma ? 2u : 1u));
+            bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);
+            for (int c = 0; c < chunks; ++c) {
+              tma_load_2d(&S.m[s][c * K * FW_BOX], &tm_m, (int)pbase + c * FW_BOX, 0, &S.full[s]);
+              if (gtma) tma_load_2d(&S.g[s][c * K * FW_BOX], &tm_g, (int)goff + c * FW_BOX, 0, &S.full[s]);
+            }
           }
         }
       }
@@ -146,14 +177,66 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     return;
   }
 
-  // ---------------- consumers ----------------
+  const float Kf = (float)K;
+  if (warp > FW_WARPS) {
+    // ---------------- averagers: ebar' = (1/K) sum_k ( fma(eta_prev, m_k, ebar) - C(.) ), k in order ----------------
+    constexpr int NA = FW_AVG_WARPS * 32;
+    constexpr int EPT = G::TILEF / NA;               // elements per thread: 2, 4, 8 or 16
+    constexpr int V = EPT < 4 ? EPT : 4;             // handled in chunks of V consecutive elements
+    constexpr int CH = EPT / V;
+    const int ta = tid - (FW_WARPS + 1) * 32;
+    long long w = blockIdx.x;
+    for (int i = 0; w < nitems; ++i, w += gridDim.x) {
+      const int s = i % FW_STAGES;
+      if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
+        if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
+        return;
+      }
+      const FwItem it = S.item[s];
+      if (it.cnt > 0) {
+        const float* sm = S.m[s];
+        float* se = S.e[s];
+        const float* sc = S.sc[s];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+          const int e0 = c * (NA * V) + ta * V;
+          if (e0 < it.cnt) {
+            float eb[V], a[V];
+#pragma unroll
+            for (int v = 0; v < V; ++v) { eb[v] = se[e0 + v]; a[v] = 0.0f; }
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+              const float sk = sc[k];
+#pragma unroll
+              for (int v = 0; v < V; ++v) {
+                const float dk = __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[v]);
+                a[v] = __fadd_rn(a[v], __fsub_rn(dk, sign_code(dk, sk)));
+              }
+            }
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+              if (e0 + v < it.cnt) {
+                const float en = __fdiv_rn(a[v], Kf);
+                se[e0 + v] = en;
+                A.ebar[it.pbase + e0 + v] = en;
+              }
+            }
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&S.avgd[s]);
+    }
+    return;
+  }
+
+  // ---------------- workers ----------------
   LaneAcc acc[G::WPW];
 #pragma unroll
   for (int a = 0; a < G::WPW; ++a) lane_acc_init(acc[a]);
   int acc_j = -1;
   const int row0 = warp * G::RPW;                       // first row of this warp inside an item
   const int k0 = row0 / G::ROWS_PER_WORKER;             // its (first) worker
-  const float Kf = (float)K;
   long long w = blockIdx.x;
   for (int i = 0; w < nitems; ++i, w += gridDim.x) {
     const int s = i % FW_STAGES;
@@ -173,29 +256,15 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         }
         acc_j = it.j;
       }
-      const bool gfast = it.gvec && it.cnt == G::TILEF;
-      // ---- phase A: the pending average, ebar' ----
       const float* sm = S.m[s];
-      float* se = S.e[s];
-      {
-        const float* sc = S.sc[s];
-        for (int e = tid; e < it.cnt; e += FW_WARPS * 32) {
-          {
-            const float eb = se[e];
-            float a = 0.0f;
-#pragma unroll
-            for (int k = 0; k < K; ++k) {
-              const float dk = __fmaf_rn(A.eta_prev, sm[k * G::TILEF + e], eb);
-              a = __fadd_rn(a, __fsub_rn(dk, sign_code(dk, sc[k])));
-            }
-            const float en = __fdiv_rn(a, Kf);
-            se[e] = en;
-            A.ebar[it.pbase + e] = en;
-          }
-        }
+      const float* sg = S.g[s];
+      const float* se = S.e[s];
+      // ebar' of this tile comes from the averager warps
+      if (!mbar_wait(&S.avgd[s], (i / FW_STAGES) & 1)) {
+        if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
+        return;
       }
-      asm volatile("bar.sync 1, %0;" ::"n"(FW_WARPS * 32) : "memory");
-      // ---- phase B: worker lines with e^(k) = ebar' ----
+      // ---- worker lines with e^(k) = ebar' ----
 #pragma unroll
       for (int q = 0; q < G::RPW; ++q) {
         const int r = row0 + q;
@@ -203,12 +272,11 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         const int a = (G::WPW == 1) ? 0 : (k - k0);
         float* mp = A.m + (long long)k * P.dpad + it.pbase;
         u32* wp = A.words + (long long)k * P.nwords + (it.pbase >> 5);
-        const float* smk = sm + k * G::TILEF;
-        const float* sgk = S.g[s] + k * G::TILEF;
-        if (gfast) {
+        const int rbase = G::idx(k, rr * 128);                 // the row's position in the stage buffers
+        if (it.gvec && rr * 128 + 128 <= it.cnt) {
           const int e0 = rr * 128 + lane * 4;
-          const float4 Gq = *reinterpret_cast<const float4*>(sgk + e0);
-          const float4 M = *reinterpret_cast<const float4*>(smk + e0);
+          const float4 Gq = *reinterpret_cast<const float4*>(sg + rbase + lane * 4);
+          const float4 M = *reinterpret_cast<const float4*>(sm + rbase + lane * 4);
           const float4 E = *reinterpret_cast<const float4*>(se + e0);
           float4 X = make_float4(0.f, 0.f, 0.f, 0.f);
           if (WD) X = ld4(A.x + it.pbase + e0);
@@ -224,6 +292,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
           if ((lane & 7) == 0) wp[e0 >> 5] = wd;
         } else if (rr * 128 < it.cnt) {
+          // ragged last row of a tensor, or gradients that could not be fetched by TMA
           const float* gp = A.g + (long long)k * P.d + it.goff;
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -232,8 +301,9 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
             float dl = 0.0f;
             if (valid) {
               const float xv = WD ? A.x[it.pbase + e] : 0.0f;
+              const float gv = it.gvec ? sg[rbase + c * 32 + lane] : __ldcs(gp + e);
               float mn;
-              dl = worker_update<WD>(__ldcs(gp + e), smk[e], se[e], xv, sp, mn);
+              dl = worker_update<WD>(gv, sm[rbase + c * 32 + lane], se[e], xv, sp, mn);
               mp[e] = mn;
               if (G::WPW == 1) lane_add(acc[0], dl);
               else if (a == 0) lane_add(acc[0], dl);

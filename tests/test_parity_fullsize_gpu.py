@@ -15,7 +15,8 @@ pytestmark = pytest.mark.gpu
 
 def sample_tensors(sizes, budget):
     order = np.argsort(sizes)
-    pick = [int(order[-1]), int(order[0]), int(order[len(order) // 2]), len(sizes) - 1, 0, len(sizes) - 2]
+    fits = [int(j) for j in order[::-1] if sizes[j] <= budget]
+    pick = fits[:1] + [int(order[0]), int(order[len(order) // 2]), len(sizes) - 1, len(sizes) - 2]
     rng = np.random.default_rng(0)
     pick += [int(j) for j in rng.permutation(len(sizes))[:12]]
     out, total = [], 0
