@@ -30,7 +30,8 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one worker-pass launch per worker-element, from the committed ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case of the same kernel, which grows in
 # proportion to the elements processed).  None until a capture exists for the variant.
-WORKER_PASS_DRAM_BYTES_PER_ELEM = {"sign_p1": 12.76, "sign_general": 19.63, "topk": None}   # profiles/worker_pass_sign_cfg2shapes_4workers.md
+# sign_p1: 13.64 B at K = 4 = 12 B per worker-element + (8 B of ebar + sign words) per parameter.
+WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0), "topk": None}   # (per worker-element, per parameter), profiles/worker_pass_sign_cfg2shapes_4workers.md
 
 
 def measured_peak():
@@ -125,7 +126,7 @@ def cpu_baseline(w, avg_period, seed, steps, warmup, target_elems=40_000_000):
         orc.step(grads[t % 2], w.lr)
         warm_dt = time.perf_counter() - t0
     if steps <= 0:                      # aim at ~15 s of CPU work
-        steps = int(max(2, min(200, 15.0 / max(warm_dt, 1e-3))))
+        steps = int(max(2, min(1000, 15.0 / max(warm_dt, 1e-3))))
     t0 = time.perf_counter()
     for t in range(steps):
         orc.step(grads[t % 2], w.lr)
@@ -176,7 +177,7 @@ def algorithmic_bytes(w, avg_period):
     Wd, d = w.num_workers * w.d, w.d
     if avg_period == 1:
         step = 12 * Wd + 24 * d              # g R, m RW | x RW, e_srv RW, ebar RW
-        worker = 12 * Wd + 4 * d             # g R, m RW | ebar R once
+        worker = 12 * Wd + 8 * d             # g R, m RW | ebar RW (the pending average is formed in this pass)
         variant = "sign_p1" if w.compressor == 1 else "topk"
     else:
         step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW
@@ -290,9 +291,9 @@ def main():
     peak, peak_source = measured_peak()
     wk_ms = kernels["worker_pass"]["ms_per_launch"]
     achieved = worker_bytes / (wk_ms * 1e-3) / 1e9
-    per_elem = WORKER_PASS_DRAM_BYTES_PER_ELEM.get(variant)
+    per = WORKER_PASS_DRAM_BYTES.get(variant)
     roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": (per_elem * K * d) if per_elem else None,
+                "frac": achieved / peak, "traffic": (per[0] * K * d + per[1] * d) if per else None,
                 "algorithmic_bytes_per_launch": worker_bytes, "ms_per_launch": wk_ms, "peak_source": peak_source,
                 "frac_of_nominal_8TBs": achieved / 8000.0,
                 "step": {"algorithmic_bytes": step_bytes, "achieved_GBs": step_bytes / (ms_per_step * 1e-3) / 1e9,
