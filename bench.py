@@ -237,6 +237,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # Everything runs on one non-default stream: on such a stream sae_step replays cached CUDA graphs.
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+
     K, d = w.num_workers, w.d
     scales = synth.workload_scales(w, args.seed)
     gen = synth.DeviceGenerator(w.tensor_sizes, scales, device=dev)

@@ -87,7 +87,11 @@ int sae_init(const sae_config *cfg, const float *x0, sae_handle **out);
  *   e^(k) = Delta^(k) - C(Delta^(k));  Delta = e + (1/K) sum_k C(Delta^(k));  e = Delta - C(Delta);
  *   x = x - C(Delta).
  * grads: device, [K][d] floats, caller layout, read-only, must stay valid until the step has run.
- * lr: eta_t > 0.  Enqueues kernels only; allocates nothing.
+ * lr: eta_t > 0.  Enqueues kernels only; allocates no device memory.
+ * On a stream other than the default stream the kernels of a step are captured once per distinct
+ * (state, grads pointer, lr) into a CUDA graph and later steps with the same key replay it with one
+ * graph launch (the host cost of a step drops from one launch per kernel to one launch); if the
+ * caller is itself capturing the stream, the kernels simply join that capture.
  */
 int sae_step(sae_handle *h, const float *grads, float lr);
 

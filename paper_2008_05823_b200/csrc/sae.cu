@@ -25,6 +25,9 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
+struct StepGraphKey { int esrc, last, avg_after; const float* grads; float lr, eta_prev; };
+struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after; uint64_t stamp; };
+
 }  // namespace
 
 struct sae_handle {
@@ -58,6 +61,10 @@ struct sae_handle {
   int last_cuda_error;
   int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
   int64_t launches;
+  // cached step graphs
+  int graphs_enabled, graph_misses;
+  uint64_t graph_clock;
+  std::vector<StepGraph> graphs;
   // profiling
   int profiling;
   std::vector<EventPair> pending;
@@ -131,6 +138,7 @@ void free_all(sae_handle* h) {
                   h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (h->status_host) cudaFreeHost(h->status_host);
+  for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& ep : h->pending) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
   for (auto e : h->pool) cudaEventDestroy(e);
 }
@@ -240,7 +248,7 @@ void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa) {
   }
 }
 
-int do_step(sae_handle* h, const float* grads, float lr) {
+int do_step_direct(sae_handle* h, const float* grads, float lr) {
   const sae_config& c = h->cfg;
   const Plan& P = h->P;
   const bool avg_after = c.avg_period > 0 && ((h->t + 2) % c.avg_period == 0);
@@ -310,6 +318,69 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   return check_launch(h);
 }
 
+// One step through a cached CUDA graph.  The launch sequence of a step depends only on the handle's
+// small state (how the error is held, which scale buffer is current, whether the pre-step averages),
+// the gradient pointer and the learning rate; a step with a key seen before is replayed with a single
+// cudaGraphLaunch, which takes the per-kernel launch cost off the host (small workloads are bound by it).
+int do_step(sae_handle* h, const float* grads, float lr) {
+  bool usable = h->graphs_enabled && !h->profiling && h->stream != nullptr && h->stream != cudaStreamLegacy &&
+                h->stream != cudaStreamPerThread;
+  if (usable) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(h->stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+      cudaGetLastError();
+      usable = false;          // the caller is capturing this stream: our launches simply join that capture
+    }
+  }
+  if (!usable) return do_step_direct(h, grads, lr);
+
+  StepGraphKey key;
+  key.esrc = h->esrc; key.last = h->last;
+  key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
+  key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
+  for (size_t q = 0; q < h->graphs.size(); ++q) {
+    StepGraph& e = h->graphs[q];
+    if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
+        e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+      SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
+      h->launches += e.kernels;
+      h->esrc = e.esrc_after; h->last = e.last_after; h->eta_prev = lr; h->t += 1;
+      e.stamp = ++h->graph_clock;
+      h->graph_misses = 0;
+      return SAE_OK;
+    }
+  }
+  // Not seen before.  A caller whose key changes every step (say, a new learning rate each time) would
+  // only pay for captures: give up on graphs after a run of misses.
+  if (++h->graph_misses > 64) { h->graphs_enabled = 0; return do_step_direct(h, grads, lr); }
+  const int64_t launches0 = h->launches;
+  SAE_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+  int rc = do_step_direct(h, grads, lr);
+  cudaGraph_t graph = nullptr;
+  cudaError_t ce = cudaStreamEndCapture(h->stream, &graph);
+  if (rc != SAE_OK || ce != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); }
+    return rc != SAE_OK ? rc : SAE_ERR_CUDA;
+  }
+  StepGraph e;
+  e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
+  e.esrc_after = h->esrc; e.last_after = h->last; e.stamp = ++h->graph_clock;
+  ce = cudaGraphInstantiate(&e.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); return SAE_ERR_CUDA; }
+  SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
+  if (h->graphs.size() >= 32) {               // evict the least recently used graph
+    size_t victim = 0;
+    for (size_t q = 1; q < h->graphs.size(); ++q) if (h->graphs[q].stamp < h->graphs[victim].stamp) victim = q;
+    cudaGraphExecDestroy(h->graphs[victim].exec);
+    h->graphs[victim] = e;
+  } else {
+    h->graphs.push_back(e);
+  }
+  return SAE_OK;
+}
+
 int export_vec(sae_handle* h, int what, int k, float* out) {
   ExportArgs ea;
   ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = h->ebar;
@@ -363,6 +434,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f;
+  h->graphs_enabled = 1; h->graph_misses = 0; h->graph_clock = 0;
   h->fused_ok = (cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
                  (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
   for (int i = 0; i < SAE_NUM_KERNELS; ++i) { h->ms[i] = 0; h->cnt[i] = 0; }

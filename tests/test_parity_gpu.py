@@ -193,6 +193,35 @@ def test_step_host_and_get_params_host_match_device_path():
         assert_same("host path x", out_host.numpy(), a.get_params().cpu().numpy())
 
 
+@pytest.mark.parametrize("comp,p", [(so.SIGN, 1), (so.SIGN, 3), (so.TOPK, 2)])
+def test_graph_replay_on_a_side_stream(comp, p):
+    """On a non-default stream a step is captured into a CUDA graph per (state, gradient pointer, lr)
+    and replayed: cycle through two gradient buffers for many steps, compare with the oracle at the end
+    and along the way."""
+    import torch
+    K, sizes = 4, RAGGED
+    d = sum(sizes)
+    scales = synth.tensor_scales(3, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(3, d)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        orc = so.Oracle(K, sizes, x0, compressor=comp, avg_period=p, weight_decay=1e-4, topk_den=20, threads=4)
+        gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=comp, avg_period=p, weight_decay=1e-4, topk_den=20)
+        gs = [synth.grads_numpy(3, t, K, sizes, scales) for t in range(2)]
+        bufs = [torch.from_numpy(g).cuda() for g in gs]
+        launches = []
+        for t in range(14):
+            orc.step(gs[t % 2], 0.1 if t < 10 else 0.05)
+            gpu.step(bufs[t % 2], 0.1 if t < 10 else 0.05)
+            launches.append(gpu.kernel_launches)
+            if t in (5, 9, 13):
+                compare_state(gpu, orc, comp, tag=f"graph comp={comp} p={p} t={t + 1}")
+                compare_server_messages(gpu, orc, comp, 1, tag=f"graph comp={comp} p={p} t={t + 1}")
+        per_step = np.diff(np.array(launches))
+        assert per_step.min() >= 3          # replayed steps still account for their kernels
+        gpu.close()
+
+
 def _trajectory(idx, p, steps, seed):
     w = configs.workload(idx)
     run_pair(w.num_workers, w.tensor_sizes, w.compressor, steps, seed=seed, p=p, mu=w.momentum, lam=w.weight_decay,
