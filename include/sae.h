@@ -128,6 +128,9 @@ int sae_get_step_ahead(sae_handle *h, int32_t worker, float *out);
 #define SAE_STATE_SERVER_TAU 8    /* same for the server, T uint32                                      */
 #define SAE_STATE_WORKER_MASK 9   /* Top-K: selected set of the last step as bit words (format below)   */
 #define SAE_STATE_SERVER_MASK 10  /* same for the server                                                */
+#define SAE_STATE_TOPK_FALLBACKS 11 /* Top-K diagnostics, 2 uint32: how many (worker, tensor) pairs and how
+                                     many server tensors so far needed the full radix select because the
+                                     candidate window around the previous threshold did not hold it    */
 int sae_get_state(sae_handle *h, int32_t which, int32_t worker, void *out, size_t bytes);
 /*
  * Bit-word format (sign message and Top-K mask): per tensor ceil(n_j/32) little-endian uint32 words,

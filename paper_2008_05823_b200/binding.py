@@ -14,7 +14,7 @@ NUM_KERNELS = 12
 
 (STATE_MOMENTUM, STATE_WORKER_ERROR, STATE_SERVER_ERROR, STATE_WORKER_SCALES, STATE_SERVER_SCALES,
  STATE_WORKER_WORDS, STATE_SERVER_WORDS, STATE_WORKER_TAU, STATE_SERVER_TAU, STATE_WORKER_MASK,
- STATE_SERVER_MASK) = range(11)
+ STATE_SERVER_MASK, STATE_TOPK_FALLBACKS) = range(12)
 
 OK, ERR_INVALID_ARG, ERR_NOMEM, ERR_CUDA, ERR_RANGE, ERR_TIMEOUT, ERR_ABI, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
 
@@ -162,6 +162,8 @@ class Sae:
             out = self._vec(n=self.T)
         elif which in (STATE_WORKER_TAU, STATE_SERVER_TAU):
             out = self._vec(dtype=t.int32, n=self.T)
+        elif which == STATE_TOPK_FALLBACKS:
+            out = self._vec(dtype=t.int32, n=2)
         else:
             out = self._vec(dtype=t.int32, n=self.nwords)
         _check(lib().sae_get_state(self.h, which, worker, out.data_ptr(), out.numel() * out.element_size()),

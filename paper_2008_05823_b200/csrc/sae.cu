@@ -49,6 +49,14 @@ struct sae_handle {
   L1Record *recs, *recs_srv;
   u32 *hist;
   SelectState* sel;
+  // Top-K candidate windows: key lists, per-tensor region offsets / capacities, cursors, fallback flags
+  u32 *cand_keys, *cand_keys_srv, *cand_count, *cand_count_srv, *fb, *fb_srv, *fb_total;
+  long long* d_cand_off;
+  int* d_cand_cap;
+  int2* work;            // work list of the radix select: data items and candidate chunks
+  u32* work_count;
+  u32* cand_n;           // [K][T] candidates captured for this step's select
+  long long cand_stride;
   u32* status;
   u32* status_host;      // pinned
   float* staging;        // sae_step_host
@@ -135,7 +143,9 @@ cudaError_t dalloc(T** p, size_t count) {
 void free_all(sae_handle* h) {
   void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
-                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage};
+                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage,
+                  h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
+                  h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (h->status_host) cudaFreeHost(h->status_host);
   for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
@@ -144,22 +154,40 @@ void free_all(sae_handle* h) {
 }
 
 // ---- Top-K threshold of every (row, tensor) of buf[rows][dpad] ---------------------------------------
-void topk_thresholds(sae_handle* h, const float* buf, int rows, u32* tau_out) {
+// Candidate-window refine first; the three-level radix select then runs only where the window failed.
+void topk_thresholds(sae_handle* h, const float* buf, int rows, const CandArgs& cand, const u32* tau_guess, u32* tau_out,
+                     u32* fb, u32* fb_total) {
   const Plan& P = h->P;
+  const int pairs = rows * P.T;
+  LAUNCH(h, S_TOPK_SELECT, k_topk_decide, (pairs + THREADS - 1) / THREADS, cand, rows, h->d_n, h->cfg.topk_num,
+         h->cfg.topk_den, tau_guess, h->cand_n, fb, fb_total, h->work, h->work_count);
+  const long long items = (long long)P.ntiles * rows;
+  LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, h->work, h->work_count);
+  const long long hist_grid = 8LL * h->persistent_blocks;
   for (int level = 0; level < 3; ++level) {
-    LAUNCH(h, S_TOPK_HIST, k_topk_hist, (long long)P.ntiles * rows, P, rows, level, buf, h->sel, h->hist);
-    LAUNCH(h, S_TOPK_SELECT, k_topk_select, rows * P.T, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, h->hist,
-           h->sel, tau_out);
+    LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, buf, h->cand_n, h->sel, h->hist, h->work,
+           h->work_count);
+    LAUNCH(h, S_TOPK_SELECT, k_topk_select, pairs, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, h->hist, h->sel,
+           tau_out, h->work_count);
   }
+}
+
+CandArgs cand_args(sae_handle* h, bool server) {
+  CandArgs c;
+  c.keys = server ? h->cand_keys_srv : h->cand_keys;
+  c.off = h->d_cand_off; c.cap = h->d_cand_cap; c.stride = h->cand_stride;
+  c.count = server ? h->cand_count_srv : h->cand_count;
+  c.T = h->P.T;
+  return c;
 }
 
 constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
 
-template <int ESRC, bool SIGN, bool WRITE_D, bool WD>
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK>
 void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
   static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
   if (configured_device != h->device) {
-    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)kWorkerSmem);
     configured_device = h->device;
   }
@@ -170,13 +198,13 @@ void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa)
   if (h->P.K <= grid) grid -= grid % h->P.K;
   if (nitems < grid) grid = nitems;
   LaunchScope ls(h, S_WORKER);
-  k_worker_tma<ESRC, SIGN, WRITE_D, WD><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
+  k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
 }
 
-template <int ESRC, bool SIGN, bool WRITE_D>
+template <int ESRC, bool SIGN, bool WRITE_D, bool TOPK = false>
 void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
-  if (sp.wd) launch_worker_wd<ESRC, SIGN, WRITE_D, true>(h, sp, wa);
-  else launch_worker_wd<ESRC, SIGN, WRITE_D, false>(h, sp, wa);
+  if (sp.wd) launch_worker_wd<ESRC, SIGN, WRITE_D, true, TOPK>(h, sp, wa);
+  else launch_worker_wd<ESRC, SIGN, WRITE_D, false, TOPK>(h, sp, wa);
 }
 
 template <int COMP, int SRV>
@@ -261,9 +289,11 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = h->ebar; wa.x = h->x;
   wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
+  wa.cand = cand_args(h, false);
   ServerArgs sa;
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
   sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
+  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0;
   ApplyArgs aa;
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.m = h->m; aa.D = h->D;
   aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv; aa.tau_cur = h->tau[cur];
@@ -297,11 +327,11 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
     h->esrc = defer_avg ? ESRC_PENDING_AVG : (avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN);
   } else if (c.compressor == SAE_COMPRESSOR_TOPK) {
-    if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
-    else launch_worker<ESRC_LAZY_TOPK, false, true>(h, sp, wa);
-    topk_thresholds(h, h->D, P.K, h->tau[cur]);
+    if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
+    else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
+    topk_thresholds(h, h->D, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
     LAUNCH(h, S_SERVER, k_server_dense<2>, P.ntiles, P, sa);
-    if (dc) topk_thresholds(h, h->e_srv, 1, h->tau_srv);
+    if (dc) topk_thresholds(h, h->e_srv, 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
     const int avg = avg_after ? AVG_FROM_D : AVG_NONE;
     if (dc) launch_apply<2, 2>(h, avg, aa); else launch_apply<2, 0>(h, avg, aa);
     h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
@@ -483,6 +513,27 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   ALLOC0(h->recs, sign ? KT : 0); ALLOC0(h->recs_srv, sign ? T : 0);
   ALLOC0(h->hist, topk ? KT * HIST_BINS : 0);
   ALLOC0(h->sel, topk ? KT : 0);
+  std::vector<long long> cand_off(T, 0);
+  std::vector<int> cand_cap(T, 0);
+  h->cand_stride = 0;
+  if (topk) {
+    // room for 8 k_j + 1024 keys per (row, tensor): the window normally catches about 2 k_j
+    for (int j = 0; j < T; ++j) {
+      unsigned long long kk = ((unsigned long long)h->sizes[j] * cfg->topk_num) / cfg->topk_den;
+      if (kk < 1) kk = 1;
+      unsigned long long cap = 8 * kk + 1024;
+      if (cap > (unsigned long long)h->sizes[j]) cap = (unsigned long long)h->sizes[j];
+      cand_off[j] = h->cand_stride; cand_cap[j] = (int)cap;
+      h->cand_stride += (long long)((cap + 3) / 4 * 4);
+    }
+  }
+  ALLOC0(h->cand_keys, topk ? (size_t)K * h->cand_stride : 0);
+  ALLOC0(h->cand_keys_srv, topk ? (size_t)h->cand_stride : 0);
+  ALLOC0(h->cand_count, topk ? KT : 0); ALLOC0(h->cand_count_srv, topk ? T : 0);
+  ALLOC0(h->fb, topk ? KT : 0); ALLOC0(h->fb_srv, topk ? T : 0); ALLOC0(h->fb_total, 2);
+  ALLOC0(h->d_cand_off, T); ALLOC0(h->d_cand_cap, T);
+  ALLOC0(h->work, topk ? (size_t)ntiles * K + (size_t)K * (h->cand_stride / CAND_CHUNK + T) : 0);
+  ALLOC0(h->work_count, 1); ALLOC0(h->cand_n, topk ? KT : 0);
   ALLOC0(h->status, 1);
   TRY(cudaMallocHost((void**)&h->status_host, sizeof(u32)));
   TRY(cudaMemcpyAsync(h->d_tile_tensor, tile_tensor.data(), sizeof(int) * ntiles, cudaMemcpyHostToDevice, h->stream));
@@ -490,6 +541,8 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   TRY(cudaMemcpyAsync(h->d_n, n32.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
   TRY(cudaMemcpyAsync(h->d_off, off.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
   TRY(cudaMemcpyAsync(h->d_poff, poff.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_cand_off, cand_off.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_cand_cap, cand_cap.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
 #undef ALLOC0
   if (rc == SAE_OK) {
     Plan& P = h->P;
@@ -578,6 +631,7 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
     case SAE_STATE_WORKER_TAU: if (!topk) return SAE_ERR_INVALID_ARG; src = h->tau[h->last] + (size_t)worker * P.T; need = tb; break;
     case SAE_STATE_SERVER_TAU: if (!topk) return SAE_ERR_INVALID_ARG; src = h->tau_srv; need = tb; break;
     case SAE_STATE_SERVER_MASK: if (!topk) return SAE_ERR_INVALID_ARG; src = h->mask_srv; need = wb; break;
+    case SAE_STATE_TOPK_FALLBACKS: if (!topk) return SAE_ERR_INVALID_ARG; src = h->fb_total; need = 2 * sizeof(u32); break;
     case SAE_STATE_WORKER_MASK:
       if (!topk || bytes < wb) return SAE_ERR_INVALID_ARG;
       LAUNCH(h, S_MASK, k_mask_words, P.ntiles, P, h->D + (size_t)worker * P.dpad, h->tau[h->last] + (size_t)worker * P.T,

@@ -4,6 +4,7 @@
 // misaligned gradient rows take a lane-strided scalar path.  Both produce identical bits.
 #pragma once
 #include "sae_device.cuh"
+#include "sae_topk.cuh"
 
 namespace sae {
 
@@ -46,7 +47,8 @@ struct WorkerArgs {
   const float* ebar;      // [dpad]
   const float* x;         // [dpad]
   const float* scale_prev;  // [K][T]
-  const u32* tau_prev;      // [K][T]
+  const u32* tau_prev;      // [K][T] last step's thresholds (lazy error, and the guess of the candidate window)
+  CandArgs cand;            // Top-K candidate lists of the workers
   u32* words;             // [K][nwords]
   float* scale_cur;       // [K][T]
   L1Record* recs;         // [K][T]
@@ -64,6 +66,9 @@ struct ServerArgs {
   float* scale_srv;        // [T]
   L1Record* recs_srv;      // [T]
   u32* status;
+  CandArgs cand_srv;       // Top-K candidate list of the server (one row)
+  const u32* tau_srv_prev; // [T] last step's server thresholds: the guess of the server's window
+  int emit_srv;            // double-way Top-K: collect the server's candidates in this pass
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -145,8 +150,12 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
 template <int COMP>
 __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
+  __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
+  const bool emit = (COMP == 2) && A.emit_srv;
+  const u32 lo = emit ? window_lo(A.tau_srv_prev[ti.j]) : NO_GUESS;
+  WarpStage stg; stg.buf = cstage + ((COMP == 2) ? (tid >> 5) * CAND_STAGE : 0); stg.n = 0;
   if (COMP == 2) {
     for (int k = tid; k < P.K; k += THREADS) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
     __syncthreads();
@@ -176,20 +185,31 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       ds.z = __fadd_rn(e.z, __fdiv_rn(a2, Kf));
       ds.w = __fadd_rn(e.w, __fdiv_rn(a3, Kf));
       st4(ep + i, ds);
+      if (COMP == 2 && lo != NO_GUESS) {
+        if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand_srv, 0, ti.j);
+        stage_row4(stg, lo, mag_key(ds.x), mag_key(ds.y), mag_key(ds.z), mag_key(ds.w));
+      }
     }
   } else {
     for (int r = 0; r < ROWS; ++r) {
       const int i = r * THREADS + tid;
+      float ds = 0.0f;
       if (i < ti.cnt) {
         float a = 0.f;
         for (int k = 0; k < P.K; ++k) {
           const float v = dp[(long long)k * P.dpad + i];
           a = __fadd_rn(a, (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f);
         }
-        ep[i] = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+        ds = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+        ep[i] = ds;
+      }
+      if (COMP == 2 && lo != NO_GUESS) {
+        if (stg.n > CAND_STAGE - 32) stage_flush(stg, A.cand_srv, 0, ti.j);
+        stage_row1(stg, lo, i < ti.cnt, mag_key(ds));
       }
     }
   }
+  if (COMP == 2) stage_flush(stg, A.cand_srv, 0, ti.j);
 }
 
 // Between the worker pass and the server pass: one thread per (worker, tensor) record turns the exact
@@ -348,112 +368,6 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Top-K threshold: exact k-th largest 31-bit magnitude key per (row, tensor) by a three-level radix
-// select (11 + 10 + 10 bits).  Level L histograms the digit of every key whose higher digits equal the
-// prefix found so far; a select kernel then walks the histogram from the top.
-struct SelectState {     // per (row, tensor)
-  u32 prefix;            // digits found so far, right-aligned
-  u32 rank;              // rank (1-based, from the top) still to find inside the prefix bucket
-};
-
-constexpr int HIST_BINS = 2048;
-
-__device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* hist) {
-  if (level == 0) atomicAdd(hist + (key >> 20), 1u);
-  else if (level == 1) { if ((key >> 20) == prefix) atomicAdd(hist + ((key >> 10) & 1023u), 1u); }
-  else { if ((key >> 10) == prefix) atomicAdd(hist + (key & 1023u), 1u); }
-}
-
-// grid = ntiles * rows; buf is [rows][dpad]; hist is [rows][T][HIST_BINS]
-__global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, int rows, int level, const float* __restrict__ buf,
-                                                        const SelectState* __restrict__ st, u32* hist) {
-  __shared__ u32 sh[HIST_BINS];
-  const int tile = blockIdx.x / rows;
-  const int k = blockIdx.x - tile * rows;
-  const TileInfo ti = tile_info(P, tile);
-  const int tid = threadIdx.x;
-  const float* __restrict__ bp = buf + (long long)k * P.dpad + ti.poff + ti.t0;
-  u32* gh = hist + ((long long)k * P.T + ti.j) * HIST_BINS;
-  const u32 prefix = level ? st[(long long)k * P.T + ti.j].prefix : 0u;
-  if (level == 0) {
-    for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
-    __syncthreads();
-  }
-  u32* target = (level == 0) ? sh : gh;
-  if (ti.cnt == TILE) {
-#pragma unroll
-    for (int it = 0; it < VEC_ITERS; ++it) {
-      const float4 v = ld4(bp + it * (THREADS * 4) + tid * 4);
-      hist_elem(mag_key(v.x), level, prefix, target);
-      hist_elem(mag_key(v.y), level, prefix, target);
-      hist_elem(mag_key(v.z), level, prefix, target);
-      hist_elem(mag_key(v.w), level, prefix, target);
-    }
-  } else {
-    for (int i = tid; i < ti.cnt; i += THREADS) hist_elem(mag_key(bp[i]), level, prefix, target);
-  }
-  if (level == 0) {
-    __syncthreads();
-    for (int b = tid; b < HIST_BINS; b += THREADS) {
-      u32 c = sh[b];
-      if (c) atomicAdd(gh + b, c);
-    }
-  }
-}
-
-// One block per (row, tensor): find the bin holding the rank-th largest key, update prefix/rank, clear
-// the histogram.  After level 2 the prefix is the threshold key itself.
-__global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const int* __restrict__ n, u32 num, u32 den,
-                                                          u32* hist, SelectState* st, u32* tau) {
-  __shared__ u32 part[THREADS];
-  __shared__ u32 above[THREADS];
-  const int rj = blockIdx.x;              // row * T + j
-  const int j = rj % T;
-  const int tid = threadIdx.x;
-  const int bins = (level == 0) ? HIST_BINS : 1024;
-  const int per = bins / THREADS;         // 8 or 4
-  u32* gh = hist + (long long)rj * HIST_BINS;
-  u32 rank;
-  if (level == 0) {
-    unsigned long long kk = ((unsigned long long)n[j] * num) / den;
-    if (kk < 1) kk = 1;
-    if (kk > (unsigned long long)n[j]) kk = n[j];
-    rank = (u32)kk;
-  } else {
-    rank = st[rj].rank;
-  }
-  // thread t owns bins [hi - per*t - per + 1 .. hi - per*t] counted from the top
-  u32 c[8];
-  u32 sum = 0;
-  for (int q = 0; q < per; ++q) {
-    const int b = bins - 1 - (tid * per + q);
-    c[q] = gh[b];
-    gh[b] = 0u;
-    sum += c[q];
-  }
-  part[tid] = sum;
-  __syncthreads();
-  if (tid == 0) {
-    u32 run = 0;
-    for (int t = 0; t < THREADS; ++t) { above[t] = run; run += part[t]; }
-  }
-  __syncthreads();
-  u32 run = above[tid];
-  if (run < rank && rank <= run + sum) {
-    for (int q = 0; q < per; ++q) {
-      if (rank <= run + c[q]) {
-        const u32 b = (u32)(bins - 1 - (tid * per + q));
-        const u32 prefix = (level == 0) ? b : ((st[rj].prefix << 10) | b);
-        st[rj].prefix = prefix;
-        st[rj].rank = rank - run;
-        if (level == 2) tau[rj] = prefix;
-        break;
-      }
-      run += c[q];
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------------------
 // Layout conversion and getters (not on the hot path).
 constexpr int EXP_X = 0, EXP_ESRV = 1, EXP_M = 2, EXP_WERR = 3, EXP_STEP_AHEAD = 4;

@@ -50,6 +50,7 @@ struct WtItem {          // description of one work item, written by the produce
   int k, j, cnt, tiles_j, n, vec;
   float sprev;
   u32 tprev;
+  u32 lo;               // Top-K: lower edge of the candidate window (NO_GUESS: collect nothing)
 };
 
 struct WtSmem {
@@ -57,6 +58,7 @@ struct WtSmem {
   alignas(8) u64 full[WT_STAGES];
   alignas(8) u64 empty[WT_STAGES];
   WtItem item[WT_STAGES];
+  u32 cstage[WT_CONSUMER_WARPS][CAND_STAGE];   // Top-K: per-warp staging of candidate keys
 };
 
 __device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
@@ -168,11 +170,11 @@ __device__ __forceinline__ void warp_commit(const LaneAcc& a, L1Record* rec, u32
 }
 
 // Tile-table lookup of work item w (cnt = 0 marks "no such item").
-template <int ESRC>
+template <int ESRC, bool TOPK>
 __device__ __forceinline__ WtItem wt_lookup(const Plan& P, const WorkerArgs& A, long long w, long long nitems) {
   WtItem it;
   it.cnt = 0; it.vec = 0; it.gofs = 0; it.pbase = 0; it.wbase = 0; it.k = 0; it.j = 0; it.tiles_j = 0; it.n = 0;
-  it.sprev = 0.0f; it.tprev = 0u;
+  it.sprev = 0.0f; it.tprev = 0u; it.lo = NO_GUESS;
   if (w >= nitems) return it;
   const int tile = (int)(w / P.K);
   const int k = (int)(w - (long long)tile * P.K);
@@ -182,12 +184,13 @@ __device__ __forceinline__ WtItem wt_lookup(const Plan& P, const WorkerArgs& A, 
   it.wbase = (long long)k * P.dpad + it.pbase;
   it.k = k; it.j = ti.j; it.cnt = ti.cnt; it.tiles_j = ti.tiles_j; it.n = ti.n;
   if (ESRC == ESRC_LAZY_SIGN) it.sprev = A.scale_prev[(long long)k * P.T + ti.j];
-  if (ESRC == ESRC_LAZY_TOPK) it.tprev = A.tau_prev[(long long)k * P.T + ti.j];
+  if (ESRC == ESRC_LAZY_TOPK || TOPK) it.tprev = A.tau_prev[(long long)k * P.T + ti.j];
+  if (TOPK) it.lo = window_lo(it.tprev);
   it.vec = (ti.cnt == TILE) && ((reinterpret_cast<uintptr_t>(A.g + it.gofs) & 15) == 0);
   return it;
 }
 
-template <int ESRC, bool SIGN, bool WRITE_D, bool WD>
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK>
 __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma(Plan P, StepParams sp, WorkerArgs A,
                                                                                   long long nitems) {
   extern __shared__ unsigned char smem_raw[];
@@ -206,10 +209,10 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
     // one is being issued); the lanes then take turns, in item order, to publish and issue.
     const long long G = gridDim.x;
     long long wb = blockIdx.x;                               // first item of the current batch
-    WtItem nxt = wt_lookup<ESRC>(P, A, wb + lane * G, nitems);
+    WtItem nxt = wt_lookup<ESRC, TOPK>(P, A, wb + lane * G, nitems);
     for (int i0 = 0; wb < nitems; i0 += 32, wb += 32 * G) {
       const WtItem cur = nxt;
-      nxt = wt_lookup<ESRC>(P, A, wb + (32 + lane) * G, nitems);
+      nxt = wt_lookup<ESRC, TOPK>(P, A, wb + (32 + lane) * G, nitems);
       bool ok = true;
       for (int l = 0; l < 32; ++l) {
         if (lane == l && cur.cnt > 0) {
@@ -246,6 +249,9 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
   LaneAcc acc; lane_acc_init(acc);
   int acc_k = 0, acc_j = 0;
   u32 acc_items = 0;
+  // Top-K: candidate keys are staged per warp and appended to the (worker, tensor) list in batches
+  WarpStage stg; stg.buf = S.cstage[warp]; stg.n = 0;
+  int stg_k = 0, stg_j = 0;
   long long w = blockIdx.x;
   for (int i = 0; w < nitems; ++i, w += gridDim.x) {
     const int s = i % WT_STAGES;
@@ -257,6 +263,9 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
     float* __restrict__ mp = A.m + it.wbase;
     float* dp = A.D + it.wbase;
     u32* wp = A.words + (long long)it.k * P.nwords + (it.pbase >> 5);
+    if (TOPK) {
+      if (it.k != stg_k || it.j != stg_j) { stage_flush(stg, A.cand, stg_k, stg_j); stg_k = it.k; stg_j = it.j; }
+    }
     if (SIGN) {
       if (acc_items && (it.k != acc_k || it.j != acc_j)) {
         warp_commit(acc, A.recs + (long long)acc_k * P.T + acc_j, A.status);
@@ -285,6 +294,10 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
         dl.w = worker_update<WD>(G.w, M.w, prev_error<ESRC>(E.w, it.sprev, it.tprev), X.w, sp, mn.w);
         st4(mp + e0, mn);
         if (WRITE_D) st4(dp + e0, dl);
+        if (TOPK && it.lo != NO_GUESS) {
+          if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand, stg_k, stg_j);
+          stage_row4(stg, it.lo, mag_key(dl.x), mag_key(dl.y), mag_key(dl.z), mag_key(dl.w));
+        }
         if (SIGN) {
           lane_add4(acc, dl);
           const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
@@ -314,6 +327,10 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
           if (WRITE_D) dp[e0] = dl;
           if (SIGN) lane_add(acc, dl);
         }
+        if (TOPK && it.lo != NO_GUESS) {
+          if (stg.n > CAND_STAGE - 32) stage_flush(stg, A.cand, stg_k, stg_j);
+          stage_row1(stg, it.lo, valid, mag_key(dl));
+        }
         if (SIGN) {
           const u32 wd = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
           if (lane == 0 && (base + r * 32) < it.cnt) wp[(base + r * 32) >> 5] = wd;
@@ -322,6 +339,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
     }
   }
   if (SIGN && acc_items) warp_commit(acc, A.recs + (long long)acc_k * P.T + acc_j, A.status);
+  if (TOPK) stage_flush(stg, A.cand, stg_k, stg_j);
 }
 
 }  // namespace sae

@@ -76,6 +76,28 @@ def test_sign_aligned_rows_vector_path():
     run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.TOPK, 6, p=3)
 
 
+def test_topk_candidate_window_is_used_and_exact():
+    """Steady gradients: after the first steps the threshold of a step is found among the candidates
+    collected around the previous one (no extra pass over the data); every step stays exact."""
+    import torch
+    K, sizes, steps = 4, [20000, 3 * 4096, 100000, 700], 12
+    d = sum(sizes)
+    scales = synth.tensor_scales(5, len(sizes), -3.0, -2.0)
+    x0 = synth.x0_numpy(5, d)
+    orc = so.Oracle(K, sizes, x0, compressor=so.TOPK, avg_period=4, momentum=0.9, topk_num=1, topk_den=100, threads=4)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=sb.TOPK, avg_period=4, momentum=0.9, topk_num=1,
+                 topk_den=100)
+    for t in range(steps):
+        g = synth.grads_numpy(5, t, K, sizes, scales, 66, 100.0)
+        orc.step(g, 0.1)
+        gpu.step(torch.from_numpy(g).cuda(), 0.1)
+        compare_state(gpu, orc, so.TOPK, tag=f"window t={t + 1}")
+        compare_server_messages(gpu, orc, so.TOPK, 1, tag=f"window t={t + 1}")
+    fb = gpu.get_state(sb.STATE_TOPK_FALLBACKS).cpu().numpy()
+    assert K * len(sizes) <= fb[0] < K * len(sizes) * steps // 2, fb      # the first step always falls back
+    assert len(sizes) <= fb[1] < len(sizes) * steps // 2, fb
+
+
 def test_topk_ties_and_zeros():
     """Gradients quantised to a few levels: many exact ties at the threshold and exact zeros."""
     import torch
