@@ -69,6 +69,25 @@ def test_identity(K):
     run_pair(K, RAGGED, so.IDENTITY, 5, p=2, lam=1e-3)
 
 
+@pytest.mark.parametrize("K", [5, 40, 64])
+def test_worker_counts_outside_the_folded_path(K):
+    """K not a power of two, or above 32: p = 1 runs the plain worker pass and averages in the apply kernel."""
+    run_pair(K, [33, 4096, 5000, 700], so.SIGN, 4, p=1, seed=4)
+    run_pair(K, [33, 4096, 5000, 700], so.TOPK, 3, p=1, num=1, den=20, seed=4)
+
+
+def test_single_large_ragged_tensor():
+    """One tensor over many tiles whose size is not a multiple of 4 (ragged last row, odd gradient rows)."""
+    run_pair(2, [9 * 4096 + 1235], so.SIGN, 5, p=1)
+    run_pair(4, [9 * 4096 + 1235], so.SIGN, 5, p=2)
+    run_pair(2, [9 * 4096 + 1235], so.TOPK, 5, p=2, num=1, den=50)
+
+
+def test_topk_keep_everything():
+    """num = den: k = n, Top-K is the identity except that exact zeros are never 'selected'."""
+    run_pair(2, [100, 4096, 5000], so.TOPK, 4, p=2, num=1, den=1)
+
+
 def test_sign_aligned_rows_vector_path():
     """d a multiple of 4 and tensors of whole tiles: every tile takes the 128-bit path."""
     run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.SIGN, 6, p=1)
