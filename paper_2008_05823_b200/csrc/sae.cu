@@ -546,7 +546,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
 #undef ALLOC0
   if (rc == SAE_OK) {
     Plan& P = h->P;
-    P.K = K; P.T = T; P.ntiles = (int)ntiles; P.d = d; P.dpad = dpad; P.nwords = nwords;
+    P.K = K; P.T = T; P.k_pow2 = ((K & (K - 1)) == 0) ? 1 : 0; P.inv_k = 1.0f / (float)K; P.ntiles = (int)ntiles; P.d = d; P.dpad = dpad; P.nwords = nwords;
     P.tile_tensor = h->d_tile_tensor; P.first_tile = h->d_first_tile; P.n = h->d_n; P.off = h->d_off; P.poff = h->d_poff;
     LAUNCH(h, S_IMPORT, k_import, P.ntiles, P, x0, h->x);
     TRY(cudaGetLastError());

@@ -28,6 +28,8 @@ constexpr u32 STATUS_RANGE = 1u;  // a model difference was non-finite or >= 2^3
 // tensor start is 128-byte aligned and owns whole bit words; padding elements stay zero.
 struct Plan {
   int K, T;
+  int k_pow2;            // K is a power of two: dividing by K is the exact multiplication by inv_k (same bits)
+  float inv_k;           // 1 / K (exact when k_pow2)
   int ntiles;            // tiles over all tensors
   long long d;           // sum n_j (caller layout length)
   long long dpad;        // padded length, multiple of 32
@@ -58,6 +60,12 @@ __device__ __forceinline__ TileInfo tile_info(const Plan& P, int tile) {
   ti.off = P.off[ti.j];
   ti.poff = P.poff[ti.j];
   return ti;
+}
+
+// acc / (float)K, one correctly rounded operation.  For a power-of-two K the product with 2^-log2(K) is the
+// same real number as the quotient, so the cheaper multiply gives identical bits (denormals included).
+__device__ __forceinline__ float div_by_k(const Plan& P, float a) {
+  return P.k_pow2 ? __fmul_rn(a, P.inv_k) : __fdiv_rn(a, (float)P.K);
 }
 
 // ---- streaming loads/stores ------------------------------------------------------------------------
@@ -129,6 +137,61 @@ __device__ __forceinline__ void acc_block_reduce(Acc128& a, u64* sh) {
     for (int w = 0; w < NW; ++w) { acc_add_u(r, sh[w], sh[NW + w]); r.bad |= (u32)sh[2 * NW + w]; }
     a = r;
   }
+}
+
+// Per-lane L1 accumulator of the streaming passes: a 96-bit sum (lo0, lo1, carry) fed by a three-instruction
+// carry chain, plus a 64-bit word for the integer parts of the rare values >= 1.
+struct LaneAcc {
+  u32 lo0, lo1, carry;
+  u64 hi;
+  u32 bad;
+};
+
+__device__ __forceinline__ void lane_acc_init(LaneAcc& a) { a.lo0 = 0; a.lo1 = 0; a.carry = 0; a.hi = 0; a.bad = 0; }
+
+// += floor(m 2^64) for 0 <= m < 1 (exact: power-of-two scaling, then a round-down conversion)
+__device__ __forceinline__ void lane_add_small(LaneAcc& a, float m) {
+  const u64 f = __float2ull_rd(__fmul_rn(m, 18446744073709551616.0f));
+  const u32 f0 = (u32)f, f1 = (u32)(f >> 32);
+  asm("add.cc.u32 %0, %0, %3;\n\taddc.cc.u32 %1, %1, %4;\n\taddc.u32 %2, %2, 0;"
+      : "+r"(a.lo0), "+r"(a.lo1), "+r"(a.carry)
+      : "r"(f0), "r"(f1));
+}
+
+// any magnitude: the general (rare) path splits off the integer part, non-finite / >= 2^32 flags RANGE
+__device__ __forceinline__ void lane_add(LaneAcc& a, float v) {
+  const float m = fabsf(v);
+  if (m < 1.0f) {
+    lane_add_small(a, m);
+  } else if (m < 4294967296.0f) {
+    const float ip = floorf(m);
+    lane_add_small(a, __fsub_rn(m, ip));
+    a.hi += __float2ull_rd(ip);
+  } else {
+    a.bad = 1u;
+  }
+}
+
+// Four values at once: one test decides whether all of them are below 1 (the bit pattern of |v| orders
+// magnitudes and puts NaN / Inf above every finite value), so the common case has no per-element branch.
+__device__ __forceinline__ void lane_add4(LaneAcc& a, float4 v) {
+  const u32 k0 = __float_as_uint(v.x) & 0x7fffffffu, k1 = __float_as_uint(v.y) & 0x7fffffffu;
+  const u32 k2 = __float_as_uint(v.z) & 0x7fffffffu, k3 = __float_as_uint(v.w) & 0x7fffffffu;
+  if (max(max(k0, k1), max(k2, k3)) < 0x3f800000u) {
+    lane_add_small(a, __uint_as_float(k0)); lane_add_small(a, __uint_as_float(k1));
+    lane_add_small(a, __uint_as_float(k2)); lane_add_small(a, __uint_as_float(k3));
+  } else {
+    lane_add(a, v.x); lane_add(a, v.y); lane_add(a, v.z); lane_add(a, v.w);
+  }
+}
+
+// the lane's sum as a 128-bit value
+__device__ __forceinline__ Acc128 lane_acc_total(const LaneAcc& a) {
+  Acc128 r;
+  r.lo = ((u64)a.lo1 << 32) | a.lo0;
+  r.hi = a.hi + a.carry;
+  r.bad = a.bad;
+  return r;
 }
 
 // The per-(row, tensor) accumulator in global memory: three 43-bit limbs in 64-bit words (21 bits of

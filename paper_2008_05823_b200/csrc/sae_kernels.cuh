@@ -105,10 +105,10 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
         a3 = __fadd_rn(a3, (w & 8u) ? s : -s);
       }
       float4 ds;
-      ds.x = __fadd_rn(e.x, __fdiv_rn(a0, Kf));
-      ds.y = __fadd_rn(e.y, __fdiv_rn(a1, Kf));
-      ds.z = __fadd_rn(e.z, __fdiv_rn(a2, Kf));
-      ds.w = __fadd_rn(e.w, __fdiv_rn(a3, Kf));
+      ds.x = __fadd_rn(e.x, div_by_k(P, a0));
+      ds.y = __fadd_rn(e.y, div_by_k(P, a1));
+      ds.z = __fadd_rn(e.z, div_by_k(P, a2));
+      ds.w = __fadd_rn(e.w, div_by_k(P, a3));
       st4(ep + i, ds);
       if (DC) {
         acc_add(acc, ds.x); acc_add(acc, ds.y); acc_add(acc, ds.z); acc_add(acc, ds.w);
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
           const float s = s_k[k];
           a = __fadd_rn(a, (w & 1u) ? s : -s);
         }
-        ds = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+        ds = __fadd_rn(ep[i], div_by_k(P, a));
         ep[i] = ds;
         if (DC) acc_add(acc, ds);
       }
@@ -180,10 +180,10 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
         a3 = __fadd_rn(a3, (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f);
       }
       float4 ds;
-      ds.x = __fadd_rn(e.x, __fdiv_rn(a0, Kf));
-      ds.y = __fadd_rn(e.y, __fdiv_rn(a1, Kf));
-      ds.z = __fadd_rn(e.z, __fdiv_rn(a2, Kf));
-      ds.w = __fadd_rn(e.w, __fdiv_rn(a3, Kf));
+      ds.x = __fadd_rn(e.x, div_by_k(P, a0));
+      ds.y = __fadd_rn(e.y, div_by_k(P, a1));
+      ds.z = __fadd_rn(e.z, div_by_k(P, a2));
+      ds.w = __fadd_rn(e.w, div_by_k(P, a3));
       st4(ep + i, ds);
       if (COMP == 2 && lo != NO_GUESS) {
         if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand_srv, 0, ti.j);
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
           const float v = dp[(long long)k * P.dpad + i];
           a = __fadd_rn(a, (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f);
         }
-        ds = __fadd_rn(ep[i], __fdiv_rn(a, Kf));
+        ds = __fadd_rn(ep[i], div_by_k(P, a));
         ep[i] = ds;
       }
       if (COMP == 2 && lo != NO_GUESS) {
@@ -335,7 +335,7 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
           a2 = __fadd_rn(a2, worker_err<COMP>(v.z, s, t));
           a3 = __fadd_rn(a3, worker_err<COMP>(v.w, s, t));
         }
-        st4(ebp + i, make_float4(__fdiv_rn(a0, Kf), __fdiv_rn(a1, Kf), __fdiv_rn(a2, Kf), __fdiv_rn(a3, Kf)));
+        st4(ebp + i, make_float4(div_by_k(P, a0), div_by_k(P, a1), div_by_k(P, a2), div_by_k(P, a3)));
       }
     }
   } else {
@@ -356,7 +356,7 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
             if (AVG == AVG_RECOMPUTE) v = __fmaf_rn(A.eta, v, eb);
             a = __fadd_rn(a, worker_err<COMP>(v, (COMP == 1) ? s_k[k] : 0.0f, (COMP == 2) ? t_k[k] : 0u));
           }
-          ebp[i] = __fdiv_rn(a, Kf);
+          ebp[i] = div_by_k(P, a);
         }
       }
       if (SRV == 2) {

@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 #pragma unroll
             for (int v = 0; v < V; ++v) {
               if (e0 + v < it.cnt) {
-                const float en = __fdiv_rn(a[v], Kf);
+                const float en = div_by_k(P, a[v]);
                 se[e0 + v] = en;
                 A.ebar[it.pbase + e0 + v] = en;
               }
@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(THREADS) k_materialize_avg(Plan P, const float
       const float dk = __fmaf_rn(eta_prev, m[(long long)k * P.dpad + p], eb);
       a = __fadd_rn(a, __fsub_rn(dk, sign_code(dk, scale_prev[(long long)k * P.T + ti.j])));
     }
-    etmp[p] = __fdiv_rn(a, Kf);
+    etmp[p] = div_by_k(P, a);
   }
 }
 

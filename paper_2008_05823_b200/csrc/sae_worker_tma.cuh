@@ -96,52 +96,6 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes,
                : "memory");
 }
 
-// Per-lane L1 accumulator of the worker pass: a 96-bit sum (lo0, lo1, carry) fed by a three-instruction
-// carry chain, plus a 64-bit word for the integer parts of the rare values >= 1.
-struct LaneAcc {
-  u32 lo0, lo1, carry;
-  u64 hi;
-  u32 bad;
-};
-
-__device__ __forceinline__ void lane_acc_init(LaneAcc& a) { a.lo0 = 0; a.lo1 = 0; a.carry = 0; a.hi = 0; a.bad = 0; }
-
-// += floor(m 2^64) for 0 <= m < 1 (exact: power-of-two scaling, then a round-down conversion)
-__device__ __forceinline__ void lane_add_small(LaneAcc& a, float m) {
-  const u64 f = __float2ull_rd(__fmul_rn(m, 18446744073709551616.0f));
-  const u32 f0 = (u32)f, f1 = (u32)(f >> 32);
-  asm("add.cc.u32 %0, %0, %3;\n\taddc.cc.u32 %1, %1, %4;\n\taddc.u32 %2, %2, 0;"
-      : "+r"(a.lo0), "+r"(a.lo1), "+r"(a.carry)
-      : "r"(f0), "r"(f1));
-}
-
-// any magnitude: the general (rare) path splits off the integer part, non-finite / >= 2^32 flags RANGE
-__device__ __forceinline__ void lane_add(LaneAcc& a, float v) {
-  const float m = fabsf(v);
-  if (m < 1.0f) {
-    lane_add_small(a, m);
-  } else if (m < 4294967296.0f) {
-    const float ip = floorf(m);
-    lane_add_small(a, __fsub_rn(m, ip));
-    a.hi += __float2ull_rd(ip);
-  } else {
-    a.bad = 1u;
-  }
-}
-
-// Four values at once: one test decides whether all of them are below 1 (the bit pattern of |v| orders
-// magnitudes and puts NaN / Inf above every finite value), so the common case has no per-element branch.
-__device__ __forceinline__ void lane_add4(LaneAcc& a, float4 v) {
-  const u32 k0 = __float_as_uint(v.x) & 0x7fffffffu, k1 = __float_as_uint(v.y) & 0x7fffffffu;
-  const u32 k2 = __float_as_uint(v.z) & 0x7fffffffu, k3 = __float_as_uint(v.w) & 0x7fffffffu;
-  if (max(max(k0, k1), max(k2, k3)) < 0x3f800000u) {
-    lane_add_small(a, __uint_as_float(k0)); lane_add_small(a, __uint_as_float(k1));
-    lane_add_small(a, __uint_as_float(k2)); lane_add_small(a, __uint_as_float(k3));
-  } else {
-    lane_add(a, v.x); lane_add(a, v.y); lane_add(a, v.z); lane_add(a, v.w);
-  }
-}
-
 // Warp-level sum of the lanes' 128-bit partials, added by lane 0 to the (worker, tensor) record.
 // The low 64 bits are split into 22-bit pieces so that a 32-lane sum fits a 32-bit redux add; the
 // high word (almost always a small carry count) takes one more redux, or a shuffle tree if large.

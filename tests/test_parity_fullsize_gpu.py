@@ -28,6 +28,14 @@ def sample_tensors(sizes, budget):
 
 
 def run_fullsize(idx, p, steps, budget, seed=0):
+    """Runs on a non-default stream, as bench.py does: the steps are captured and replayed as CUDA graphs."""
+    import torch
+    with torch.cuda.stream(torch.cuda.Stream()):
+        _run_fullsize(idx, p, steps, budget, seed)
+    torch.cuda.synchronize()
+
+
+def _run_fullsize(idx, p, steps, budget, seed):
     import psutil
     import torch
     w = configs.workload(idx)
@@ -47,9 +55,10 @@ def run_fullsize(idx, p, steps, budget, seed=0):
     orc = so.Oracle(K, sub_sizes, x0_sub, compressor=w.compressor, avg_period=p, momentum=w.momentum,
                     weight_decay=w.weight_decay, topk_num=w.topk_num, topk_den=w.topk_den, threads=so.max_threads())
     idx_sub = torch.from_numpy(np.concatenate([np.arange(offs[j], offs[j + 1]) for j in js])).cuda()
-    g = torch.empty(K, d, device="cuda")
+    gbuf = [torch.empty(K, d, device="cuda") for _ in range(2)]     # two buffers, as the bench's ring: graph keys repeat
     take = lambda t: t[idx_sub].cpu().numpy()
     for t in range(steps):
+        g = gbuf[t % 2]
         gen.grads(g, K, seed, t, w.outlier_per_65536, w.outlier_mult)
         gpu.step(g, w.lr)
         g_sub = np.stack([np.concatenate([synth.grads_numpy_range(seed, t, k, int(offs[j]), sizes[j], scales[j],
