@@ -293,7 +293,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   ServerArgs sa;
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
   sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
-  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0;
+  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = h->ebar;
   ApplyArgs aa;
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.m = h->m; aa.D = h->D;
   aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv; aa.tau_cur = h->tau[cur];
@@ -330,15 +330,16 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
     else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
     topk_thresholds(h, h->D, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
-    LAUNCH(h, S_SERVER, k_server_dense<2>, P.ntiles, P, sa);
+    // the averaged error (if the pre-step averages) comes out of the same pass over D as the server's sum
+    if (avg_after) LAUNCH(h, S_SERVER, (k_server_dense<2, true>), P.ntiles, P, sa);
+    else LAUNCH(h, S_SERVER, (k_server_dense<2, false>), P.ntiles, P, sa);
     if (dc) topk_thresholds(h, h->e_srv, 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
-    const int avg = avg_after ? AVG_FROM_D : AVG_NONE;
-    if (dc) launch_apply<2, 2>(h, avg, aa); else launch_apply<2, 0>(h, avg, aa);
+    if (dc) launch_apply<2, 2>(h, AVG_NONE, aa); else launch_apply<2, 0>(h, AVG_NONE, aa);
     h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
   } else {
     // identity: every error stays exactly zero, so e^(k) is the (all-zero) uniform vector forever
     launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
-    LAUNCH(h, S_SERVER, k_server_dense<0>, P.ntiles, P, sa);
+    LAUNCH(h, S_SERVER, (k_server_dense<0, false>), P.ntiles, P, sa);
     launch_apply<0, 0>(h, AVG_NONE, aa);
     h->esrc = ESRC_UNIFORM;
   }

@@ -69,6 +69,7 @@ struct ServerArgs {
   CandArgs cand_srv;       // Top-K candidate list of the server (one row)
   const u32* tau_srv_prev; // [T] last step's server thresholds: the guess of the server's window
   int emit_srv;            // double-way Top-K: collect the server's candidates in this pass
+  float* ebar;             // [dpad] averaged local error (dense variants, when the pre-step averages)
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -147,7 +148,10 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
 
 // K3 (identity / Top-K): the same aggregation from the dense model differences.
 // COMP 0: C = identity, 2: Top-K with this step's thresholds.
-template <int COMP>
+// AVG: the next pre-step averages the local errors; they are functions of the same D^(k) and thresholds
+// this pass already reads, so ebar = (1/K) sum_k (D^(k) - C(D^(k))) is formed here, in k order, instead of
+// in a further pass over D.
+template <int COMP, bool AVG>
 __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
@@ -170,15 +174,22 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       const int i = it * (THREADS * 4) + tid * 4;
       const float4 e = ld4(ep + i);
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
 #pragma unroll 4
       for (int k = 0; k < P.K; ++k) {
         const float4 v = ld4(dp + (long long)k * P.dpad + i);
         const u32 t = (COMP == 2) ? t_k[k] : 0u;
-        a0 = __fadd_rn(a0, (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f);
-        a1 = __fadd_rn(a1, (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f);
-        a2 = __fadd_rn(a2, (COMP == 0 || topk_selected(v.z, t)) ? v.z : 0.0f);
-        a3 = __fadd_rn(a3, (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f);
+        const float c0 = (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f;
+        const float c1 = (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f;
+        const float c2 = (COMP == 0 || topk_selected(v.z, t)) ? v.z : 0.0f;
+        const float c3 = (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f;
+        a0 = __fadd_rn(a0, c0); a1 = __fadd_rn(a1, c1); a2 = __fadd_rn(a2, c2); a3 = __fadd_rn(a3, c3);
+        if (AVG) {
+          b0 = __fadd_rn(b0, __fsub_rn(v.x, c0)); b1 = __fadd_rn(b1, __fsub_rn(v.y, c1));
+          b2 = __fadd_rn(b2, __fsub_rn(v.z, c2)); b3 = __fadd_rn(b3, __fsub_rn(v.w, c3));
+        }
       }
+      if (AVG) st4(A.ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
       float4 ds;
       ds.x = __fadd_rn(e.x, div_by_k(P, a0));
       ds.y = __fadd_rn(e.y, div_by_k(P, a1));
@@ -195,11 +206,14 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       const int i = r * THREADS + tid;
       float ds = 0.0f;
       if (i < ti.cnt) {
-        float a = 0.f;
+        float a = 0.f, b = 0.f;
         for (int k = 0; k < P.K; ++k) {
           const float v = dp[(long long)k * P.dpad + i];
-          a = __fadd_rn(a, (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f);
+          const float c = (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f;
+          a = __fadd_rn(a, c);
+          if (AVG) b = __fadd_rn(b, __fsub_rn(v, c));
         }
+        if (AVG) A.ebar[pbase + i] = div_by_k(P, b);
         ds = __fadd_rn(ep[i], div_by_k(P, a));
         ep[i] = ds;
       }
