@@ -118,14 +118,23 @@ __device__ __forceinline__ void walk_from_top(u32* hist, int bins, u32 rank, u32
     hist[b] = 0u;
     sum += c[q];
   }
-  part[tid] = sum;
+  // exclusive prefix sum of the per-thread sums over the block: shuffle scan inside each warp, then the
+  // warp totals
+  const int lane = tid & 31, wrp = tid >> 5;
+  u32 inc = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const u32 v = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += v;
+  }
+  if (lane == 31) part[wrp] = inc;
   __syncthreads();
   if (tid == 0) {
     u32 run = 0;
-    for (int t = 0; t < THREADS; ++t) { above[t] = run; run += part[t]; }
+    for (int t = 0; t < THREADS / 32; ++t) { above[t] = run; run += part[t]; }
   }
   __syncthreads();
-  u32 run = above[tid];
+  u32 run = above[wrp] + inc - sum;
   if (run < rank && rank <= run + sum) {
     for (int q = 0; q < per; ++q) {
       if (rank <= run + c[q]) {
@@ -181,8 +190,9 @@ __device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* h
   else { if ((key >> 10) == prefix) atomicAdd(hist + (key & 1023u), 1u); }
 }
 
-// Level L histogram over the work list (a fixed grid of blocks strides over it).  Level 0 accumulates
-// in shared memory first; the deeper levels touch few keys and add to global memory directly.
+// Level L histogram over the work list (a fixed grid of blocks strides over it).  Every item accumulates
+// in shared memory first (the candidates of a pair nearly all share their leading digits, so direct
+// global atomics would pile up on a few addresses) and adds its non-zero bins to the pair's histogram.
 // buf is [rows][dpad]; hist is [rows][T][HIST_BINS]
 __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int rows, int level, const float* __restrict__ buf,
                                                         const u32* __restrict__ cand_n, const SelectState* __restrict__ st,
@@ -194,10 +204,9 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
   for (u32 q = blockIdx.x; q < nwork; q += gridDim.x) {
     const int2 w = work[q];
     int rj;
-    if (level == 0) {
-      for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
-      __syncthreads();
-    }
+    const int bins = level == 0 ? HIST_BINS : 1024;
+    for (int b = tid; b < bins; b += THREADS) sh[b] = 0u;
+    __syncthreads();
     if (w.y < 0) {
       const int tile = w.x / rows;
       const int k = w.x - tile * rows;
@@ -205,7 +214,7 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
       rj = k * P.T + ti.j;
       const float* __restrict__ bp = buf + (long long)k * P.dpad + ti.poff + ti.t0;
       const u32 prefix = level ? st[rj].prefix : 0u;
-      u32* target = (level == 0) ? sh : hist + (long long)rj * HIST_BINS;
+      u32* target = sh;
       if (ti.cnt == TILE) {
 #pragma unroll
         for (int it = 0; it < VEC_ITERS; ++it) {
@@ -224,18 +233,16 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
       const u32* __restrict__ keys = C.keys + (long long)row * C.stride + C.off[j] + (long long)w.y * CAND_CHUNK;
       const int cnt = min((int)(cand_n[rj] - (u32)w.y * CAND_CHUNK), CAND_CHUNK);
       const u32 prefix = level ? st[rj].prefix : 0u;
-      u32* target = (level == 0) ? sh : hist + (long long)rj * HIST_BINS;
+      u32* target = sh;
       for (int i = tid; i < cnt; i += THREADS) hist_elem(keys[i], level, prefix, target);
     }
-    if (level == 0) {
-      __syncthreads();
-      u32* gh = hist + (long long)rj * HIST_BINS;
-      for (int b = tid; b < HIST_BINS; b += THREADS) {
-        const u32 c = sh[b];
-        if (c) atomicAdd(gh + b, c);
-      }
-      __syncthreads();
+    __syncthreads();
+    u32* gh = hist + (long long)rj * HIST_BINS;
+    for (int b = tid; b < bins; b += THREADS) {
+      const u32 c = sh[b];
+      if (c) atomicAdd(gh + b, c);
     }
+    __syncthreads();
   }
 }
 
