@@ -116,8 +116,9 @@ def cpu_baseline(w, avg_period, seed, steps, warmup, target_elems=40_000_000):
     scales = synth.workload_scales(w, seed)
     threads = max(1, min(so.max_threads(), len(os.sched_getaffinity(0))))
     x0 = np.concatenate([synth.x0_numpy_range(seed, int(offs[j]), sizes[j]) for j in js])
-    orc = so.Oracle(K, sub, x0, compressor=w.compressor, avg_period=avg_period, momentum=w.momentum,
-                    weight_decay=w.weight_decay, topk_num=w.topk_num, topk_den=w.topk_den, threads=threads)
+    orc = so.Oracle(K, sub, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
+                    avg_period=avg_period, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
+                    topk_den=w.topk_den, threads=threads)
     grads = [np.stack([np.concatenate([synth.grads_numpy_range(seed, t, k, int(offs[j]), sizes[j], scales[j],
                                                                w.outlier_per_65536, w.outlier_mult) for j in js])
                        for k in range(K)]) for t in range(2)]
@@ -199,6 +200,11 @@ def main():
     ap.add_argument("--ring", type=int, default=0, help="gradient sets kept in HBM (0 = auto)")
     ap.add_argument("--workers", type=int, default=0,
                     help="override the workload's worker count (smaller cases of the same kernels for ncu captures)")
+    # the paper's variant grid "(EF,SAEF)-(SGD,SGDM,SignSGD,SignSGDM)-(SC,DC)-(TopK)" on the same kernels
+    ap.add_argument("--mode", choices=["saef", "ef"], default=None, help="step-ahead or plain local error feedback")
+    ap.add_argument("--single-way", action="store_true", help="server sends its Delta uncompressed (SC)")
+    ap.add_argument("--momentum", type=float, default=None, help="0 gives the SGD / SignSGD variants")
+    ap.add_argument("--topk-percent", type=float, default=None, help="Top-K sparsity in percent (Table 1: 1, 5, 10)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -209,6 +215,19 @@ def main():
     if args.workers > 0:
         w.num_workers = args.workers
         w.name += f"_workers{args.workers}"
+    if args.mode is not None:
+        w.mode = configs.SAEF if args.mode == "saef" else configs.EF
+        w.name += f"_{args.mode}"
+    if args.single_way:
+        w.server_compress = 0
+        w.name += "_sc"
+    if args.momentum is not None:
+        w.momentum = args.momentum
+        w.name += f"_mu{args.momentum:g}"
+    if args.topk_percent is not None:
+        w.compressor = configs.TOPK
+        w.topk_num, w.topk_den = int(round(args.topk_percent * 10)), 1000
+        w.name += f"_top{args.topk_percent:g}pct"
     p = args.avg_period
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -347,6 +366,9 @@ def main():
                 "config": {"workload": w.name, "num_workers": K, "d": d, "num_tensors": w.num_tensors,
                            "compressor": {0: "identity", 1: "scaled_sign", 2: "topk"}[w.compressor],
                            "avg_period": p, "momentum": w.momentum, "lr": w.lr, "weight_decay": w.weight_decay,
+                           "mode": "saef" if w.mode == configs.SAEF else "ef",
+                           "server_compress": "double-way" if w.server_compress else "single-way",
+                           "topk": f"{w.topk_num}/{w.topk_den}" if w.compressor == configs.TOPK else None,
                            "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
                            "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient set "
                                  f"(ring of {ring})"},
