@@ -138,6 +138,26 @@ int sae_get_state(sae_handle *h, int32_t which, int32_t worker, void *out, size_
  * 1 <-> selected; padding bits 0; the tensors' word arrays concatenated in list order.
  */
 
+/*
+ * Checkpoint / resume.  sae_save_state copies everything later steps and getters depend on (x, e, m^(k),
+ * the held form of e^(k), last scales / thresholds / messages, t, the last learning rate) into `out`
+ * (DEVICE buffer of at least sae_state_bytes(h) bytes; stream-ordered except for a short synchronisation).
+ * sae_load_state restores it into a handle created with the SAME configuration (anything else is
+ * SAE_ERR_INVALID_ARG); the run then continues bit for bit as the saved one would have.
+ */
+int64_t sae_state_bytes(sae_handle *h);
+int sae_save_state(sae_handle *h, void *out, size_t bytes);
+int sae_load_state(sae_handle *h, const void *in, size_t bytes);
+
+/*
+ * Gradient-mismatch bounds of Section 3 (Fig. 3, right; the factors L^2 and the sigma^2 term are left out),
+ * for the current errors, with ebar = (1/K) sum_k e^(k):
+ *   out_host[0] = || e + ebar ||^2                         -- local error feedback
+ *   out_host[1] = (1/K) sum_k || e + ebar - e^(k) ||^2      -- step ahead
+ * accumulated in fp64 on the device.  out_host: HOST, 2 doubles.  Synchronises the stream.
+ */
+int sae_get_mismatch(sae_handle *h, double *out_host);
+
 /* Number of iterations performed so far (t). */
 int64_t sae_iteration(const sae_handle *h);
 /* d = sum n_j, and the number of bit words per worker, sum_j ceil(n_j/32). */

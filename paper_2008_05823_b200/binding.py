@@ -23,7 +23,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsae.so")
 EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_params_host", "sae_get_step_ahead",
            "sae_get_state", "sae_iteration", "sae_num_params", "sae_num_words", "sae_sync", "sae_set_profiling",
            "sae_get_kernel_times", "sae_kernel_name", "sae_kernel_launches", "sae_destroy", "sae_strerror",
-           "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements"]
+           "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements", "sae_state_bytes",
+           "sae_save_state", "sae_load_state", "sae_get_mismatch"]
 
 
 class SaeConfig(C.Structure):
@@ -74,6 +75,11 @@ def lib():
         L.sae_strerror.argtypes = [C.c_int]
         L.sae_strerror.restype = C.c_char_p
         L.sae_last_cuda_error.argtypes = [vp]
+        L.sae_state_bytes.argtypes = [vp]
+        L.sae_state_bytes.restype = i64
+        L.sae_save_state.argtypes = [vp, vp, C.c_size_t]
+        L.sae_load_state.argtypes = [vp, vp, C.c_size_t]
+        L.sae_get_mismatch.argtypes = [vp, vp]
         L.sae_sign_compress_noalloc.argtypes = [vp, i64, vp, vp, vp, vp]
         L.sae_noalloc_max_elements.argtypes = []
         L.sae_noalloc_max_elements.restype = i64
@@ -169,6 +175,20 @@ class Sae:
         _check(lib().sae_get_state(self.h, which, worker, out.data_ptr(), out.numel() * out.element_size()),
                "sae_get_state", self.h)
         return out
+
+    def save_state(self):
+        t = self.torch
+        blob = t.empty(int(lib().sae_state_bytes(self.h)), dtype=t.uint8, device=self.device)
+        _check(lib().sae_save_state(self.h, blob.data_ptr(), blob.numel()), "sae_save_state", self.h)
+        return blob
+
+    def load_state(self, blob):
+        _check(lib().sae_load_state(self.h, blob.data_ptr(), blob.numel()), "sae_load_state", self.h)
+
+    def get_mismatch(self):
+        out = (C.c_double * 2)()
+        _check(lib().sae_get_mismatch(self.h, out), "sae_get_mismatch", self.h)
+        return float(out[0]), float(out[1])
 
     @property
     def iteration(self):

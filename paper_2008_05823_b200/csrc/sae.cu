@@ -61,6 +61,7 @@ struct sae_handle {
   u32* status_host;      // pinned
   float* staging;        // sae_step_host
   float* out_stage;      // sae_get_params_host
+  double* mismatch;      // sae_get_mismatch
   int64_t t;
   int esrc;              // how e^(k) is held now (ESRC_*)
   int fused_ok;          // p = 1, scaled sign, K a power of two <= 32: averaging is folded into the next worker pass
@@ -143,7 +144,7 @@ cudaError_t dalloc(T** p, size_t count) {
 void free_all(sae_handle* h) {
   void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
-                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage,
+                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -412,20 +413,61 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   return SAE_OK;
 }
 
-int export_vec(sae_handle* h, int what, int k, float* out) {
+ExportArgs export_args(sae_handle* h, int what, int k, bool need_error) {
   ExportArgs ea;
   ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = h->ebar;
   ea.scale_last = h->scale[h->last]; ea.tau_last = h->tau[h->last];
   ea.esrc = h->esrc; ea.what = what; ea.k = k; ea.saef = (h->cfg.mode == SAE_MODE_SAEF);
   if (h->esrc == ESRC_PENDING_AVG) {
     // the averaged error exists only implicitly: form it in a scratch vector, leave the state alone
-    if (what == EXP_WERR || what == EXP_STEP_AHEAD)
+    if (need_error)
       LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, h->ebar, h->scale[h->last], h->eta_prev, h->etmp);
     ea.ebar = h->etmp;
     ea.esrc = ESRC_UNIFORM;
   }
+  return ea;
+}
+
+int export_vec(sae_handle* h, int what, int k, float* out) {
+  const ExportArgs ea = export_args(h, what, k, what == EXP_WERR || what == EXP_STEP_AHEAD);
   LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
   return check_launch(h);
+}
+
+// ---- checkpoint: every buffer a later step or getter depends on, in a fixed order ----
+struct CkptHeader {
+  uint64_t magic;
+  int32_t K, T, compressor, server_compress, mode, avg_period;
+  uint32_t topk_num, topk_den;
+  float momentum, weight_decay;
+  int64_t d, t;
+  int32_t esrc, last;
+  float eta_prev;
+  int32_t pad;
+};
+constexpr uint64_t kCkptMagic = 0x5341455F434B5031ull;   // "SAE_CKP1"
+
+struct CkptSection { void* ptr; size_t bytes; };
+
+std::vector<CkptSection> ckpt_sections(sae_handle* h) {
+  const Plan& P = h->P;
+  const size_t KT = (size_t)P.K * P.T, f = sizeof(float);
+  const bool sign = h->cfg.compressor == SAE_COMPRESSOR_SIGN, topk = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
+  std::vector<CkptSection> v;
+  v.push_back({h->x, (size_t)P.dpad * f}); v.push_back({h->e_srv, (size_t)P.dpad * f});
+  v.push_back({h->ebar, (size_t)P.dpad * f}); v.push_back({h->m, (size_t)P.K * P.dpad * f});
+  if (h->D) v.push_back({h->D, (size_t)P.K * P.dpad * f});
+  if (sign) { v.push_back({h->words, (size_t)P.K * P.nwords * 4}); v.push_back({h->words_srv, (size_t)P.nwords * 4}); }
+  if (topk) v.push_back({h->mask_srv, (size_t)P.nwords * 4});
+  v.push_back({h->scale[0], KT * f}); v.push_back({h->scale[1], KT * f}); v.push_back({h->scale_srv, (size_t)P.T * f});
+  v.push_back({h->tau[0], KT * 4}); v.push_back({h->tau[1], KT * 4}); v.push_back({h->tau_srv, (size_t)P.T * 4});
+  return v;
+}
+
+size_t ckpt_bytes(sae_handle* h) {
+  size_t total = 256;                       // header, padded
+  for (const auto& s : ckpt_sections(h)) total += (s.bytes + 255) / 256 * 256;
+  return total;
 }
 
 }  // namespace
@@ -642,6 +684,67 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
   }
   if (bytes < need) return SAE_ERR_INVALID_ARG;
   SAE_CUDA(h, cudaMemcpyAsync(out, src, need, cudaMemcpyDeviceToDevice, h->stream));
+  return SAE_OK;
+}
+
+int64_t sae_state_bytes(sae_handle* h) { return h ? (int64_t)ckpt_bytes(h) : -1; }
+
+int sae_save_state(sae_handle* h, void* out, size_t bytes) {
+  if (!h || !out || bytes < ckpt_bytes(h)) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  CkptHeader hd;
+  memset(&hd, 0, sizeof(hd));
+  hd.magic = kCkptMagic; hd.K = h->P.K; hd.T = h->P.T; hd.compressor = h->cfg.compressor;
+  hd.server_compress = h->cfg.server_compress; hd.mode = h->cfg.mode; hd.avg_period = h->cfg.avg_period;
+  hd.topk_num = h->cfg.topk_num; hd.topk_den = h->cfg.topk_den; hd.momentum = h->cfg.momentum;
+  hd.weight_decay = h->cfg.weight_decay; hd.d = h->P.d; hd.t = h->t; hd.esrc = h->esrc; hd.last = h->last;
+  hd.eta_prev = h->eta_prev;
+  SAE_CUDA(h, cudaMemcpyAsync(out, &hd, sizeof(hd), cudaMemcpyHostToDevice, h->stream));
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));        // hd lives on this stack frame
+  char* q = (char*)out + 256;
+  for (const auto& s : ckpt_sections(h)) {
+    SAE_CUDA(h, cudaMemcpyAsync(q, s.ptr, s.bytes, cudaMemcpyDeviceToDevice, h->stream));
+    q += (s.bytes + 255) / 256 * 256;
+  }
+  return SAE_OK;
+}
+
+int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
+  if (!h || !in || bytes < ckpt_bytes(h)) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  CkptHeader hd;
+  SAE_CUDA(h, cudaMemcpyAsync(&hd, in, sizeof(hd), cudaMemcpyDeviceToHost, h->stream));
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  const sae_config& c = h->cfg;
+  if (hd.magic != kCkptMagic || hd.K != h->P.K || hd.T != h->P.T || hd.d != h->P.d || hd.compressor != c.compressor ||
+      hd.server_compress != c.server_compress || hd.mode != c.mode || hd.avg_period != c.avg_period ||
+      hd.topk_num != c.topk_num || hd.topk_den != c.topk_den || hd.momentum != c.momentum ||
+      hd.weight_decay != c.weight_decay)
+    return SAE_ERR_INVALID_ARG;                         // a checkpoint of a different configuration
+  if (hd.esrc == ESRC_PENDING_AVG && !h->fused_ok) return SAE_ERR_INVALID_ARG;
+  const char* q = (const char*)in + 256;
+  for (const auto& s : ckpt_sections(h)) {
+    SAE_CUDA(h, cudaMemcpyAsync(s.ptr, q, s.bytes, cudaMemcpyDeviceToDevice, h->stream));
+    q += (s.bytes + 255) / 256 * 256;
+  }
+  h->t = hd.t; h->esrc = hd.esrc; h->last = hd.last; h->eta_prev = hd.eta_prev;
+  return SAE_OK;
+}
+
+int sae_get_mismatch(sae_handle* h, double* out_host) {
+  if (!h || !out_host) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  if (!h->mismatch) SAE_CUDA(h, dalloc(&h->mismatch, 2));
+  SAE_CUDA(h, cudaMemsetAsync(h->mismatch, 0, 2 * sizeof(double), h->stream));
+  const ExportArgs ea = export_args(h, EXP_WERR, 0, true);
+  LAUNCH(h, S_EXPORT, k_mismatch, h->P.ntiles, h->P, ea, h->mismatch);
+  int rc = check_launch(h);
+  if (rc != SAE_OK) return rc;
+  SAE_CUDA(h, cudaMemcpyAsync(out_host, h->mismatch, 2 * sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
   return SAE_OK;
 }
 

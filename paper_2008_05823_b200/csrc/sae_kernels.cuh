@@ -418,6 +418,35 @@ __global__ void __launch_bounds__(THREADS) k_export(Plan P, ExportArgs A, float*
   }
 }
 
+// Gradient-mismatch bounds of Section 3 (the quantities plotted in Fig. 3, right; L and sigma ignored):
+//   out[0] = || e + ebar ||^2                         (local error feedback; ebar = mean_k e^(k))
+//   out[1] = (1/K) sum_k || e + ebar - e^(k) ||^2      (step ahead)
+// accumulated in fp64.  current_error needs A.k; it is set per worker inside the loop.
+__global__ void __launch_bounds__(THREADS) k_mismatch(Plan P, ExportArgs A, double* out) {
+  __shared__ double red[2][THREADS / 32];
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  double s0 = 0.0, s1 = 0.0;
+  for (int i = threadIdx.x; i < ti.cnt; i += THREADS) {
+    const long long p = ti.poff + ti.t0 + i;
+    double sum = 0.0;
+    for (int k = 0; k < P.K; ++k) { A.k = k; sum += (double)current_error(A, P, ti.j, p); }
+    const double base = (double)A.e_srv[p] + sum / (double)P.K;
+    s0 += base * base;
+    double acc = 0.0;
+    for (int k = 0; k < P.K; ++k) { A.k = k; const double v = base - (double)current_error(A, P, ti.j, p); acc += v * v; }
+    s1 += acc / (double)P.K;
+  }
+  for (int o = 16; o > 0; o >>= 1) { s0 += __shfl_xor_sync(0xffffffffu, s0, o); s1 += __shfl_xor_sync(0xffffffffu, s1, o); }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = s0; red[1][threadIdx.x >> 5] = s1; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0.0, b = 0.0;
+    for (int w = 0; w < THREADS / 32; ++w) { a += red[0][w]; b += red[1][w]; }
+    atomicAdd(out, a);
+    atomicAdd(out + 1, b);
+  }
+}
+
 // caller layout -> padded layout
 __global__ void __launch_bounds__(THREADS) k_import(Plan P, const float* __restrict__ in, float* __restrict__ out) {
   const TileInfo ti = tile_info(P, blockIdx.x);
