@@ -176,14 +176,17 @@ def algorithmic_bytes(w, avg_period):
     """Bytes the method itself must move per step (each gradient read once, each persistent state word
     read and written once) and per launch of the worker pass."""
     Wd, d = w.num_workers * w.d, w.d
+    topk = w.compressor != 1
     if avg_period == 1:
         step = 12 * Wd + 24 * d              # g R, m RW | x RW, e_srv RW, ebar RW
-        worker = 12 * Wd + 8 * d             # g R, m RW | ebar RW (the pending average is formed in this pass)
-        variant = "sign_p1" if w.compressor == 1 else "topk"
+        # scaled sign: g R, m RW | ebar RW (the pending average is formed in this pass);
+        # Top-K: g R, m RW, Delta W | ebar R (Delta is stored for the dense server pass)
+        worker = 16 * Wd + 4 * d if topk else 12 * Wd + 8 * d
+        variant = "topk" if topk else "sign_p1"
     else:
         step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW
         worker = 20 * Wd                     # g R, m RW, Delta(e) RW
-        variant = "sign_general" if w.compressor == 1 else "topk"
+        variant = "topk" if topk else "sign_general"
     return step, worker, variant
 
 
