@@ -457,3 +457,46 @@ def test_range_flag_and_bad_config():
         Oracle(0, sizes, x0)
     with pytest.raises(ValueError):
         Oracle(1, [0], np.zeros(0, dtype=np.float32))
+
+
+# ------------------------------------------------------------------------------------------------
+# randomised property checks (hypothesis): the identities must hold for any shape and schedule
+# ------------------------------------------------------------------------------------------------
+from hypothesis import given, settings, strategies as st
+
+
+@settings(max_examples=40, deadline=None)
+@given(K=st.integers(1, 6), sizes=st.lists(st.integers(1, 300), min_size=1, max_size=5), comp=st.sampled_from([SIGN, TOPK]),
+       mode=st.sampled_from([EF, SAEF]), p=st.integers(0, 4), dc=st.integers(0, 1), steps=st.integers(1, 6),
+       seed=st.integers(0, 10 ** 6), mu=st.sampled_from([0.0, 0.5, 0.9]), lam=st.sampled_from([0.0, 1e-3]))
+def test_auxiliary_identity_random_configurations(K, sizes, comp, mode, p, dc, steps, seed, mu, lam):
+    """Eq. 3 per step and the telescoped sum x_0 - x_T = sum_t C(Delta_t), fp64, random configurations."""
+    x0, gs = rand_sizes_grads(K, sizes, steps, np.float64, seed=seed)
+    o = Oracle(K, sizes, x0, compressor=comp, server_compress=dc, mode=mode, avg_period=p, momentum=mu, weight_decay=lam,
+               topk_num=1, topk_den=7, dtype=np.float64)
+    xt = aux(o)
+    applied = np.zeros_like(x0)
+    for g in gs:
+        o.step(g, 0.1)
+        m = o.get_all(o.M)
+        xt_new = aux(o)
+        np.testing.assert_allclose(xt_new, xt - 0.1 * m.mean(axis=0), rtol=0, atol=1e-12)
+        xt = xt_new
+        applied += o.get(o.C_DELTA_SRV)
+        # Assumption 4 for every worker tensor: ||C(v) - v||^2 <= ||v||^2
+        D, c = o.get_all(o.DELTA), o.get_all(o.C_DELTA)
+        assert ((D - c) ** 2).sum() <= (D ** 2).sum() * (1 + 1e-12) + 1e-300
+    np.testing.assert_allclose(x0 - o.get(o.X), applied, atol=1e-12)
+
+
+@settings(max_examples=30, deadline=None)
+@given(n=st.integers(1, 400), scale_exp=st.integers(-30, 20), seed=st.integers(0, 10 ** 6))
+def test_fixed_point_l1_random(n, scale_exp, seed):
+    """Exact L1 against rational arithmetic for random magnitudes (including values >= 1 and tiny ones)."""
+    rng = np.random.default_rng(seed)
+    v = (rng.standard_normal(n) * 2.0 ** scale_exp).astype(np.float32)
+    S, rg = so.l1_fixed(v)
+    if np.all(np.abs(v) < 2.0 ** 32):
+        assert not rg and S == _exact_fixed_sum(v)
+    else:
+        assert rg
