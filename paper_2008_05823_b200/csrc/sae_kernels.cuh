@@ -74,13 +74,26 @@ struct ServerArgs {
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
 // compression also the server's L1 partials and sign words.  grid = ntiles.
+constexpr int SERVER_TABLE_MAX_K = 64;
+
 template <bool DC>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
   __shared__ u64 sh_red[3 * (THREADS / 32)];
   __shared__ float s_k[MAX_WORKERS];
+  // For up to 64 workers: the four codes (+-s_k) of every 4-bit group of message bits, so that a group
+  // costs one shift/mask and one 16-byte shared load instead of four bit tests and selects -- this
+  // kernel is bound by instruction issue (K order-fixed adds per parameter), not by memory.
+  __shared__ float4 tbl[SERVER_TABLE_MAX_K * 16];
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int k = tid; k < P.K; k += THREADS) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
+  const bool use_tbl = P.K <= SERVER_TABLE_MAX_K;
+  if (use_tbl) {
+    for (int q = tid; q < P.K * 16; q += THREADS) {
+      const float s = A.scale_cur[(long long)(q >> 4) * P.T + ti.j];
+      tbl[q] = make_float4((q & 1) ? s : -s, (q & 2) ? s : -s, (q & 4) ? s : -s, (q & 8) ? s : -s);
+    }
+  }
   __syncthreads();
   const long long pbase = ti.poff + ti.t0;
   float* ep = A.e_srv + pbase;
@@ -96,14 +109,27 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
       const float4 e = ld4(ep + i);
       const int wi = i >> 5, sh = i & 31;
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      const u32* wk = wp + wi;                     // worker k's word: stepped by the row pitch, no multiply
+      if (use_tbl) {
+        const float4* tk = tbl;
 #pragma unroll 8
-      for (int k = 0; k < P.K; ++k) {
-        const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> sh;
-        const float s = s_k[k];
-        a0 = __fadd_rn(a0, (w & 1u) ? s : -s);
-        a1 = __fadd_rn(a1, (w & 2u) ? s : -s);
-        a2 = __fadd_rn(a2, (w & 4u) ? s : -s);
-        a3 = __fadd_rn(a3, (w & 8u) ? s : -s);
+        for (int k = 0; k < P.K; ++k) {
+          const u32 nib = (__ldg(wk) >> sh) & 15u;
+          const float4 c = tk[nib];
+          wk += P.nwords; tk += 16;
+          a0 = __fadd_rn(a0, c.x); a1 = __fadd_rn(a1, c.y); a2 = __fadd_rn(a2, c.z); a3 = __fadd_rn(a3, c.w);
+        }
+      } else {
+#pragma unroll 8
+        for (int k = 0; k < P.K; ++k) {
+          const u32 w = __ldg(wk) >> sh;
+          wk += P.nwords;
+          const float s = s_k[k];
+          a0 = __fadd_rn(a0, (w & 1u) ? s : -s);
+          a1 = __fadd_rn(a1, (w & 2u) ? s : -s);
+          a2 = __fadd_rn(a2, (w & 4u) ? s : -s);
+          a3 = __fadd_rn(a3, (w & 8u) ? s : -s);
+        }
       }
       float4 ds;
       ds.x = __fadd_rn(e.x, div_by_k(P, a0));
