@@ -263,6 +263,27 @@ def test_graph_replay_on_a_side_stream(comp, p):
         gpu.close()
 
 
+@pytest.mark.parametrize("comp", [so.SIGN, so.TOPK])
+def test_two_runs_give_identical_bytes(comp):
+    """Run-to-run determinism: the exact L1 is an integer sum (atomics in any order), histograms are integer
+    counts, every float reduction has a fixed order -- two runs must agree byte for byte (zero signs included)."""
+    import torch
+    K, sizes = 4, RAGGED + [40000]
+    d = sum(sizes)
+    scales = synth.tensor_scales(9, len(sizes), -4.0, -1.0)
+    x0 = torch.from_numpy(synth.x0_numpy(9, d)).cuda()
+    gs = [torch.from_numpy(synth.grads_numpy(9, t, K, sizes, scales, 66, 100.0)).cuda() for t in range(6)]
+    snaps = []
+    for run in range(2):
+        h = sb.Sae(K, sizes, x0, compressor=comp, avg_period=3, weight_decay=1e-4, topk_den=50)
+        for g in gs:
+            h.step(g, 0.1)
+        h.sync()
+        snaps.append(h.save_state().cpu().numpy().copy())
+        h.close()
+    assert np.array_equal(snaps[0], snaps[1])
+
+
 def _trajectory(idx, p, steps, seed):
     w = configs.workload(idx)
     run_pair(w.num_workers, w.tensor_sizes, w.compressor, steps, seed=seed, p=p, mu=w.momentum, lam=w.weight_decay,
