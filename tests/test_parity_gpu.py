@@ -291,6 +291,32 @@ def _trajectory(idx, p, steps, seed):
              every=max(1, steps // 4))
 
 
+def _trajectory_device_inputs(idx, p, steps, seed):
+    """Whole trajectory of a workload with the gradients made by the device generator (itself checked against
+    the numpy generator in test_device_generator_matches_numpy) and copied to the host for the oracle."""
+    import torch
+    w = configs.workload(idx)
+    K, sizes, d = w.num_workers, w.tensor_sizes, w.d
+    scales = synth.workload_scales(w, seed)
+    gen = synth.DeviceGenerator(sizes, scales)
+    x0 = torch.empty(d, device="cuda")
+    gen.x0(x0, seed)
+    kw = dict(compressor=w.compressor, avg_period=p, momentum=w.momentum, weight_decay=w.weight_decay,
+              topk_num=w.topk_num, topk_den=w.topk_den)
+    orc = so.Oracle(K, sizes, x0.cpu().numpy(), threads=so.max_threads(), **kw)
+    gpu = sb.Sae(K, sizes, x0, **kw)
+    g = torch.empty(K, d, device="cuda")
+    for t in range(steps):
+        gen.grads(g, K, seed, t, w.outlier_per_65536, w.outlier_mult)
+        gpu.step(g, w.lr)
+        orc.step(g.cpu().numpy(), w.lr)
+        if (t + 1) % max(1, steps // 5) == 0 or t == steps - 1:
+            compare_state(gpu, orc, w.compressor, tag=f"cfg{idx} p={p} t={t + 1}")
+            compare_server_messages(gpu, orc, w.compressor, 1, tag=f"cfg{idx} p={p} t={t + 1}")
+    assert not orc.range_flag
+    gpu.close()
+
+
 @pytest.mark.parametrize("seed", [0, 1, 2])
 @pytest.mark.parametrize("p", [1, 5])
 def test_config0_full_trajectory(seed, p):
@@ -298,5 +324,6 @@ def test_config0_full_trajectory(seed, p):
 
 
 @pytest.mark.parametrize("p", [1, 20])
-def test_config1_trajectory(p):
-    _trajectory(1, p, 60, 0)
+def test_config1_full_trajectory(p):
+    """All 200 iterations of config 1 (heavy-tailed gradients, weight decay)."""
+    _trajectory_device_inputs(1, p, 200, 0)
