@@ -201,9 +201,9 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       const float4 e = ld4(ep + i);
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
-#pragma unroll 4
+#pragma unroll 8
       for (int k = 0; k < P.K; ++k) {
-        const float4 v = ld4(dp + (long long)k * P.dpad + i);
+        const float4 v = ld4_stream(dp + (long long)k * P.dpad + i);
         const u32 t = (COMP == 2) ? t_k[k] : 0u;
         const float c0 = (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f;
         const float c1 = (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f;
