@@ -69,6 +69,7 @@ struct sae_handle {
   int last;              // which of scale[2]/tau[2] holds the last step's values
   int last_cuda_error;
   int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
+  int num_sms;
   int64_t launches;
   // cached step graphs
   int graphs_enabled, graph_misses;
@@ -322,8 +323,11 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     }
     LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
            h->scale[cur], h->recs_srv);
-    if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, P.ntiles, P, sa);
-    else LAUNCH(h, S_SERVER, k_server_sign<false>, P.ntiles, P, sa);
+    // consecutive tiles per block: enough blocks to fill the device several times over, at most 8 tiles each
+    const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
+    const int nblk = (P.ntiles + tpb - 1) / tpb;
+    if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
+    else LAUNCH(h, S_SERVER, k_server_sign<false>, nblk, P, sa, tpb);
     const int avg = (avg_after && !defer_avg) ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
     if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
     h->esrc = defer_avg ? ESRC_PENDING_AVG : (avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN);
@@ -515,6 +519,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms < 1) sms = 148;
     h->persistent_blocks = sms * SAE_WT_BLOCKS_PER_SM;
+    h->num_sms = sms;
   }
 
   std::vector<int> tile_tensor((size_t)ntiles), first_tile(T), n32(T);

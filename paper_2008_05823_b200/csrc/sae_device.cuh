@@ -237,6 +237,33 @@ __device__ __forceinline__ void l1_add_partial(const Acc128& a, L1Record* rec, u
   if (l2) atomicAdd(&rec->limb[2], l2);
 }
 
+// Warp-level sum of the lanes' 128-bit partials, added by lane 0 to the (worker, tensor) record.
+// The low 64 bits are split into 22-bit pieces so that a 32-lane sum fits a 32-bit redux add; the
+// high word (almost always a small carry count) takes one more redux, or a shuffle tree if large.
+__device__ __forceinline__ void warp_commit(const LaneAcc& a, L1Record* rec, u32* status) {
+  const u32 full = 0xffffffffu;
+  const u64 lo = ((u64)a.lo1 << 32) | a.lo0;
+  const u32 r0 = __reduce_add_sync(full, (u32)(lo & 0x3fffffu));
+  const u32 r1 = __reduce_add_sync(full, (u32)((lo >> 22) & 0x3fffffu));
+  const u32 r2 = __reduce_add_sync(full, (u32)(lo >> 44));                   // 20 bits
+  u64 hi = a.hi + a.carry;
+  if (__any_sync(full, hi >> 24)) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) hi += __shfl_xor_sync(full, hi, o);
+  } else {
+    hi = __reduce_add_sync(full, (u32)hi);
+  }
+  const u32 bad = __any_sync(full, a.bad);
+  if ((threadIdx.x & 31) == 0) {
+    Acc128 s; acc_init(s);
+    s.lo = r0;
+    acc_add_u(s, (u64)r1 << 22, 0ull);
+    acc_add_u(s, (u64)r2 << 44, hi + (u64)(r2 >> 20));
+    s.bad = bad;
+    l1_add_partial(s, rec, status);
+  }
+}
+
 // ---- sign bits -----------------------------------------------------------------------------------
 // Four consecutive elements per lane (lane l holds elements 4l..4l+3 of a 128-element row): the four
 // words of the row are assembled by OR-ing nibbles across each group of 8 lanes.  Every lane of group

@@ -73,103 +73,147 @@ struct ServerArgs {
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
-// compression also the server's L1 partials and sign words.  grid = ntiles.
-constexpr int SERVER_TABLE_MAX_K = 64;
+// compression also the server's L1 partials and sign words.  A block walks `tiles_per_block` consecutive
+// tiles, so the scales are staged and the L1 partials committed once per run of tiles of one tensor.
+//
+// The pass is bound by instruction issue, not by memory: K order-fixed additions per parameter, each of
+// +-s_k chosen by one message bit.  A thread owns 16 consecutive parameters (half a sign word): per worker
+// it loads the word once, and per parameter moves the bit to the sign position (shift), flips the sign of
+// s_k with it (one three-input logic operation) and adds; the additions are issued two at a time as
+// packed fp32 pairs (add.rn.f32x2: two independent round-to-nearest fp32 additions, same results as two
+// scalar ones).
+constexpr int SRV_E = 16;   // consecutive parameters per thread; THREADS * SRV_E == TILE
+constexpr int SRV_B = 8;    // workers per batch of word loads
+static_assert(THREADS * SRV_E == TILE, "one pass of the block covers one tile");
+
+__device__ __forceinline__ u64 pack2(u32 lo, u32 hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
+  u64 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
 
 template <bool DC>
-__global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A) {
-  __shared__ u64 sh_red[3 * (THREADS / 32)];
+__global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
-  // For up to 64 workers: the four codes (+-s_k) of every 4-bit group of message bits, so that a group
-  // costs one shift/mask and one 16-byte shared load instead of four bit tests and selects -- this
-  // kernel is bound by instruction issue (K order-fixed adds per parameter), not by memory.
-  __shared__ float4 tbl[SERVER_TABLE_MAX_K * 16];
-  const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int k = tid; k < P.K; k += THREADS) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
-  const bool use_tbl = P.K <= SERVER_TABLE_MAX_K;
-  if (use_tbl) {
-    for (int q = tid; q < P.K * 16; q += THREADS) {
-      const float s = A.scale_cur[(long long)(q >> 4) * P.T + ti.j];
-      tbl[q] = make_float4((q & 1) ? s : -s, (q & 2) ? s : -s, (q & 4) ? s : -s, (q & 8) ? s : -s);
-    }
-  }
-  __syncthreads();
-  const long long pbase = ti.poff + ti.t0;
-  float* ep = A.e_srv + pbase;
-  const u32* __restrict__ wp = A.words + (pbase >> 5);
-  u32* wsp = A.words_srv + (pbase >> 5);
-  const float Kf = (float)P.K;
-  Acc128 acc; acc_init(acc);
+  const int tile0 = blockIdx.x * tiles_per_block;
+  const int tile1 = min(P.ntiles, tile0 + tiles_per_block);
+  LaneAcc acc; lane_acc_init(acc);
+  int cur_j = -1;
 
-  if (ti.cnt == TILE) {
-#pragma unroll 2
-    for (int it = 0; it < VEC_ITERS; ++it) {
-      const int i = it * (THREADS * 4) + tid * 4;
-      const float4 e = ld4(ep + i);
-      const int wi = i >> 5, sh = i & 31;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  for (int tile = tile0; tile < tile1; ++tile) {
+    const TileInfo ti = tile_info(P, tile);
+    if (ti.j != cur_j) {
+      if (DC && cur_j >= 0) { warp_commit(acc, A.recs_srv + cur_j, A.status); lane_acc_init(acc); }
+      __syncthreads();                            // the previous tensor's scales are no longer read
+      for (int k = tid; k < P.K; k += THREADS) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
+      __syncthreads();
+      cur_j = ti.j;
+    }
+    const long long pbase = ti.poff + ti.t0;
+    float* ep = A.e_srv + pbase;
+    const u32* __restrict__ wp = A.words + (pbase >> 5);
+    u32* wsp = A.words_srv + (pbase >> 5);
+
+    if (ti.cnt == TILE) {
+      const int i = tid * SRV_E;
+      const int wi = i >> 5, sh = (32 - SRV_E) - (i & 31);   // this thread's bits go to the top of the word
+      u64 a2[SRV_E / 2];
+#pragma unroll
+      for (int j = 0; j < SRV_E / 2; ++j) a2[j] = 0ull;      // (+0, +0)
+      // Single-way: the server error is fetched ahead of the worker loop, so that its latency hides under
+      // the loop.  (Double-way has enough independent work after the loop; fetching early there only
+      // costs registers.)
+      float4 ev[DC ? 1 : SRV_E / 4];
+      if constexpr (!DC) {
+#pragma unroll
+        for (int q = 0; q < SRV_E / 4; ++q) ev[q] = ld4(ep + i + 4 * q);
+      }
+      // The words of SRV_B workers are fetched as one batch of independent loads, the next batch while
+      // this one is consumed: without that the loop waits out one memory latency per worker.
       const u32* wk = wp + wi;                     // worker k's word: stepped by the row pitch, no multiply
-      if (use_tbl) {
-        const float4* tk = tbl;
-#pragma unroll 8
-        for (int k = 0; k < P.K; ++k) {
-          const u32 nib = (__ldg(wk) >> sh) & 15u;
-          const float4 c = tk[nib];
-          wk += P.nwords; tk += 16;
-          a0 = __fadd_rn(a0, c.x); a1 = __fadd_rn(a1, c.y); a2 = __fadd_rn(a2, c.z); a3 = __fadd_rn(a3, c.w);
-        }
-      } else {
-#pragma unroll 8
-        for (int k = 0; k < P.K; ++k) {
-          const u32 w = __ldg(wk) >> sh;
-          wk += P.nwords;
-          const float s = s_k[k];
-          a0 = __fadd_rn(a0, (w & 1u) ? s : -s);
-          a1 = __fadd_rn(a1, (w & 2u) ? s : -s);
-          a2 = __fadd_rn(a2, (w & 4u) ? s : -s);
-          a3 = __fadd_rn(a3, (w & 8u) ? s : -s);
+      u32 wn[SRV_B];
+#pragma unroll
+      for (int u = 0; u < SRV_B; ++u) wn[u] = (u < P.K) ? __ldg(wk + (long long)u * P.nwords) : 0u;
+      for (int k0 = 0; k0 < P.K; k0 += SRV_B) {
+        u32 w[SRV_B];
+#pragma unroll
+        for (int u = 0; u < SRV_B; ++u) w[u] = wn[u];
+        wk += (long long)SRV_B * P.nwords;
+#pragma unroll
+        for (int u = 0; u < SRV_B; ++u) wn[u] = (k0 + SRV_B + u < P.K) ? __ldg(wk + (long long)u * P.nwords) : 0u;
+#pragma unroll
+        for (int u = 0; u < SRV_B; ++u) {
+          if (k0 + u < P.K) {
+            const u32 t = ~(w[u] << sh);           // a clear bit is a negative code: it flips the sign of s_k
+            const u32 sb = __float_as_uint(s_k[k0 + u]);
+#pragma unroll
+            for (int j = 0; j < SRV_E; j += 2) {
+              const u32 c0 = ((t << (SRV_E - 1 - j)) & 0x80000000u) ^ sb;
+              const u32 c1 = ((t << (SRV_E - 2 - j)) & 0x80000000u) ^ sb;
+              a2[j / 2] = add_f32x2(a2[j / 2], pack2(c0, c1));
+            }
+          }
         }
       }
-      float4 ds;
-      ds.x = __fadd_rn(e.x, div_by_k(P, a0));
-      ds.y = __fadd_rn(e.y, div_by_k(P, a1));
-      ds.z = __fadd_rn(e.z, div_by_k(P, a2));
-      ds.w = __fadd_rn(e.w, div_by_k(P, a3));
-      st4(ep + i, ds);
-      if (DC) {
-        acc_add(acc, ds.x); acc_add(acc, ds.y); acc_add(acc, ds.z); acc_add(acc, ds.w);
-        u32 w = pack_row4(ds.x >= 0.0f, ds.y >= 0.0f, ds.z >= 0.0f, ds.w >= 0.0f);
-        if ((lane & 7) == 0) wsp[wi] = w;
-      }
-    }
-  } else {
-    for (int r = 0; r < ROWS; ++r) {
-      const int i = r * THREADS + tid;
-      const bool valid = i < ti.cnt;
-      float ds = 0.0f;
-      if (valid) {
-        float a = 0.f;
-        const int wi = i >> 5;
-        for (int k = 0; k < P.K; ++k) {
-          const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> lane;
-          const float s = s_k[k];
-          a = __fadd_rn(a, (w & 1u) ? s : -s);
+      u32 bits = 0;
+#pragma unroll
+      for (int q = 0; q < SRV_E / 4; ++q) {
+        float a0, a1, a3, a4;
+        unpack2(a2[2 * q], a0, a1);
+        unpack2(a2[2 * q + 1], a3, a4);
+        float4 e;
+        if constexpr (DC) e = ld4(ep + i + 4 * q); else e = ev[q];
+        float4 ds;
+        ds.x = __fadd_rn(e.x, div_by_k(P, a0));
+        ds.y = __fadd_rn(e.y, div_by_k(P, a1));
+        ds.z = __fadd_rn(e.z, div_by_k(P, a3));
+        ds.w = __fadd_rn(e.w, div_by_k(P, a4));
+        st4(ep + i + 4 * q, ds);
+        if (DC) {
+          lane_add4(acc, ds);
+          bits |= ((ds.x >= 0.0f ? 1u : 0u) | (ds.y >= 0.0f ? 2u : 0u) | (ds.z >= 0.0f ? 4u : 0u) |
+                   (ds.w >= 0.0f ? 8u : 0u)) << (4 * q);
         }
-        ds = __fadd_rn(ep[i], div_by_k(P, a));
-        ep[i] = ds;
-        if (DC) acc_add(acc, ds);
       }
       if (DC) {
-        u32 w = __ballot_sync(0xffffffffu, valid && ds >= 0.0f);
-        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wsp[(r * THREADS + warp * 32) >> 5] = w;
+        u32 w = bits << (SRV_E * (lane & 1));      // two lanes share a word
+        w |= __shfl_xor_sync(0xffffffffu, w, 1);
+        if ((lane & 1) == 0) wsp[wi] = w;
+      }
+    } else {
+      for (int r = 0; r < ROWS; ++r) {
+        const int i = r * THREADS + tid;
+        const bool valid = i < ti.cnt;
+        float ds = 0.0f;
+        if (valid) {
+          float a = 0.f;
+          const int wi = i >> 5;
+          for (int k = 0; k < P.K; ++k) {
+            const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> lane;
+            const float s = s_k[k];
+            a = __fadd_rn(a, (w & 1u) ? s : -s);
+          }
+          ds = __fadd_rn(ep[i], div_by_k(P, a));
+          ep[i] = ds;
+          if (DC) lane_add(acc, ds);
+        }
+        if (DC) {
+          u32 w = __ballot_sync(0xffffffffu, valid && ds >= 0.0f);
+          if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wsp[(r * THREADS + warp * 32) >> 5] = w;
+        }
       }
     }
   }
-  if (DC) {
-    acc_block_reduce(acc, sh_red);
-    if (tid == 0) l1_add_partial(acc, A.recs_srv + ti.j, A.status);
-  }
+  if (DC && cur_j >= 0) warp_commit(acc, A.recs_srv + cur_j, A.status);
 }
 
 // K3 (identity / Top-K): the same aggregation from the dense model differences.
