@@ -191,8 +191,8 @@ def algorithmic_bytes(w, avg_period):
     if avg_period == 1:
         step = 12 * Wd + 24 * d              # g R, m RW | x RW, e_srv RW, ebar RW
         # scaled sign: g R, m RW | ebar RW (the pending average is formed in this pass);
-        # Top-K: g R, m RW, Delta W | ebar R (Delta is stored for the dense server pass)
-        worker = 16 * Wd + 4 * d if topk else 12 * Wd + 8 * d
+        # Top-K: g R, m RW | ebar R (Delta is not stored: the server pass recomputes it from m)
+        worker = 12 * Wd + 4 * d if topk else 12 * Wd + 8 * d
         variant = "topk" if topk else "sign_p1"
     else:
         step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW

@@ -70,6 +70,8 @@ struct sae_handle {
   int last_cuda_error;
   int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
   int num_sms;
+  int topk_nod;            // Top-K with p = 1: model differences never stored, two uniform-error buffers
+  float* ebar_alt;
   int64_t launches;
   // cached step graphs
   int graphs_enabled, graph_misses;
@@ -143,7 +145,7 @@ cudaError_t dalloc(T** p, size_t count) {
 }
 
 void free_all(sae_handle* h) {
-  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->m, h->D, h->etmp,
+  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->ebar_alt, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
                   h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
@@ -157,8 +159,8 @@ void free_all(sae_handle* h) {
 
 // ---- Top-K threshold of every (row, tensor) of buf[rows][dpad] ---------------------------------------
 // Candidate-window refine first; the three-level radix select then runs only where the window failed.
-void topk_thresholds(sae_handle* h, const float* buf, int rows, const CandArgs& cand, const u32* tau_guess, u32* tau_out,
-                     u32* fb, u32* fb_total) {
+void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArgs& cand, const u32* tau_guess,
+                     u32* tau_out, u32* fb, u32* fb_total) {
   const Plan& P = h->P;
   const int pairs = rows * P.T;
   LAUNCH(h, S_TOPK_SELECT, k_topk_decide, (pairs + THREADS - 1) / THREADS, cand, rows, h->d_n, h->cfg.topk_num,
@@ -167,12 +169,23 @@ void topk_thresholds(sae_handle* h, const float* buf, int rows, const CandArgs& 
   LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, h->work, h->work_count);
   const long long hist_grid = 8LL * h->persistent_blocks;
   for (int level = 0; level < 3; ++level) {
-    LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, buf, h->cand_n, h->sel, h->hist, h->work,
+    LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, src, h->cand_n, h->sel, h->hist, h->work,
            h->work_count);
     LAUNCH(h, S_TOPK_SELECT, k_topk_select, pairs, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, h->hist, h->sel,
            tau_out, h->work_count);
   }
 }
+
+DeltaSrc stored_rows(const float* buf) {
+  DeltaSrc s; s.buf = buf; s.m = nullptr; s.ebar = nullptr; s.eta = 0.0f; s.recompute = 0;
+  return s;
+}
+
+// The uniform local error as the next step will read it.  Top-K with p = 1 alternates between two buffers
+// (the server pass reads the old one while writing the new one, and the getters of the last step's
+// selection still need the old one); index `last` flips every step, like the scale and threshold buffers.
+float* ebar_now(sae_handle* h) { return (h->topk_nod && h->last) ? h->ebar_alt : h->ebar; }
+float* ebar_other(sae_handle* h) { return (h->topk_nod && !h->last) ? h->ebar_alt : h->ebar; }
 
 CandArgs cand_args(sae_handle* h, bool server) {
   CandArgs c;
@@ -288,16 +301,17 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   sp.mu = c.momentum; sp.eta = lr; sp.lambda = c.weight_decay;
   sp.saef = (c.mode == SAE_MODE_SAEF); sp.wd = (c.weight_decay != 0.0f);
   WorkerArgs wa;
-  wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = h->ebar; wa.x = h->x;
+  wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = ebar_now(h); wa.x = h->x;
   wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
   wa.cand = cand_args(h, false);
   ServerArgs sa;
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
   sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
-  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = h->ebar;
+  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = ebar_now(h);
+  sa.m = h->m; sa.ebar_in = ebar_now(h); sa.eta = lr;
   ApplyArgs aa;
-  aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.m = h->m; aa.D = h->D;
+  aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = ebar_now(h); aa.m = h->m; aa.D = h->D;
   aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv; aa.tau_cur = h->tau[cur];
   aa.tau_srv = h->tau_srv;
   aa.mask_srv = h->mask_srv; aa.eta = lr;
@@ -312,7 +326,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     const bool defer_avg = avg_after && !write_d && h->fused_ok;
     if (pending_in) {
       FusedArgs fa;
-      fa.g = grads; fa.m = h->m; fa.ebar = h->ebar; fa.x = h->x; fa.scale_prev = h->scale[h->last];
+      fa.g = grads; fa.m = h->m; fa.ebar = ebar_now(h); fa.x = h->x; fa.scale_prev = h->scale[h->last];
       fa.words = h->words; fa.recs = h->recs; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
       launch_fused(h, sp, fa);
     } else if (h->esrc == ESRC_UNIFORM) {
@@ -332,13 +346,24 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
     h->esrc = defer_avg ? ESRC_PENDING_AVG : (avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN);
   } else if (c.compressor == SAE_COMPRESSOR_TOPK) {
-    if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
+    // p = 1 (previous error uniform, pre-step averages, every step): the model differences are not stored;
+    // whoever needs them after the worker pass recomputes them from m and the old uniform error
+    const bool nod = h->topk_nod;
+    if (nod && !(h->esrc == ESRC_UNIFORM && avg_after)) return SAE_ERR_INVALID_ARG;
+    if (!nod && !h->D) return SAE_ERR_INVALID_ARG;
+    DeltaSrc src = stored_rows(h->D);
+    if (nod) { src.m = h->m; src.ebar = ebar_now(h); src.eta = lr; src.recompute = 1; }
+    if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
+    else if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
     else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
-    topk_thresholds(h, h->D, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+    topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
     // the averaged error (if the pre-step averages) comes out of the same pass over D as the server's sum
-    if (avg_after) LAUNCH(h, S_SERVER, (k_server_dense<2, true>), P.ntiles, P, sa);
+    if (nod) {
+      sa.ebar = ebar_other(h);          // becomes the current one when `last` flips below
+      LAUNCH(h, S_SERVER, (k_server_dense<2, true, true>), P.ntiles, P, sa);
+    } else if (avg_after) LAUNCH(h, S_SERVER, (k_server_dense<2, true>), P.ntiles, P, sa);
     else LAUNCH(h, S_SERVER, (k_server_dense<2, false>), P.ntiles, P, sa);
-    if (dc) topk_thresholds(h, h->e_srv, 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
+    if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
     if (dc) launch_apply<2, 2>(h, AVG_NONE, aa); else launch_apply<2, 0>(h, AVG_NONE, aa);
     h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
   } else {
@@ -419,13 +444,13 @@ int do_step(sae_handle* h, const float* grads, float lr) {
 
 ExportArgs export_args(sae_handle* h, int what, int k, bool need_error) {
   ExportArgs ea;
-  ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = h->ebar;
+  ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = ebar_now(h);
   ea.scale_last = h->scale[h->last]; ea.tau_last = h->tau[h->last];
   ea.esrc = h->esrc; ea.what = what; ea.k = k; ea.saef = (h->cfg.mode == SAE_MODE_SAEF);
   if (h->esrc == ESRC_PENDING_AVG) {
     // the averaged error exists only implicitly: form it in a scratch vector, leave the state alone
     if (need_error)
-      LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, h->ebar, h->scale[h->last], h->eta_prev, h->etmp);
+      LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, ebar_now(h), h->scale[h->last], h->eta_prev, h->etmp);
     ea.ebar = h->etmp;
     ea.esrc = ESRC_UNIFORM;
   }
@@ -461,6 +486,7 @@ std::vector<CkptSection> ckpt_sections(sae_handle* h) {
   v.push_back({h->x, (size_t)P.dpad * f}); v.push_back({h->e_srv, (size_t)P.dpad * f});
   v.push_back({h->ebar, (size_t)P.dpad * f}); v.push_back({h->m, (size_t)P.K * P.dpad * f});
   if (h->D) v.push_back({h->D, (size_t)P.K * P.dpad * f});
+  if (h->ebar_alt) v.push_back({h->ebar_alt, (size_t)P.dpad * f});
   if (sign) { v.push_back({h->words, (size_t)P.K * P.nwords * 4}); v.push_back({h->words_srv, (size_t)P.nwords * 4}); }
   if (topk) v.push_back({h->mask_srv, (size_t)P.nwords * 4});
   v.push_back({h->scale[0], KT * f}); v.push_back({h->scale[1], KT * f}); v.push_back({h->scale_srv, (size_t)P.T * f});
@@ -535,7 +561,8 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
     }
   }
   const bool sign = cfg->compressor == SAE_COMPRESSOR_SIGN, topk = cfg->compressor == SAE_COMPRESSOR_TOPK;
-  const bool need_D = !(sign && cfg->avg_period == 1);
+  h->topk_nod = (topk && cfg->avg_period == 1) ? 1 : 0;
+  const bool need_D = !((sign || topk) && cfg->avg_period == 1);
   const long long nwords = dpad / 32;
   const size_t KT = (size_t)K * T;
 
@@ -553,6 +580,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   ALLOC0(h->m, (size_t)K * dpad);
   if (h->fused_ok) ALLOC0(h->etmp, dpad);
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
+  if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);
   ALLOC0(h->mask_srv, topk ? nwords : 0);
@@ -682,8 +710,13 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
     case SAE_STATE_TOPK_FALLBACKS: if (!topk) return SAE_ERR_INVALID_ARG; src = h->fb_total; need = 2 * sizeof(u32); break;
     case SAE_STATE_WORKER_MASK:
       if (!topk || bytes < wb) return SAE_ERR_INVALID_ARG;
-      LAUNCH(h, S_MASK, k_mask_words, P.ntiles, P, h->D + (size_t)worker * P.dpad, h->tau[h->last] + (size_t)worker * P.T,
-             (u32*)out);
+      {
+        DeltaSrc src = stored_rows(h->D ? h->D + (size_t)worker * P.dpad : nullptr);
+        if (h->topk_nod) {     // the last step's differences: its learning rate, the uniform error it started from
+          src.m = h->m + (size_t)worker * P.dpad; src.ebar = ebar_other(h); src.eta = h->eta_prev; src.recompute = 1;
+        }
+        LAUNCH(h, S_MASK, k_mask_words, P.ntiles, P, src, h->tau[h->last] + (size_t)worker * P.T, (u32*)out);
+      }
       return check_launch(h);
     default: return SAE_ERR_INVALID_ARG;
   }

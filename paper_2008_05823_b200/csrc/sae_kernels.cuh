@@ -70,6 +70,9 @@ struct ServerArgs {
   const u32* tau_srv_prev; // [T] last step's server thresholds: the guess of the server's window
   int emit_srv;            // double-way Top-K: collect the server's candidates in this pass
   float* ebar;             // [dpad] averaged local error (dense variants, when the pre-step averages)
+  const float* m;          // [K][dpad] } recompute variant: Delta^(k) = fma(eta, m^(k), ebar_in), not stored
+  const float* ebar_in;    // [dpad]    } (ebar_in and ebar are different buffers)
+  float eta;
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -221,7 +224,10 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 // AVG: the next pre-step averages the local errors; they are functions of the same D^(k) and thresholds
 // this pass already reads, so ebar = (1/K) sum_k (D^(k) - C(D^(k))) is formed here, in k order, instead of
 // in a further pass over D.
-template <int COMP, bool AVG>
+// RECOMP (Top-K with p = 1: the previous error is uniform and the pre-step averages, every step): the worker
+// pass did not store D^(k); it is recomputed here from m^(k) and the previous uniform error with the fused
+// operation that formed it, so the step moves 4 bytes per worker-element less.
+template <int COMP, bool AVG, bool RECOMP = false>
 __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
@@ -236,18 +242,25 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   }
   const long long pbase = ti.poff + ti.t0;
   float* ep = A.e_srv + pbase;
-  const float* __restrict__ dp = A.D + pbase;
+  const float* __restrict__ dp = (RECOMP ? A.m : A.D) + pbase;
+  const float* __restrict__ eo = A.ebar_in + pbase;      // read only when RECOMP
   const float Kf = (float)P.K;
   if (ti.cnt == TILE) {
 #pragma unroll 2
     for (int it = 0; it < VEC_ITERS; ++it) {
       const int i = it * (THREADS * 4) + tid * 4;
       const float4 e = ld4(ep + i);
+      float4 eold = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (RECOMP) eold = ld4(eo + i);
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
 #pragma unroll 8
       for (int k = 0; k < P.K; ++k) {
-        const float4 v = ld4_stream(dp + (long long)k * P.dpad + i);
+        float4 v = RECOMP ? ld4(dp + (long long)k * P.dpad + i) : ld4_stream(dp + (long long)k * P.dpad + i);
+        if (RECOMP) {
+          v.x = __fmaf_rn(A.eta, v.x, eold.x); v.y = __fmaf_rn(A.eta, v.y, eold.y);
+          v.z = __fmaf_rn(A.eta, v.z, eold.z); v.w = __fmaf_rn(A.eta, v.w, eold.w);
+        }
         const u32 t = (COMP == 2) ? t_k[k] : 0u;
         const float c0 = (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f;
         const float c1 = (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f;
@@ -277,8 +290,10 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       float ds = 0.0f;
       if (i < ti.cnt) {
         float a = 0.f, b = 0.f;
+        const float eold = RECOMP ? eo[i] : 0.0f;
         for (int k = 0; k < P.K; ++k) {
-          const float v = dp[(long long)k * P.dpad + i];
+          float v = dp[(long long)k * P.dpad + i];
+          if (RECOMP) v = __fmaf_rn(A.eta, v, eold);
           const float c = (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f;
           a = __fadd_rn(a, c);
           if (AVG) b = __fadd_rn(b, __fsub_rn(v, c));
@@ -523,8 +538,9 @@ __global__ void __launch_bounds__(THREADS) k_import(Plan P, const float* __restr
   for (int i = threadIdx.x; i < ti.cnt; i += THREADS) out[ti.poff + ti.t0 + i] = in[ti.off + ti.t0 + i];
 }
 
-// Top-K selection of row k of buf as bit words
-__global__ void __launch_bounds__(THREADS) k_mask_words(Plan P, const float* __restrict__ buf,
+// Top-K selection of one row as bit words; the row is stored (src.buf) or recomputed (src.m, both already
+// offset to the row)
+__global__ void __launch_bounds__(THREADS) k_mask_words(Plan P, DeltaSrc src,
                                                          const u32* __restrict__ tau, u32* __restrict__ out) {
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -533,7 +549,9 @@ __global__ void __launch_bounds__(THREADS) k_mask_words(Plan P, const float* __r
   for (int r = 0; r < ROWS; ++r) {
     const int i = r * THREADS + tid;
     const bool valid = i < ti.cnt;
-    const bool q = valid && topk_selected(buf[pbase + i], t);
+    float v = 0.0f;
+    if (valid) v = src.recompute ? __fmaf_rn(src.eta, src.m[pbase + i], src.ebar[pbase + i]) : src.buf[pbase + i];
+    const bool q = valid && topk_selected(v, t);
     u32 w = __ballot_sync(0xffffffffu, q);
     if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) out[(pbase + r * THREADS + warp * 32) >> 5] = w;
   }

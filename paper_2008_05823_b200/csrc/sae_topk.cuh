@@ -184,6 +184,16 @@ __global__ void __launch_bounds__(THREADS) k_topk_worklist(Plan P, int rows, con
   if (fallback[(long long)k * P.T + P.tile_tensor[tile]]) work[atomicAdd(work_count, 1u)] = make_int2((int)mine, -1);
 }
 
+// The rows whose Top-K thresholds are wanted: stored ([rows][dpad] in buf), or -- when the worker pass did
+// not store the model differences -- recomputed as fma(eta, m^(k), ebar), the operation that formed them.
+struct DeltaSrc {
+  const float* buf;
+  const float* m;
+  const float* ebar;
+  float eta;
+  int recompute;
+};
+
 __device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* hist) {
   if (level == 0) atomicAdd(hist + (key >> 20), 1u);
   else if (level == 1) { if ((key >> 20) == prefix) atomicAdd(hist + ((key >> 10) & 1023u), 1u); }
@@ -193,8 +203,8 @@ __device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* h
 // Level L histogram over the work list (a fixed grid of blocks strides over it).  Every item accumulates
 // in shared memory first (the candidates of a pair nearly all share their leading digits, so direct
 // global atomics would pile up on a few addresses) and adds its non-zero bins to the pair's histogram.
-// buf is [rows][dpad]; hist is [rows][T][HIST_BINS]
-__global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int rows, int level, const float* __restrict__ buf,
+// hist is [rows][T][HIST_BINS]
+__global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int rows, int level, DeltaSrc src,
                                                         const u32* __restrict__ cand_n, const SelectState* __restrict__ st,
                                                         u32* hist, const int2* __restrict__ work,
                                                         const u32* __restrict__ work_count) {
@@ -212,20 +222,27 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
       const int k = w.x - tile * rows;
       const TileInfo ti = tile_info(P, tile);
       rj = k * P.T + ti.j;
-      const float* __restrict__ bp = buf + (long long)k * P.dpad + ti.poff + ti.t0;
+      const float* __restrict__ bp = (src.recompute ? src.m : src.buf) + (long long)k * P.dpad + ti.poff + ti.t0;
+      const float* __restrict__ eb = src.ebar + ti.poff + ti.t0;     // read only when recomputing
       const u32 prefix = level ? st[rj].prefix : 0u;
       u32* target = sh;
       if (ti.cnt == TILE) {
 #pragma unroll
         for (int it = 0; it < VEC_ITERS; ++it) {
-          const float4 v = ld4(bp + it * (THREADS * 4) + tid * 4);
+          float4 v = ld4(bp + it * (THREADS * 4) + tid * 4);
+          if (src.recompute) {
+            const float4 e = ld4(eb + it * (THREADS * 4) + tid * 4);
+            v.x = __fmaf_rn(src.eta, v.x, e.x); v.y = __fmaf_rn(src.eta, v.y, e.y);
+            v.z = __fmaf_rn(src.eta, v.z, e.z); v.w = __fmaf_rn(src.eta, v.w, e.w);
+          }
           hist_elem(mag_key(v.x), level, prefix, target);
           hist_elem(mag_key(v.y), level, prefix, target);
           hist_elem(mag_key(v.z), level, prefix, target);
           hist_elem(mag_key(v.w), level, prefix, target);
         }
       } else {
-        for (int i = tid; i < ti.cnt; i += THREADS) hist_elem(mag_key(bp[i]), level, prefix, target);
+        for (int i = tid; i < ti.cnt; i += THREADS)
+          hist_elem(mag_key(src.recompute ? __fmaf_rn(src.eta, bp[i], eb[i]) : bp[i]), level, prefix, target);
       }
     } else {
       rj = w.x;
