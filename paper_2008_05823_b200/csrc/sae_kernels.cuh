@@ -244,7 +244,6 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   float* ep = A.e_srv + pbase;
   const float* __restrict__ dp = (RECOMP ? A.m : A.D) + pbase;
   const float* __restrict__ eo = A.ebar_in + pbase;      // read only when RECOMP
-  const float Kf = (float)P.K;
   if (ti.cnt == TILE) {
 #pragma unroll 2
     for (int it = 0; it < VEC_ITERS; ++it) {
@@ -397,7 +396,6 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
   float* ebp = A.ebar + pbase;
   const float* __restrict__ src = (AVG == AVG_RECOMPUTE) ? A.m + pbase : A.D + pbase;
   u32* mwp = A.mask_srv + (pbase >> 5);
-  const float Kf = (float)P.K;
 
   if (ti.cnt == TILE) {
 #pragma unroll 2

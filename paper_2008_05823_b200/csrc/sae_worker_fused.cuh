@@ -177,7 +177,6 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     return;
   }
 
-  const float Kf = (float)K;
   if (warp > FW_WARPS) {
     // ---------------- averagers: ebar' = (1/K) sum_k ( fma(eta_prev, m_k, ebar) - C(.) ), k in order ----------------
     constexpr int NA = FW_AVG_WARPS * 32;
@@ -330,7 +329,6 @@ __global__ void __launch_bounds__(THREADS) k_materialize_avg(Plan P, const float
                                                               const float* __restrict__ scale_prev, float eta_prev,
                                                               float* __restrict__ etmp) {
   const TileInfo ti = tile_info(P, blockIdx.x);
-  const float Kf = (float)P.K;
   for (int i = threadIdx.x; i < ti.cnt; i += THREADS) {
     const long long p = ti.poff + ti.t0 + i;
     const float eb = ebar[p];

@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 SIZES = [33, 4096, 5000, 700, 3 * 4096]
 
 
-@pytest.mark.parametrize("comp,p,K", [(so.SIGN, 1, 4), (so.SIGN, 3, 3), (so.TOPK, 2, 4), (so.SIGN, 0, 2)])
+@pytest.mark.parametrize("comp,p,K", [(so.SIGN, 1, 4), (so.SIGN, 3, 3), (so.TOPK, 2, 4), (so.TOPK, 1, 3), (so.SIGN, 0, 2)])
 def test_resume_continues_bit_for_bit(comp, p, K):
     """Save after 5 steps, restore into a fresh handle (different x0), continue: same bits as the oracle."""
     import torch
@@ -47,7 +47,7 @@ def test_resume_continues_bit_for_bit(comp, p, K):
         sb._check(sb.lib().sae_save_state(c.h, blob.data_ptr(), 16), "sae_save_state", c.h)
 
 
-@pytest.mark.parametrize("comp,p", [(so.SIGN, 0), (so.SIGN, 1), (so.SIGN, 3), (so.TOPK, 2)])
+@pytest.mark.parametrize("comp,p", [(so.SIGN, 0), (so.SIGN, 1), (so.SIGN, 3), (so.TOPK, 2), (so.TOPK, 1)])
 def test_gradient_mismatch_bounds(comp, p):
     """|| e + ebar ||^2 and (1/K) sum_k || e + ebar - e^(k) ||^2 (Section 3) from the oracle's errors."""
     import torch
