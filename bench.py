@@ -219,6 +219,8 @@ def main():
     ap.add_argument("--single-way", action="store_true", help="server sends its Delta uncompressed (SC)")
     ap.add_argument("--momentum", type=float, default=None, help="0 gives the SGD / SignSGD variants")
     ap.add_argument("--topk-percent", type=float, default=None, help="Top-K sparsity in percent (Table 1: 1, 5, 10)")
+    ap.add_argument("--block-size", type=int, default=0,
+                    help="block-wise compression: cut every tensor into segments of this many elements")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -242,6 +244,9 @@ def main():
         w.compressor = configs.TOPK
         w.topk_num, w.topk_den = int(round(args.topk_percent * 10)), 1000
         w.name += f"_top{args.topk_percent:g}pct"
+    if args.block_size > 0:
+        w.tensor_sizes = configs.blockwise_sizes(w.tensor_sizes, args.block_size)
+        w.name += f"_blk{args.block_size}"
     p = args.avg_period
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -51,6 +51,21 @@ def encoder_sizes(layers: int = 12, hidden: int = 768, ffn: int = 3072, vocab: i
     return sizes
 
 
+def blockwise_sizes(tensor_sizes: List[int], block: int) -> List[int]:
+    """Block-wise compression (the block-wise scaled sign of the related work, Section 2): every tensor is
+    cut into consecutive segments of `block` elements (the last one of a tensor may be shorter) and each
+    segment is compressed on its own.  To the library a segment is simply a tensor of the list."""
+    if block < 1:
+        raise ValueError("block must be >= 1")
+    out: List[int] = []
+    for n in tensor_sizes:
+        full, rest = divmod(n, block)
+        out += [block] * full
+        if rest:
+            out.append(rest)
+    return out
+
+
 @dataclass
 class Workload:
     name: str

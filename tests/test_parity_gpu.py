@@ -327,3 +327,12 @@ def test_config0_full_trajectory(seed, p):
 def test_config1_full_trajectory(p):
     """All 200 iterations of config 1 (heavy-tailed gradients, weight decay)."""
     _trajectory_device_inputs(1, p, 200, 0)
+
+
+@pytest.mark.parametrize("block,p", [(4096, 1), (4096, 0), (8192, 3), (1000, 1)])
+def test_blockwise_sign(block, p):
+    """Block-wise scaled sign (related work, Section 2): fixed-size segments of every tensor, each with its
+    own scale; to the library a segment is a tensor of the list."""
+    sizes = configs.blockwise_sizes([3 * 4096 + 17, 4096, 5, 20000, 8192], block)
+    assert sum(sizes) == 3 * 4096 + 17 + 4096 + 5 + 20000 + 8192
+    run_pair(4, sizes, so.SIGN, 6, p=p, lrs=[0.1, 0.05])

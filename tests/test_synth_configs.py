@@ -56,3 +56,16 @@ def test_x0():
     x = synth.x0_numpy(0, 100000)
     assert abs(x.std() - 0.05) < 0.002 and abs(x.mean()) < 0.001
     np.testing.assert_array_equal(x[:1000], synth.x0_numpy(0, 1000))
+
+
+def test_blockwise_sizes():
+    from paper_2008_05823_b200 import configs
+    assert configs.blockwise_sizes([10, 4, 3], 4) == [4, 4, 2, 4, 3]
+    assert configs.blockwise_sizes([8], 4) == [4, 4]
+    sizes = configs.resnet50_sizes()
+    blk = configs.blockwise_sizes(sizes, 4096)
+    assert sum(blk) == sum(sizes) and max(blk) == 4096
+    assert len(blk) == sum((n + 4095) // 4096 for n in sizes)
+    import pytest
+    with pytest.raises(ValueError):
+        configs.blockwise_sizes([8], 0)
