@@ -2,7 +2,8 @@
  * sae.h -- C ABI of the Step-Ahead Error Feedback hot path (sm_100a CUDA library, libsae.so).
  *
  * One handle holds the whole state of Algorithm 1 ("Distributed Momentum SGD with Double-Way
- * Compression") for K data-parallel workers simulated as a batch axis on ONE GPU: parameters x,
+ * Compression") for K data-parallel workers simulated as a batch axis on ONE GPU (or, in sharded
+ * operation, the rows of some of the workers: see sae_init_shard): parameters x,
  * server error e, per-worker momentum m^(k) and per-worker error e^(k).  The caller supplies the
  * stochastic gradients; the library performs every other line of the algorithm in CUDA kernels.
  *
@@ -179,6 +180,47 @@ int sae_get_kernel_times(sae_handle *h, float *ms_host, int64_t *launches_host);
 const char *sae_kernel_name(int32_t slot);
 /* Total kernels launched by this handle so far. */
 int64_t sae_kernel_launches(const sae_handle *h);
+
+/*
+ * Sharded operation: the K workers of Algorithm 1 spread over several handles ("shards": one per GPU /
+ * process), scaled-sign compressor.  A shard owns workers worker_begin .. worker_begin+num_local_workers-1:
+ * their momentum, error and message rows live in its memory.  The server lines ("Server: receive ...,
+ * send C(Delta)") are replicated: every shard keeps x and the server error e and computes the same bits,
+ * because it reads all K messages (1 scale per tensor + 1 bit per element per worker, Eq. 2) in k order.
+ * The exchange of Algorithm 1 ("send C(Delta^(k)) to the server") is not a separate copy: the server pass
+ * reads every worker's sign words and scales in place from the owner's memory through a table of row
+ * pointers -- plain loads, over NVLink when the owner is another GPU -- so gather and aggregation are one
+ * kernel.  Error averaging (pre-step, every p iterations) likewise reads the owners' stored model
+ * differences in place.
+ *
+ *   sae_init_shard    cfg->num_workers is K of the whole job; otherwise as sae_init (compressor must be
+ *                     SAE_COMPRESSOR_SIGN).  Worker indices of the getters are LOCAL (0 .. num_local-1).
+ *   sae_shard_export  writes SAE_SHARD_BLOB_BYTES bytes (HOST) describing where this shard's rows live: raw
+ *                     pointers for handles of the same process, CUDA IPC handles for other processes.
+ *   sae_shard_attach  makes the rows of one exported blob (any shard's, including this handle's own) known
+ *                     to this handle.  Every handle must attach the blobs of all shards before stepping.
+ *                     Buffers of another process are mapped with cudaIpcOpenMemHandle (peer access enabled
+ *                     lazily) and unmapped by sae_shard_detach or sae_destroy.
+ *   sae_shard_detach  forgets every attached row and unmaps other processes' buffers (waits for the stream
+ *                     first).  An owner must not be destroyed while another process still maps its rows:
+ *                     detach everywhere, synchronise the ranks, then destroy.
+ *   sae_step_begin    worker lines of iteration t for the local workers: grads_local is [num_local][d].
+ *   sae_step_end      server lines, re-update and the pre-step of iteration t+1.
+ *
+ * Ordering is the caller's duty (a host barrier after synchronising the streams, or a collective that is
+ * stream-ordered on every shard): every shard's sae_step_begin work must be complete before any shard's
+ * sae_step_end work starts (the messages are read remotely), and every shard's sae_step_end work before
+ * any shard's next sae_step_begin (which overwrites them).  Shards of one process on one stream need
+ * nothing: stream order already gives both.  sae_step and sae_step_host refuse a sharded handle.
+ */
+#define SAE_SHARD_BLOB_BYTES 512
+int sae_init_shard(const sae_config *cfg, int32_t worker_begin, int32_t num_local_workers, const float *x0,
+                   sae_handle **out);
+int sae_shard_export(sae_handle *h, void *blob_host, size_t bytes);
+int sae_shard_attach(sae_handle *h, const void *blob_host, size_t bytes);
+int sae_shard_detach(sae_handle *h);
+int sae_step_begin(sae_handle *h, const float *grads_local, float lr);
+int sae_step_end(sae_handle *h);
 
 /* Frees everything the handle owns (synchronises first). NULL is allowed. */
 void sae_destroy(sae_handle *h);

@@ -24,7 +24,10 @@ EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_p
            "sae_get_state", "sae_iteration", "sae_num_params", "sae_num_words", "sae_sync", "sae_set_profiling",
            "sae_get_kernel_times", "sae_kernel_name", "sae_kernel_launches", "sae_destroy", "sae_strerror",
            "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements", "sae_state_bytes",
-           "sae_save_state", "sae_load_state", "sae_get_mismatch"]
+           "sae_save_state", "sae_load_state", "sae_get_mismatch", "sae_init_shard", "sae_shard_export",
+           "sae_shard_attach", "sae_shard_detach", "sae_step_begin", "sae_step_end"]
+
+SHARD_BLOB_BYTES = 512
 
 
 class SaeConfig(C.Structure):
@@ -80,6 +83,12 @@ def lib():
         L.sae_save_state.argtypes = [vp, vp, C.c_size_t]
         L.sae_load_state.argtypes = [vp, vp, C.c_size_t]
         L.sae_get_mismatch.argtypes = [vp, vp]
+        L.sae_init_shard.argtypes = [C.POINTER(SaeConfig), i32, i32, vp, C.POINTER(vp)]
+        L.sae_shard_export.argtypes = [vp, vp, C.c_size_t]
+        L.sae_shard_attach.argtypes = [vp, vp, C.c_size_t]
+        L.sae_shard_detach.argtypes = [vp]
+        L.sae_step_begin.argtypes = [vp, vp, f32]
+        L.sae_step_end.argtypes = [vp]
         L.sae_sign_compress_noalloc.argtypes = [vp, i64, vp, vp, vp, vp]
         L.sae_noalloc_max_elements.argtypes = []
         L.sae_noalloc_max_elements.restype = i64
@@ -93,10 +102,14 @@ def _check(status, what, handle=None):
 
 
 class Sae:
-    """One Algorithm-1 run on one GPU.  Methods mirror the C entry points one to one."""
+    """One Algorithm-1 run on one GPU.  Methods mirror the C entry points one to one.
+
+    With `shard=(worker_begin, num_local_workers)` the handle is one shard of a run whose K = num_workers
+    workers are spread over several handles (sae_init_shard): `step_begin` / `step_end` replace `step`,
+    gradients are [num_local][d], and worker indices of the getters are local."""
 
     def __init__(self, num_workers, tensor_sizes, x0, compressor=SIGN, server_compress=1, mode=SAEF, avg_period=0,
-                 momentum=0.9, weight_decay=0.0, topk_num=1, topk_den=100, device=None, stream=None):
+                 momentum=0.9, weight_decay=0.0, topk_num=1, topk_den=100, device=None, stream=None, shard=None):
         import torch
         self.torch = torch
         if not (x0.is_cuda and x0.dtype == torch.float32 and x0.is_contiguous()):
@@ -113,7 +126,14 @@ class Sae:
                         server_compress, mode, avg_period, momentum, weight_decay, topk_num, topk_den,
                         self.device.index or 0, C.c_void_p(self.stream))
         h = C.c_void_p()
-        _check(lib().sae_init(C.byref(cfg), x0.data_ptr(), C.byref(h)), "sae_init")
+        self.shard = shard
+        self.K_total = self.K
+        if shard is None:
+            _check(lib().sae_init(C.byref(cfg), x0.data_ptr(), C.byref(h)), "sae_init")
+        else:
+            _check(lib().sae_init_shard(C.byref(cfg), int(shard[0]), int(shard[1]), x0.data_ptr(), C.byref(h)),
+                   "sae_init_shard")
+            self.K = int(shard[1])          # rows held here: gradients are [K][d], getters take 0..K-1
         self.h = h
         self.d = int(lib().sae_num_params(h))
         self.nwords = int(lib().sae_num_words(h))
@@ -138,6 +158,29 @@ class Sae:
         if not (grads.is_cuda and grads.dtype == t.float32 and grads.is_contiguous() and grads.numel() == self.K * self.d):
             raise ValueError("grads must be a contiguous float32 CUDA tensor of K*d elements")
         _check(lib().sae_step(self.h, grads.data_ptr(), lr), "sae_step", self.h)
+
+    def shard_export(self):
+        """Where this shard's message rows live, as SHARD_BLOB_BYTES bytes to hand to every shard."""
+        buf = (C.c_ubyte * SHARD_BLOB_BYTES)()
+        _check(lib().sae_shard_export(self.h, buf, SHARD_BLOB_BYTES), "sae_shard_export", self.h)
+        return bytes(buf)
+
+    def shard_attach(self, blob):
+        buf = (C.c_ubyte * SHARD_BLOB_BYTES).from_buffer_copy(blob)
+        _check(lib().sae_shard_attach(self.h, buf, SHARD_BLOB_BYTES), "sae_shard_attach", self.h)
+
+    def shard_detach(self):
+        _check(lib().sae_shard_detach(self.h), "sae_shard_detach", self.h)
+
+    def step_begin(self, grads_local, lr):
+        t = self.torch
+        if not (grads_local.is_cuda and grads_local.dtype == t.float32 and grads_local.is_contiguous()
+                and grads_local.numel() == self.K * self.d):
+            raise ValueError("grads_local must be a contiguous float32 CUDA tensor of num_local*d elements")
+        _check(lib().sae_step_begin(self.h, grads_local.data_ptr(), lr), "sae_step_begin", self.h)
+
+    def step_end(self):
+        _check(lib().sae_step_end(self.h), "sae_step_end", self.h)
 
     def step_host(self, grads_host, lr):
         t = self.torch

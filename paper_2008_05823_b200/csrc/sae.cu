@@ -9,6 +9,7 @@
 #include <cudaTypedefs.h>
 #include <cstdio>
 #include <cstring>
+#include <unistd.h>
 #include <new>
 #include <vector>
 
@@ -73,6 +74,18 @@ struct sae_handle {
   int topk_nod;            // Top-K with p = 1: model differences never stored, two uniform-error buffers
   float* ebar_alt;
   int64_t launches;
+  // sharded operation: this handle owns workers k0 .. k0+P.K-1 of K_total; the server lines run on every shard
+  int shard, k0, K_total;
+  Plan P_all;                       // the plan with K = K_total (server pass, averaging)
+  int attached;                     // workers whose message rows are known
+  int mid_step;                     // sae_step_begin done, sae_step_end due
+  float lr_pending;
+  std::vector<const u32*> h_word_rows;
+  std::vector<const float*> h_scale_rows[2], h_d_rows;
+  const u32** d_word_rows;
+  const float** d_scale_rows[2];
+  const float** d_d_rows;
+  std::vector<void*> ipc_opened;    // mappings of other processes' buffers, closed by sae_destroy
   // cached step graphs
   int graphs_enabled, graph_misses;
   uint64_t graph_clock;
@@ -151,6 +164,9 @@ void free_all(sae_handle* h) {
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
+  void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows};
+  for (void* p : tabs) if (p) cudaFree(p);
+  for (void* p : h->ipc_opened) cudaIpcCloseMemHandle(p);
   if (h->status_host) cudaFreeHost(h->status_host);
   for (auto& g : h->graphs) cudaGraphExecDestroy(g.exec);
   for (auto& ep : h->pending) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
@@ -472,9 +488,10 @@ struct CkptHeader {
   int64_t d, t;
   int32_t esrc, last;
   float eta_prev;
+  int32_t worker_begin, num_workers_total;     // which workers of how many this handle owns (sharded operation)
   int32_t pad;
 };
-constexpr uint64_t kCkptMagic = 0x5341455F434B5031ull;   // "SAE_CKP1"
+constexpr uint64_t kCkptMagic = 0x5341455F434B5032ull;   // "SAE_CKP2"
 
 struct CkptSection { void* ptr; size_t bytes; };
 
@@ -504,7 +521,12 @@ size_t ckpt_bytes(sae_handle* h) {
 
 extern "C" {
 
-int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
+}  // extern "C"
+
+namespace {
+
+// sae_init and sae_init_shard: worker rows k0 .. k0+K_loc-1 of cfg->num_workers are held here
+int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float* x0, sae_handle** out) {
   if (out) *out = nullptr;
   if (!cfg || !x0 || !out) return SAE_ERR_INVALID_ARG;
   if (cfg->abi_version != SAE_ABI_VERSION) return SAE_ERR_ABI;
@@ -517,7 +539,9 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   if (cfg->compressor == SAE_COMPRESSOR_TOPK && (cfg->topk_den == 0 || cfg->topk_num > cfg->topk_den))
     return SAE_ERR_INVALID_ARG;
   if (cfg->device < 0) return SAE_ERR_INVALID_ARG;
-  const int T = cfg->num_tensors, K = cfg->num_workers;
+  if (k0 < 0 || K_loc < 1 || k0 + K_loc > cfg->num_workers) return SAE_ERR_INVALID_ARG;
+  if (shard && cfg->compressor != SAE_COMPRESSOR_SIGN) return SAE_ERR_INVALID_ARG;
+  const int T = cfg->num_tensors, K = K_loc;          // K: worker rows held by this handle
   long long d = 0, dpad = 0, ntiles = 0;
   for (int j = 0; j < T; ++j) {
     const int64_t n = cfg->tensor_sizes[j];
@@ -538,8 +562,9 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f;
   h->graphs_enabled = 1; h->graph_misses = 0; h->graph_clock = 0;
-  h->fused_ok = (cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
+  h->fused_ok = (!shard && cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
                  (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
+  h->shard = shard ? 1 : 0; h->k0 = k0; h->K_total = cfg->num_workers; h->attached = 0; h->mid_step = 0;
   for (int i = 0; i < SAE_NUM_KERNELS; ++i) { h->ms[i] = 0; h->cnt[i] = 0; }
   {
     int sms = 0;
@@ -562,7 +587,7 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
   }
   const bool sign = cfg->compressor == SAE_COMPRESSOR_SIGN, topk = cfg->compressor == SAE_COMPRESSOR_TOPK;
   h->topk_nod = (topk && cfg->avg_period == 1) ? 1 : 0;
-  const bool need_D = !((sign || topk) && cfg->avg_period == 1);
+  const bool need_D = shard || !((sign || topk) && cfg->avg_period == 1);
   const long long nwords = dpad / 32;
   const size_t KT = (size_t)K * T;
 
@@ -624,6 +649,9 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
     Plan& P = h->P;
     P.K = K; P.T = T; P.k_pow2 = ((K & (K - 1)) == 0) ? 1 : 0; P.inv_k = 1.0f / (float)K; P.ntiles = (int)ntiles; P.d = d; P.dpad = dpad; P.nwords = nwords;
     P.tile_tensor = h->d_tile_tensor; P.first_tile = h->d_first_tile; P.n = h->d_n; P.off = h->d_off; P.poff = h->d_poff;
+    h->P_all = P;
+    const int Kt = h->K_total;
+    h->P_all.K = Kt; h->P_all.k_pow2 = ((Kt & (Kt - 1)) == 0) ? 1 : 0; h->P_all.inv_k = 1.0f / (float)Kt;
     LAUNCH(h, S_IMPORT, k_import, P.ntiles, P, x0, h->x);
     TRY(cudaGetLastError());
     TRY(cudaStreamSynchronize(h->stream));     // host tables above go out of scope
@@ -634,20 +662,192 @@ int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
     if (dpad >= (1ll << 31) || d >= (1ll << 31) || !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_ok = 0;
   }
   if (rc != SAE_OK) { free_all(h); delete h; return rc; }
+  if (rc == SAE_OK && shard) {
+    const size_t Kt = (size_t)h->K_total;
+    h->h_word_rows.assign(Kt, nullptr); h->h_d_rows.assign(Kt, nullptr);
+    h->h_scale_rows[0].assign(Kt, nullptr); h->h_scale_rows[1].assign(Kt, nullptr);
+    cudaError_t e = dalloc(&h->d_word_rows, Kt);
+    if (e == cudaSuccess) e = dalloc(&h->d_scale_rows[0], Kt);
+    if (e == cudaSuccess) e = dalloc(&h->d_scale_rows[1], Kt);
+    if (e == cudaSuccess) e = dalloc(&h->d_d_rows, Kt);
+    if (e != cudaSuccess) { h->last_cuda_error = (int)e; g_init_cuda_error = (int)e; cudaGetLastError(); rc = SAE_ERR_NOMEM; }
+  }
+  if (rc != SAE_OK) { free_all(h); delete h; return rc; }
   // Pre-step of iteration 0: all errors are zero, so averaging (if (0+1) mod p = 0) changes nothing.
   *out = h;
   return SAE_OK;
 }
 
+// ---- sharded operation ------------------------------------------------------------------------------
+// What a shard publishes: where its workers' message rows (sign words, the two scale buffers) and stored
+// model differences live.  Same process: the raw pointers; another process: CUDA IPC handles.
+struct ShardBlob {
+  uint64_t magic;
+  int32_t pid, device, worker_begin, num_local, T, pad;
+  int64_t nwords, dpad;
+  void* raw[4];                       // words, scale[0], scale[1], D
+  cudaIpcMemHandle_t ipc[4];
+};
+constexpr uint64_t kShardMagic = 0x5341455F53484431ull;   // "SAE_SHD1"
+static_assert(sizeof(ShardBlob) <= SAE_SHARD_BLOB_BYTES, "blob must fit the documented size");
+
+int shard_begin(sae_handle* h, const float* grads, float lr) {
+  const sae_config& c = h->cfg;
+  const Plan& P = h->P;
+  const int cur = 1 - h->last;
+  StepParams sp;
+  sp.mu = c.momentum; sp.eta = lr; sp.lambda = c.weight_decay;
+  sp.saef = (c.mode == SAE_MODE_SAEF); sp.wd = (c.weight_decay != 0.0f);
+  WorkerArgs wa;
+  wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = h->ebar; wa.x = h->x;
+  wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
+  wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
+  wa.cand = cand_args(h, false);
+  // the model differences are always stored: the averaging reads them from every owner
+  if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
+  else launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
+  LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
+         h->scale[cur], h->recs_srv);
+  h->mid_step = 1; h->lr_pending = lr;
+  return check_launch(h);
+}
+
+int shard_end(sae_handle* h) {
+  const sae_config& c = h->cfg;
+  const Plan& PA = h->P_all;
+  const int cur = 1 - h->last;
+  const bool dc = c.server_compress != 0;
+  const bool avg_after = c.avg_period > 0 && ((h->t + 2) % c.avg_period == 0);
+  ServerArgs sa;
+  memset(&sa, 0, sizeof(sa));
+  sa.e_srv = h->e_srv; sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv;
+  sa.status = h->status; sa.word_rows = h->d_word_rows; sa.scale_rows = h->d_scale_rows[cur];
+  ApplyArgs aa;
+  memset(&aa, 0, sizeof(aa));
+  aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
+  aa.eta = h->lr_pending;
+  const int tpb = std::max(1, std::min(8, PA.ntiles / (h->num_sms * 16)));
+  const int nblk = (PA.ntiles + tpb - 1) / tpb;
+  if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, true>), nblk, PA, sa, tpb);
+  else LAUNCH(h, S_SERVER, (k_server_sign<false, true>), nblk, PA, sa, tpb);
+  if (dc) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), PA.ntiles, PA, aa);
+  else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), PA.ntiles, PA, aa);
+  if (avg_after) LAUNCH(h, S_APPLY, k_avg_pull, PA.ntiles, PA, h->d_d_rows, h->d_scale_rows[cur], h->ebar);
+  h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
+  h->last = cur; h->eta_prev = h->lr_pending; h->t += 1; h->mid_step = 0;
+  return check_launch(h);
+}
+
+}  // namespace
+
+extern "C" {
+
+int sae_init(const sae_config* cfg, const float* x0, sae_handle** out) {
+  if (out) *out = nullptr;
+  if (!cfg) return SAE_ERR_INVALID_ARG;
+  return init_impl(cfg, 0, cfg->num_workers, false, x0, out);
+}
+
+int sae_init_shard(const sae_config* cfg, int32_t worker_begin, int32_t num_local_workers, const float* x0,
+                   sae_handle** out) {
+  if (out) *out = nullptr;
+  if (!cfg) return SAE_ERR_INVALID_ARG;
+  return init_impl(cfg, worker_begin, num_local_workers, true, x0, out);
+}
+
+int sae_shard_export(sae_handle* h, void* blob_host, size_t bytes) {
+  if (!h || !blob_host || bytes < SAE_SHARD_BLOB_BYTES || !h->shard) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  ShardBlob b;
+  memset(&b, 0, sizeof(b));
+  b.magic = kShardMagic; b.pid = (int32_t)getpid(); b.device = h->device; b.worker_begin = h->k0; b.num_local = h->P.K;
+  b.T = h->P.T; b.nwords = h->P.nwords; b.dpad = h->P.dpad;
+  b.raw[0] = h->words; b.raw[1] = h->scale[0]; b.raw[2] = h->scale[1]; b.raw[3] = h->D;
+  for (int q = 0; q < 4; ++q) SAE_CUDA(h, cudaIpcGetMemHandle(&b.ipc[q], b.raw[q]));
+  memset(blob_host, 0, SAE_SHARD_BLOB_BYTES);
+  memcpy(blob_host, &b, sizeof(b));
+  return SAE_OK;
+}
+
+int sae_shard_attach(sae_handle* h, const void* blob_host, size_t bytes) {
+  if (!h || !blob_host || bytes < SAE_SHARD_BLOB_BYTES || !h->shard || h->mid_step) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  ShardBlob b;
+  memcpy(&b, blob_host, sizeof(b));
+  if (b.magic != kShardMagic || b.T != h->P.T || b.nwords != h->P.nwords || b.dpad != h->P.dpad || b.worker_begin < 0 ||
+      b.num_local < 1 || b.worker_begin + b.num_local > h->K_total)
+    return SAE_ERR_INVALID_ARG;
+  for (int q = 0; q < b.num_local; ++q)
+    if (h->h_word_rows[(size_t)b.worker_begin + q]) return SAE_ERR_INVALID_ARG;      // rows already attached
+  void* base[4];
+  if (b.pid == (int32_t)getpid()) {
+    for (int q = 0; q < 4; ++q) base[q] = b.raw[q];
+  } else {
+    for (int q = 0; q < 4; ++q) {
+      SAE_CUDA(h, cudaIpcOpenMemHandle(&base[q], b.ipc[q], cudaIpcMemLazyEnablePeerAccess));
+      h->ipc_opened.push_back(base[q]);
+    }
+  }
+  for (int q = 0; q < b.num_local; ++q) {
+    const size_t k = (size_t)b.worker_begin + q;
+    h->h_word_rows[k] = (const u32*)base[0] + (size_t)q * b.nwords;
+    h->h_scale_rows[0][k] = (const float*)base[1] + (size_t)q * b.T;
+    h->h_scale_rows[1][k] = (const float*)base[2] + (size_t)q * b.T;
+    h->h_d_rows[k] = (const float*)base[3] + (size_t)q * b.dpad;
+  }
+  h->attached += b.num_local;
+  if (h->attached == h->K_total) {
+    const size_t Kt = (size_t)h->K_total;
+    SAE_CUDA(h, cudaMemcpyAsync(h->d_word_rows, h->h_word_rows.data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    SAE_CUDA(h, cudaMemcpyAsync(h->d_scale_rows[0], h->h_scale_rows[0].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    SAE_CUDA(h, cudaMemcpyAsync(h->d_scale_rows[1], h->h_scale_rows[1].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    SAE_CUDA(h, cudaMemcpyAsync(h->d_d_rows, h->h_d_rows.data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  }
+  return SAE_OK;
+}
+
+int sae_shard_detach(sae_handle* h) {
+  if (!h || !h->shard || h->mid_step) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  SAE_CUDA(h, cudaStreamSynchronize(h->stream));
+  for (void* p : h->ipc_opened) cudaIpcCloseMemHandle(p);
+  h->ipc_opened.clear();
+  for (auto& r : h->h_word_rows) r = nullptr;
+  for (auto& r : h->h_d_rows) r = nullptr;
+  for (auto& r : h->h_scale_rows[0]) r = nullptr;
+  for (auto& r : h->h_scale_rows[1]) r = nullptr;
+  h->attached = 0;
+  return SAE_OK;
+}
+
+int sae_step_begin(sae_handle* h, const float* grads_local, float lr) {
+  if (!h || !grads_local || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
+  if (!h->shard || h->mid_step || h->attached != h->K_total) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  return shard_begin(h, grads_local, lr);
+}
+
+int sae_step_end(sae_handle* h) {
+  if (!h || !h->shard || !h->mid_step) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  return shard_end(h);
+}
+
 int sae_step(sae_handle* h, const float* grads, float lr) {
-  if (!h || !grads || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
+  if (!h || !grads || !(lr > 0.0f) || !(lr < 3.0e38f) || h->shard) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   return do_step(h, grads, lr);
 }
 
 int sae_step_host(sae_handle* h, const float* grads_host, float lr) {
-  if (!h || !grads_host || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
+  if (!h || !grads_host || !(lr > 0.0f) || !(lr < 3.0e38f) || h->shard) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   const size_t count = (size_t)h->P.K * (size_t)h->P.d;
@@ -728,7 +928,7 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
 int64_t sae_state_bytes(sae_handle* h) { return h ? (int64_t)ckpt_bytes(h) : -1; }
 
 int sae_save_state(sae_handle* h, void* out, size_t bytes) {
-  if (!h || !out || bytes < ckpt_bytes(h)) return SAE_ERR_INVALID_ARG;
+  if (!h || !out || bytes < ckpt_bytes(h) || h->mid_step) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   CkptHeader hd;
@@ -737,7 +937,7 @@ int sae_save_state(sae_handle* h, void* out, size_t bytes) {
   hd.server_compress = h->cfg.server_compress; hd.mode = h->cfg.mode; hd.avg_period = h->cfg.avg_period;
   hd.topk_num = h->cfg.topk_num; hd.topk_den = h->cfg.topk_den; hd.momentum = h->cfg.momentum;
   hd.weight_decay = h->cfg.weight_decay; hd.d = h->P.d; hd.t = h->t; hd.esrc = h->esrc; hd.last = h->last;
-  hd.eta_prev = h->eta_prev;
+  hd.eta_prev = h->eta_prev; hd.worker_begin = h->k0; hd.num_workers_total = h->K_total;
   SAE_CUDA(h, cudaMemcpyAsync(out, &hd, sizeof(hd), cudaMemcpyHostToDevice, h->stream));
   SAE_CUDA(h, cudaStreamSynchronize(h->stream));        // hd lives on this stack frame
   char* q = (char*)out + 256;
@@ -749,7 +949,7 @@ int sae_save_state(sae_handle* h, void* out, size_t bytes) {
 }
 
 int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
-  if (!h || !in || bytes < ckpt_bytes(h)) return SAE_ERR_INVALID_ARG;
+  if (!h || !in || bytes < ckpt_bytes(h) || h->mid_step) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   CkptHeader hd;
@@ -759,7 +959,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
   if (hd.magic != kCkptMagic || hd.K != h->P.K || hd.T != h->P.T || hd.d != h->P.d || hd.compressor != c.compressor ||
       hd.server_compress != c.server_compress || hd.mode != c.mode || hd.avg_period != c.avg_period ||
       hd.topk_num != c.topk_num || hd.topk_den != c.topk_den || hd.momentum != c.momentum ||
-      hd.weight_decay != c.weight_decay)
+      hd.weight_decay != c.weight_decay || hd.worker_begin != h->k0 || hd.num_workers_total != h->K_total)
     return SAE_ERR_INVALID_ARG;                         // a checkpoint of a different configuration
   if (hd.esrc == ESRC_PENDING_AVG && !h->fused_ok) return SAE_ERR_INVALID_ARG;
   const char* q = (const char*)in + 256;
@@ -772,7 +972,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
 }
 
 int sae_get_mismatch(sae_handle* h, double* out_host) {
-  if (!h || !out_host) return SAE_ERR_INVALID_ARG;
+  if (!h || !out_host || h->shard) return SAE_ERR_INVALID_ARG;     // needs every worker's error in one place
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   if (!h->mismatch) SAE_CUDA(h, dalloc(&h->mismatch, 2));

@@ -73,6 +73,9 @@ struct ServerArgs {
   const float* m;          // [K][dpad] } recompute variant: Delta^(k) = fma(eta, m^(k), ebar_in), not stored
   const float* ebar_in;    // [dpad]    } (ebar_in and ebar are different buffers)
   float eta;
+  // sharded operation: worker k's message lives with its owner (possibly another GPU's memory, read in place)
+  const u32* const* word_rows;     // [K] -> worker k's [nwords] sign words
+  const float* const* scale_rows;  // [K] -> worker k's [T] scales of this step
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -85,6 +88,10 @@ struct ServerArgs {
 // s_k with it (one three-input logic operation) and adds; the additions are issued two at a time as
 // packed fp32 pairs (add.rn.f32x2: two independent round-to-nearest fp32 additions, same results as two
 // scalar ones).
+//
+// TABLE: the K messages are not rows of one local array but are read in place from their owners through a
+// table of row pointers (sharded operation: the gather of the messages and the aggregation are this one
+// pass; plain loads, also from a peer GPU's memory).
 constexpr int SRV_E = 16;   // consecutive parameters per thread; THREADS * SRV_E == TILE
 constexpr int SRV_B = 8;    // workers per batch of word loads
 static_assert(THREADS * SRV_E == TILE, "one pass of the block covers one tile");
@@ -103,10 +110,14 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
   return r;
 }
 
-template <bool DC>
+template <bool DC, bool TABLE = false>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
+  __shared__ const u32* s_row[TABLE ? MAX_WORKERS : 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (TABLE) {
+    for (int k = tid; k < P.K; k += THREADS) s_row[k] = A.word_rows[k];     // visible after the barrier below
+  }
   const int tile0 = blockIdx.x * tiles_per_block;
   const int tile1 = min(P.ntiles, tile0 + tiles_per_block);
   LaneAcc acc; lane_acc_init(acc);
@@ -117,7 +128,8 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
     if (ti.j != cur_j) {
       if (DC && cur_j >= 0) { warp_commit(acc, A.recs_srv + cur_j, A.status); lane_acc_init(acc); }
       __syncthreads();                            // the previous tensor's scales are no longer read
-      for (int k = tid; k < P.K; k += THREADS) s_k[k] = A.scale_cur[(long long)k * P.T + ti.j];
+      for (int k = tid; k < P.K; k += THREADS)
+        s_k[k] = TABLE ? A.scale_rows[k][ti.j] : A.scale_cur[(long long)k * P.T + ti.j];
       __syncthreads();
       cur_j = ti.j;
     }
@@ -143,16 +155,20 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
       // The words of SRV_B workers are fetched as one batch of independent loads, the next batch while
       // this one is consumed: without that the loop waits out one memory latency per worker.
       const u32* wk = wp + wi;                     // worker k's word: stepped by the row pitch, no multiply
+      const long long wofs = (pbase >> 5) + wi;    // (TABLE) the same word inside every worker's own row
       u32 wn[SRV_B];
 #pragma unroll
-      for (int u = 0; u < SRV_B; ++u) wn[u] = (u < P.K) ? __ldg(wk + (long long)u * P.nwords) : 0u;
+      for (int u = 0; u < SRV_B; ++u)
+        wn[u] = (u < P.K) ? __ldg(TABLE ? s_row[u] + wofs : wk + (long long)u * P.nwords) : 0u;
       for (int k0 = 0; k0 < P.K; k0 += SRV_B) {
         u32 w[SRV_B];
 #pragma unroll
         for (int u = 0; u < SRV_B; ++u) w[u] = wn[u];
         wk += (long long)SRV_B * P.nwords;
 #pragma unroll
-        for (int u = 0; u < SRV_B; ++u) wn[u] = (k0 + SRV_B + u < P.K) ? __ldg(wk + (long long)u * P.nwords) : 0u;
+        for (int u = 0; u < SRV_B; ++u)
+          wn[u] = (k0 + SRV_B + u < P.K)
+                      ? __ldg(TABLE ? s_row[k0 + SRV_B + u] + wofs : wk + (long long)u * P.nwords) : 0u;
 #pragma unroll
         for (int u = 0; u < SRV_B; ++u) {
           if (k0 + u < P.K) {
@@ -201,7 +217,7 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
           float a = 0.f;
           const int wi = i >> 5;
           for (int k = 0; k < P.K; ++k) {
-            const u32 w = __ldg(wp + (long long)k * P.nwords + wi) >> lane;
+            const u32 w = __ldg(TABLE ? s_row[k] + (pbase >> 5) + wi : wp + (long long)k * P.nwords + wi) >> lane;
             const float s = s_k[k];
             a = __fadd_rn(a, (w & 1u) ? s : -s);
           }
@@ -323,6 +339,42 @@ __global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const
   } else if (q < K * T + T) {
     L1Record* r = recs_srv + (q - K * T);
     r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0;
+  }
+}
+
+// Sharded operation, error averaging (Algorithm 1, pre-step): ebar = (1/K) sum_k e^(k) in k order, with
+// e^(k) = D^(k) - C(D^(k)) formed from every owner's stored model differences and scales, read in place
+// through row tables (the same subtraction, order and division as the unsharded averaging in k_apply).
+__global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const* __restrict__ d_rows,
+                                                       const float* const* __restrict__ scale_rows, float* ebar) {
+  __shared__ float s_k[MAX_WORKERS];
+  __shared__ const float* s_row[MAX_WORKERS];
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const int tid = threadIdx.x;
+  for (int k = tid; k < P.K; k += THREADS) { s_k[k] = scale_rows[k][ti.j]; s_row[k] = d_rows[k]; }
+  __syncthreads();
+  const long long pbase = ti.poff + ti.t0;
+  if (ti.cnt == TILE) {
+    for (int it = 0; it < VEC_ITERS; ++it) {
+      const int i = it * (THREADS * 4) + tid * 4;
+      float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
+#pragma unroll 4
+      for (int k = 0; k < P.K; ++k) {
+        const float4 v = ld4(s_row[k] + pbase + i);
+        const float s = s_k[k];
+        b0 = __fadd_rn(b0, prev_error<ESRC_LAZY_SIGN>(v.x, s, 0u));
+        b1 = __fadd_rn(b1, prev_error<ESRC_LAZY_SIGN>(v.y, s, 0u));
+        b2 = __fadd_rn(b2, prev_error<ESRC_LAZY_SIGN>(v.z, s, 0u));
+        b3 = __fadd_rn(b3, prev_error<ESRC_LAZY_SIGN>(v.w, s, 0u));
+      }
+      st4(ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
+    }
+  } else {
+    for (int i = tid; i < ti.cnt; i += THREADS) {
+      float b = 0.f;
+      for (int k = 0; k < P.K; ++k) b = __fadd_rn(b, prev_error<ESRC_LAZY_SIGN>(s_row[k][pbase + i], s_k[k], 0u));
+      ebar[pbase + i] = div_by_k(P, b);
+    }
   }
 }
 

@@ -1,0 +1,88 @@
+"""Sharded operation across processes: one rank per GPU, each owning a contiguous block of the K workers
+of Algorithm 1 (scaled sign).  torch.distributed is used for plumbing only -- exchanging the 512-byte
+descriptions of where each rank's message rows live (once, at start) and the two barriers per step; the
+messages themselves are never copied by a collective: every rank's server pass reads them in place from
+the owners' memory (CUDA IPC mappings, NVLink between GPUs), inside the aggregation kernel.
+
+The engine is injected so that the rank logic can be exercised without a GPU (tests use a recording fake).
+"""
+from typing import Callable, List, Optional, Tuple
+
+
+def worker_range(num_workers: int, world: int, rank: int) -> Tuple[int, int]:
+    """Contiguous split of K workers over `world` ranks: (first worker, how many); the first K mod world
+    ranks hold one more.  Every rank must own at least one worker."""
+    if world < 1 or not (0 <= rank < world):
+        raise ValueError("bad rank / world size")
+    if num_workers < world:
+        raise ValueError("fewer workers than ranks: every rank must own at least one worker")
+    base, rem = divmod(num_workers, world)
+    begin = rank * base + min(rank, rem)
+    return begin, base + (1 if rank < rem else 0)
+
+
+class ShardedRun:
+    """One rank of a sharded run.
+
+    make_engine(worker_begin, num_local) -> object with shard_export() -> bytes, shard_attach(bytes),
+    step_begin(grads_local, lr), step_end(), close() and optionally shard_detach().  `barrier()` must
+    return only when every rank has reached it AND the device work each rank enqueued before it is complete
+    (default: synchronise the CUDA device, then torch.distributed.barrier)."""
+
+    def __init__(self, num_workers: int, make_engine: Callable, group=None, barrier: Optional[Callable] = None):
+        import torch.distributed as dist
+        self.dist = dist
+        self.group = group
+        self.rank = dist.get_rank(group)
+        self.world = dist.get_world_size(group)
+        self.num_workers = num_workers
+        self.begin, self.count = worker_range(num_workers, self.world, self.rank)
+        self.engine = make_engine(self.begin, self.count)
+        self._barrier = barrier if barrier is not None else self._default_barrier
+        blobs: List[Optional[bytes]] = [None] * self.world
+        dist.all_gather_object(blobs, self.engine.shard_export(), group=group)
+        for b in blobs:                       # rank order; includes this rank's own rows
+            self.engine.shard_attach(b)
+        self._readers_pending = False         # peers may still be reading this rank's rows
+        self._barrier()
+
+    def _default_barrier(self):
+        import torch
+        if torch.cuda.is_available():
+            torch.cuda.synchronize()
+        self.dist.barrier(group=self.group)
+
+    def step(self, grads_local, lr: float):
+        """Iteration t for this rank's workers.  The barrier that protects the message rows from being
+        overwritten while peers still read them is taken lazily, at the start of the next step, so the
+        caller's gradient computation overlaps the slowest peer's server pass."""
+        if self._readers_pending:
+            self._barrier()
+        self.engine.step_begin(grads_local, lr)
+        self._barrier()                       # every rank's messages are complete
+        self.engine.step_end()
+        self._readers_pending = True
+
+    def finish(self):
+        """Waits until no peer reads this rank's rows any more (call before reading results)."""
+        if self._readers_pending:
+            self._barrier()
+            self._readers_pending = False
+
+    def close(self):
+        """Orderly shutdown: every rank unmaps its peers' rows before any rank frees its own."""
+        self.finish()
+        if hasattr(self.engine, "shard_detach"):
+            self.engine.shard_detach()
+        self._barrier()
+        self.engine.close()
+
+
+def sharded_sae(num_workers, tensor_sizes, x0, group=None, barrier=None, **kw) -> ShardedRun:
+    """ShardedRun over the CUDA library: every rank passes the same num_workers, tensor_sizes, x0 and options."""
+    from . import binding as sb
+
+    def make(begin, count):
+        return sb.Sae(num_workers, tensor_sizes, x0, compressor=sb.SIGN, shard=(begin, count), **kw)
+
+    return ShardedRun(num_workers, make, group=group, barrier=barrier)

@@ -1,0 +1,120 @@
+"""Sharded operation (the workers of Algorithm 1 spread over several handles) against the CPU oracle.
+
+* Shards of one process on one stream: every shard must hold the oracle's x and server error bit for bit,
+  and its own workers' momentum, error, scales and sign words -- the server pass reads all K messages in
+  place through the row tables, in k order.
+* Two processes on ONE GPU (gloo for the rendezvous and the barriers): the same through CUDA IPC mappings.
+  No kernel waits on another: the order between the ranks is enforced on the host.
+"""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+from oracle import sae_oracle as so
+from paper_2008_05823_b200 import binding as sb
+from paper_2008_05823_b200 import synth
+from paper_2008_05823_b200.sharded import worker_range
+from parity_util import assert_same
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SIZES = [1, 33, 4096, 5000, 3 * 4096 + 7, 64, 20000]
+
+
+def compare_shard(shard, begin, orc, dc, tag):
+    cpu = lambda t: t.cpu().numpy()
+    shard.sync()
+    assert shard.iteration == orc.iteration
+    assert_same(f"{tag} x", cpu(shard.get_params()), orc.get(orc.X))
+    assert_same(f"{tag} e_srv", cpu(shard.get_state(sb.STATE_SERVER_ERROR)), orc.get(orc.E_SRV))
+    for kl in range(shard.K):
+        k = begin + kl
+        assert_same(f"{tag} m[{k}]", cpu(shard.get_state(sb.STATE_MOMENTUM, kl)), orc.get(orc.M, k))
+        assert_same(f"{tag} e[{k}]", cpu(shard.get_state(sb.STATE_WORKER_ERROR, kl)), orc.get(orc.E, k))
+        assert_same(f"{tag} step_ahead[{k}]", cpu(shard.get_step_ahead(kl)), orc.step_ahead(k))
+        if orc.iteration:
+            assert_same(f"{tag} scales[{k}]", cpu(shard.get_state(sb.STATE_WORKER_SCALES, kl)), orc.get(orc.SCALES, k))
+            assert_same(f"{tag} words[{k}]", cpu(shard.get_state(sb.STATE_WORKER_WORDS, kl)).view(np.uint32),
+                        so.pack_signs(orc.get(orc.DELTA, k), orc.sizes))
+    if dc and orc.iteration:
+        assert_same(f"{tag} scales_srv", cpu(shard.get_state(sb.STATE_SERVER_SCALES)), orc.get(orc.SCALES_SRV))
+        assert_same(f"{tag} words_srv", cpu(shard.get_state(sb.STATE_SERVER_WORDS)).view(np.uint32),
+                    so.pack_signs(orc.get(orc.DELTA_SRV), orc.sizes))
+
+
+@pytest.mark.parametrize("K,world", [(4, 2), (3, 2), (5, 3), (4, 4), (2, 1)])
+@pytest.mark.parametrize("p", [0, 1, 3])
+@pytest.mark.parametrize("dc,mode,lam", [(1, so.SAEF, 0.0), (0, so.EF, 1e-4)])
+def test_shards_in_one_process_match_the_oracle(K, world, p, dc, mode, lam):
+    import torch
+    d = int(np.sum(SIZES))
+    seed = 11
+    scales = synth.tensor_scales(seed, len(SIZES), -4.0, -1.0)
+    x0 = synth.x0_numpy(seed, d)
+    kw = dict(compressor=so.SIGN, server_compress=dc, mode=mode, avg_period=p, momentum=0.9, weight_decay=lam)
+    orc = so.Oracle(K, SIZES, x0, threads=4, **kw)
+    x0d = torch.from_numpy(x0).cuda()
+    ranges = [worker_range(K, world, r) for r in range(world)]
+    shards = [sb.Sae(K, SIZES, x0d, shard=rg, **kw) for rg in ranges]
+    blobs = [s.shard_export() for s in shards]
+    for s in shards:
+        for b in blobs:
+            s.shard_attach(b)
+    lrs = [0.1, 0.05, 0.2]
+    for t in range(7):
+        g = synth.grads_numpy(seed, t, K, SIZES, scales)
+        orc.step(g, lrs[t % 3])
+        gd = torch.from_numpy(g).cuda().view(K, d)
+        for s, (b, c) in zip(shards, ranges):
+            s.step_begin(gd[b:b + c].contiguous(), lrs[t % 3])
+        for s in shards:                     # same stream: every begin is ordered before every end
+            s.step_end()
+        for s, (b, c) in zip(shards, ranges):
+            compare_shard(s, b, orc, dc, tag=f"K={K} world={world} p={p} shard@{b} t={t + 1}")
+    for s in shards:
+        s.close()
+
+
+def test_sharded_handle_checks_its_arguments():
+    import torch
+    d = int(np.sum(SIZES))
+    x0 = torch.zeros(d, device="cuda")
+    with pytest.raises(sb.SaeError):
+        sb.Sae(4, SIZES, x0, compressor=so.TOPK, shard=(0, 2))          # scaled sign only
+    with pytest.raises(sb.SaeError):
+        sb.Sae(4, SIZES, x0, shard=(3, 2))                               # rows beyond K
+    a = sb.Sae(4, SIZES, x0, shard=(0, 2))
+    g = torch.zeros(2 * d, device="cuda")
+    with pytest.raises(sb.SaeError):
+        a.step_begin(g, 0.1)                                             # peers not attached yet
+    with pytest.raises(sb.SaeError):
+        a.step(g, 0.1)                                                   # the unsharded step is refused
+    blob = a.shard_export()
+    a.shard_attach(blob)
+    with pytest.raises(sb.SaeError):
+        a.shard_attach(blob)                                             # rows attached twice
+    with pytest.raises(sb.SaeError):
+        a.step_end()                                                     # no step in flight
+    other = sb.Sae(4, SIZES + [5], torch.zeros(d + 5, device="cuda"), shard=(2, 2))
+    with pytest.raises(sb.SaeError):
+        a.shard_attach(other.shard_export())                             # a different parameter list
+    a.close()
+    other.close()
+
+
+def test_two_processes_on_one_gpu_through_ipc():
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="2")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
+           "127.0.0.1", "--master-port", "29741", os.path.join(ROOT, "tests", "shard_ipc_worker.py")]
+    res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0, (res.stdout[-2000:], res.stderr[-3000:])
+    assert res.stdout.count("SHARD_OK") == 2, res.stdout[-2000:]
+
+
+def test_unsharded_reference_run_on_the_same_sizes():
+    from test_parity_gpu import run_pair
+    run_pair(4, SIZES, so.SIGN, 5, p=3, seed=11)
