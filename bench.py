@@ -201,6 +201,112 @@ def algorithmic_bytes(w, avg_period):
     return step, worker, variant
 
 
+def run_sharded(args, w, p, rank, local_rank, world):
+    """One job whose K workers are split over the ranks (scaled sign).  Each rank runs the worker lines of
+    its own workers; the server pass of every rank reads all K messages in place from their owners."""
+    import torch
+    import torch.distributed as dist
+    from paper_2008_05823_b200 import binding as sb
+    from paper_2008_05823_b200 import configs, synth
+    from paper_2008_05823_b200.sharded import sharded_sae, worker_range
+
+    if w.compressor != configs.SIGN:
+        raise SystemExit("--sharded: scaled sign only")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(stream)
+    K, d = w.num_workers, w.d
+    begin, count = worker_range(K, world, rank)
+    scales = synth.workload_scales(w, args.seed)
+    gen = synth.DeviceGenerator(w.tensor_sizes, scales, device=dev)
+    x0 = torch.empty(d, device=dev)
+    gen.x0(x0, args.seed)
+    grad_bytes = 4 * count * d
+    ring = args.ring or int(max(2, min(4, (40 << 30) // grad_bytes, args.steps + args.warmup)))
+    grads = []
+    for t in range(ring):
+        g = torch.empty(count, d, device=dev)
+        gen.grads(g, count, args.seed + 1000 * rank, t, w.outlier_per_65536, w.outlier_mult)   # timing only
+        grads.append(g)
+    kw = dict(server_compress=w.server_compress, mode=w.mode, avg_period=p, momentum=w.momentum,
+              weight_decay=w.weight_decay)
+    if world > 1:
+        run = sharded_sae(K, w.tensor_sizes, x0, **kw)
+        eng = run.engine
+        step = lambda g: run.step(g, w.lr)
+        finish = run.finish
+    else:
+        eng = sb.Sae(K, w.tensor_sizes, x0, compressor=sb.SIGN, shard=(0, K), **kw)
+        eng.shard_attach(eng.shard_export())
+
+        def step(g):                       # one stream: begin is ordered before end, end before the next begin
+            eng.step_begin(g, w.lr)
+            eng.step_end()
+        finish = lambda: None
+    for t in range(args.warmup):
+        step(grads[t % ring])
+    finish()
+    eng.sync()
+    sampler = ClockSampler(local_rank)
+    launches0 = eng.kernel_launches
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler.start()
+    t0 = time.perf_counter()               # the barriers between the phases are host-side: wall clock around
+    for t in range(args.steps):            # a synchronised region (device events would miss the waits)
+        step(grads[(args.warmup + t) % ring])
+    finish()
+    torch.cuda.synchronize()
+    ms_total = 1e3 * (time.perf_counter() - t0)
+    clocks = sampler.stop()
+    gpu_launches = eng.kernel_launches - launches0
+    eng.sync()
+    ms_total = max_over_ranks(ms_total, dev)
+    ms_per_step = ms_total / args.steps
+    eng.set_profiling(True)
+    for t in range(args.steps):
+        step(grads[(args.warmup + t) % ring])
+    finish()
+    ktimes = eng.get_kernel_times()
+    eng.set_profiling(False)
+    total_k = sum(ms for ms, _ in ktimes.values())
+    kernels = {name: {"launches": cnt, "ms_per_launch": ms / cnt, "share": ms / total_k}
+               for name, (ms, cnt) in ktimes.items()}
+    peak, peak_source = measured_peak()
+    worker_bytes = 20 * count * d          # g R, m RW, Delta RW: the differences are always stored when sharded
+    wk_ms = kernels["worker_pass"]["ms_per_launch"]
+    achieved = worker_bytes / (wk_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": worker_bytes,
+                "ms_per_launch": wk_ms, "peak_source": peak_source, "kernels": kernels,
+                "exchange_bytes_per_rank_per_step": (K - count) * (w.num_tensors * 4 + ((d + 31) // 32) * 4)}
+    if world > 1:
+        run.close()
+    else:
+        eng.close()
+    if rank == 0:
+        line = {"metric": METRIC, "value": 1e3 * args.steps / ms_total, "unit": "steps/s", "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.name + "_sharded", "num_workers": K, "workers_per_rank": count, "d": d,
+                           "num_tensors": w.num_tensors, "compressor": "scaled_sign", "avg_period": p,
+                           "parallelism": f"sharded: {K} workers over {world} rank(s); every rank's server pass reads "
+                                          "all messages in place through row tables",
+                           "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient "
+                                 f"set (ring of {ring})"},
+                "clocks": clocks, "e2e": None, "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": None}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -221,6 +327,9 @@ def main():
     ap.add_argument("--topk-percent", type=float, default=None, help="Top-K sparsity in percent (Table 1: 1, 5, 10)")
     ap.add_argument("--block-size", type=int, default=0,
                     help="block-wise compression: cut every tensor into segments of this many elements")
+    ap.add_argument("--sharded", action="store_true",
+                    help="sharded operation: the workers are split over the ranks (strong scaling of one job); "
+                         "with one rank it times the same two-phase, table-driven path on one GPU")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -254,6 +363,9 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, w, p, rank)
+        return
+    if args.sharded:
+        run_sharded(args, w, p, rank, local_rank, world)
         return
 
     import numpy as np
