@@ -118,3 +118,46 @@ def test_two_processes_on_one_gpu_through_ipc():
 def test_unsharded_reference_run_on_the_same_sizes():
     from test_parity_gpu import run_pair
     run_pair(4, SIZES, so.SIGN, 5, p=3, seed=11)
+
+
+def test_config2_fullsize_shards_equal_the_single_handle():
+    """Config 2 at full size (16 workers x 25.6 M parameters): three shards (6 + 5 + 5 workers) against the
+    unsharded handle -- itself checked against the oracle at this size elsewhere -- on every piece of state,
+    for a schedule with and one without error averaging."""
+    import torch
+    from paper_2008_05823_b200 import configs
+    w = configs.workload(2)
+    K, sizes, d = w.num_workers, w.tensor_sizes, w.d
+    scales = synth.workload_scales(w, 0)
+    gen = synth.DeviceGenerator(sizes, scales)
+    x0 = torch.empty(d, device="cuda")
+    gen.x0(x0, 0)
+    g = torch.empty(K, d, device="cuda")
+    for p, steps in ((0, 4), (3, 7)):
+        kw = dict(compressor=so.SIGN, avg_period=p, momentum=w.momentum, weight_decay=w.weight_decay)
+        one = sb.Sae(K, sizes, x0, **kw)
+        ranges = [worker_range(K, 3, r) for r in range(3)]
+        shards = [sb.Sae(K, sizes, x0, shard=rg, **kw) for rg in ranges]
+        blobs = [s.shard_export() for s in shards]
+        for s in shards:
+            for b in blobs:
+                s.shard_attach(b)
+        for t in range(steps):
+            gen.grads(g, K, 0, t, w.outlier_per_65536, w.outlier_mult)
+            one.step(g, w.lr)
+            for s, (b, c) in zip(shards, ranges):
+                s.step_begin(g[b:b + c], w.lr)
+            for s in shards:
+                s.step_end()
+        one.sync()
+        x_ref, es_ref = one.get_params(), one.get_state(sb.STATE_SERVER_ERROR)
+        for s, (b, c) in zip(shards, ranges):
+            s.sync()
+            assert torch.equal(s.get_params().view(torch.int32), x_ref.view(torch.int32)), f"p={p} x of shard@{b}"
+            assert torch.equal(s.get_state(sb.STATE_SERVER_ERROR).view(torch.int32), es_ref.view(torch.int32))
+            for kl in (0, c - 1):
+                for which in (sb.STATE_MOMENTUM, sb.STATE_WORKER_ERROR, sb.STATE_WORKER_WORDS, sb.STATE_WORKER_SCALES):
+                    a, r = s.get_state(which, kl), one.get_state(which, b + kl)
+                    assert torch.equal(a.view(torch.int32), r.view(torch.int32)), f"p={p} state {which} worker {b + kl}"
+            s.close()
+        one.close()
