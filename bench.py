@@ -194,6 +194,10 @@ def algorithmic_bytes(w, avg_period):
         # Top-K: g R, m RW | ebar R (Delta is not stored: the server pass recomputes it from m)
         worker = 12 * Wd + 4 * d if topk else 12 * Wd + 8 * d
         variant = "topk" if topk else "sign_p1"
+    elif w.momentum == 0.0:
+        step = 12 * Wd + 16 * d              # g R, e RW | x RW, e_srv RW  (mu = 0: no momentum rows)
+        worker = 12 * Wd                     # g R, Delta(e) RW
+        variant = "mu0"
     else:
         step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW
         worker = 20 * Wd                     # g R, m RW, Delta(e) RW

@@ -65,7 +65,10 @@ typedef struct {
   int32_t mode;                /* SAE_MODE_*                                                            */
   int32_t avg_period;          /* p >= 1: worker errors are averaged in the pre-step of every iteration
                                   t with (t+1) mod p = 0 (Algorithm 1, Section 3.2); 0 = never (p = inf) */
-  float momentum;              /* mu in [0,1)                                                           */
+  float momentum;              /* mu in [0,1).  mu = 0 (the SGD / SignSGD variants) with avg_period != 1:
+                                  m^(k) equals the step's gradient term and is not kept -- no momentum
+                                  rows are allocated, read or written, SAE_STATE_MOMENTUM is refused, and
+                                  a -0 gradient term counts as +0 (fma(0, m, -0) would keep the sign of m) */
   float weight_decay;          /* lambda >= 0: coupled L2, lambda * (point where the gradient is
                                   evaluated) is added to the gradient                                    */
   uint32_t topk_num, topk_den; /* Top-K keeps k_j = max(1, floor(n_j*num/den)) entries per tensor; all

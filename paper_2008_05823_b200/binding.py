@@ -121,6 +121,7 @@ class Sae:
         self.K = int(num_workers)
         self.T = len(self.sizes)
         self.compressor = compressor
+        self.keeps_momentum = not (momentum == 0.0 and avg_period != 1)     # mu = 0: m^(k) is not state
         self.stream = torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream
         cfg = SaeConfig(ABI_VERSION, self.K, self.T, self.sizes.ctypes.data_as(C.POINTER(C.c_int64)), compressor,
                         server_compress, mode, avg_period, momentum, weight_decay, topk_num, topk_den,

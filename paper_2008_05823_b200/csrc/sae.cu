@@ -71,6 +71,7 @@ struct sae_handle {
   int last_cuda_error;
   int persistent_blocks;  // #SMs x blocks per SM of the persistent worker pass
   int num_sms;
+  int mu0;                 // momentum 0 and p != 1: no momentum rows (m^(k) is the step's gradient term, not state)
   int topk_nod;            // Top-K with p = 1: model differences never stored, two uniform-error buffers
   float* ebar_alt;
   int64_t launches;
@@ -214,11 +215,11 @@ CandArgs cand_args(sae_handle* h, bool server) {
 
 constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
 
-template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK>
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK, bool MU0 = false>
 void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
   static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
   if (configured_device != h->device) {
-    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK, MU0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                          (int)kWorkerSmem);
     configured_device = h->device;
   }
@@ -229,11 +230,19 @@ void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa)
   if (h->P.K <= grid) grid -= grid % h->P.K;
   if (nitems < grid) grid = nitems;
   LaunchScope ls(h, S_WORKER);
-  k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
+  k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK, MU0><<<(unsigned)grid, WT_THREADS, kWorkerSmem, h->stream>>>(h->P, sp, wa, nitems);
 }
 
 template <int ESRC, bool SIGN, bool WRITE_D, bool TOPK = false>
 void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
+  if constexpr (WRITE_D) {
+    if (h->mu0) {          // no momentum rows (only steps that store the model differences run in this mode)
+      if (sp.wd) launch_worker_wd<ESRC, SIGN, true, true, TOPK, true>(h, sp, wa);
+      else launch_worker_wd<ESRC, SIGN, true, false, TOPK, true>(h, sp, wa);
+      return;
+    }
+  }
+  if (h->mu0) return;      // unreachable: the callers below keep WRITE_D set when there is no momentum buffer
   if (sp.wd) launch_worker_wd<ESRC, SIGN, WRITE_D, true, TOPK>(h, sp, wa);
   else launch_worker_wd<ESRC, SIGN, WRITE_D, false, TOPK>(h, sp, wa);
 }
@@ -336,7 +345,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // The model differences need not be stored when the previous error was uniform and the next
     // pre-step averages: the averaging pass recomputes them from m and ebar with the same fused op.
     const bool pending_in = h->esrc == ESRC_PENDING_AVG;
-    const bool write_d = !((h->esrc == ESRC_UNIFORM || pending_in) && avg_after);
+    const bool write_d = h->mu0 || !((h->esrc == ESRC_UNIFORM || pending_in) && avg_after);
     if (write_d && !h->D) return SAE_ERR_INVALID_ARG;
     // p = 1: the average is not formed here but at the head of the next worker pass
     const bool defer_avg = avg_after && !write_d && h->fused_ok;
@@ -501,7 +510,8 @@ std::vector<CkptSection> ckpt_sections(sae_handle* h) {
   const bool sign = h->cfg.compressor == SAE_COMPRESSOR_SIGN, topk = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
   std::vector<CkptSection> v;
   v.push_back({h->x, (size_t)P.dpad * f}); v.push_back({h->e_srv, (size_t)P.dpad * f});
-  v.push_back({h->ebar, (size_t)P.dpad * f}); v.push_back({h->m, (size_t)P.K * P.dpad * f});
+  v.push_back({h->ebar, (size_t)P.dpad * f});
+  if (h->m) v.push_back({h->m, (size_t)P.K * P.dpad * f});
   if (h->D) v.push_back({h->D, (size_t)P.K * P.dpad * f});
   if (h->ebar_alt) v.push_back({h->ebar_alt, (size_t)P.dpad * f});
   if (sign) { v.push_back({h->words, (size_t)P.K * P.nwords * 4}); v.push_back({h->words_srv, (size_t)P.nwords * 4}); }
@@ -587,6 +597,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   }
   const bool sign = cfg->compressor == SAE_COMPRESSOR_SIGN, topk = cfg->compressor == SAE_COMPRESSOR_TOPK;
   h->topk_nod = (topk && cfg->avg_period == 1) ? 1 : 0;
+  h->mu0 = (cfg->momentum == 0.0f && cfg->avg_period != 1) ? 1 : 0;
   const bool need_D = shard || !((sign || topk) && cfg->avg_period == 1);
   const long long nwords = dpad / 32;
   const size_t KT = (size_t)K * T;
@@ -602,7 +613,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->d_tile_tensor, (size_t)ntiles); ALLOC0(h->d_first_tile, T); ALLOC0(h->d_n, T);
   ALLOC0(h->d_off, T); ALLOC0(h->d_poff, T);
   ALLOC0(h->x, dpad); ALLOC0(h->e_srv, dpad); ALLOC0(h->ebar, dpad);
-  ALLOC0(h->m, (size_t)K * dpad);
+  if (!h->mu0) ALLOC0(h->m, (size_t)K * dpad);
   if (h->fused_ok) ALLOC0(h->etmp, dpad);
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
   if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
@@ -897,7 +908,9 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
   const size_t vec = sizeof(float) * (size_t)P.d, tb = sizeof(float) * (size_t)P.T, wb = sizeof(u32) * (size_t)P.nwords;
   const void* src = nullptr; size_t need = 0;
   switch (which) {
-    case SAE_STATE_MOMENTUM: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_M, worker, (float*)out);
+    case SAE_STATE_MOMENTUM:
+      if (bytes < vec || !h->m) return SAE_ERR_INVALID_ARG;       // (mu = 0: m^(k) is not kept)
+      return export_vec(h, EXP_M, worker, (float*)out);
     case SAE_STATE_WORKER_ERROR: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_WERR, worker, (float*)out);
     case SAE_STATE_SERVER_ERROR: if (bytes < vec) return SAE_ERR_INVALID_ARG; return export_vec(h, EXP_ESRV, 0, (float*)out);
     case SAE_STATE_WORKER_SCALES: if (!sign) return SAE_ERR_INVALID_ARG; src = h->scale[h->last] + (size_t)worker * P.T; need = tb; break;

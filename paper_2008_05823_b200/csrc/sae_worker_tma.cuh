@@ -117,7 +117,9 @@ __device__ __forceinline__ WtItem wt_lookup(const Plan& P, const WorkerArgs& A, 
   return it;
 }
 
-template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK>
+// MU0: momentum constant 0 (the SGD / SignSGD variants of Section 5): m^(k) is this step's gradient term and
+// is not state, so the momentum rows are neither read nor written (12 instead of 20 bytes per element).
+template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK, bool MU0 = false>
 __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma(Plan P, StepParams sp, WorkerArgs A,
                                                                                   long long nitems) {
   extern __shared__ unsigned char smem_raw[];
@@ -152,9 +154,9 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
             S.item[s] = cur;
             if (cur.vec) {
               constexpr u32 B = TILE * sizeof(float);
-              mbar_arrive_expect_tx(&S.full[s], 3 * B);
+              mbar_arrive_expect_tx(&S.full[s], (MU0 ? 2 : 3) * B);
               bulk_load(S.buf[s][0], A.g + cur.gofs, B, &S.full[s]);
-              bulk_load(S.buf[s][1], A.m + cur.wbase, B, &S.full[s]);
+              if (!MU0) bulk_load(S.buf[s][1], A.m + cur.wbase, B, &S.full[s]);
               bulk_load(S.buf[s][2], (ESRC == ESRC_UNIFORM) ? (A.ebar + cur.pbase) : (A.D + cur.wbase), B,
                         &S.full[s]);
             } else {
@@ -210,7 +212,8 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
       for (int q = 0; q < WT_SLICE_ITERS; ++q) {
         const int e0 = base + q * 128 + lane * 4;
         const float4 G = *reinterpret_cast<const float4*>(sg + e0);
-        const float4 M = *reinterpret_cast<const float4*>(sm + e0);
+        float4 M = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!MU0) M = *reinterpret_cast<const float4*>(sm + e0);
         const float4 E = *reinterpret_cast<const float4*>(se + e0);
         float4 X = make_float4(0.f, 0.f, 0.f, 0.f);
         if (WD) X = ld4(xp + e0);
@@ -219,7 +222,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
         dl.y = worker_update<WD>(G.y, M.y, prev_error<ESRC>(E.y, it.sprev, it.tprev), X.y, sp, mn.y);
         dl.z = worker_update<WD>(G.z, M.z, prev_error<ESRC>(E.z, it.sprev, it.tprev), X.z, sp, mn.z);
         dl.w = worker_update<WD>(G.w, M.w, prev_error<ESRC>(E.w, it.sprev, it.tprev), X.w, sp, mn.w);
-        st4(mp + e0, mn);
+        if (!MU0) st4(mp + e0, mn);
         if (WRITE_D) st4(dp + e0, dl);
         if (TOPK && it.lo != NO_GUESS) {
           if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand, stg_k, stg_j);
@@ -249,8 +252,8 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
           const float e = prev_error<ESRC>((ESRC == ESRC_UNIFORM) ? ebp[e0] : dp[e0], it.sprev, it.tprev);
           const float xv = WD ? xp[e0] : 0.0f;
           float mn;
-          dl = worker_update<WD>(__ldcs(gp + e0), mp[e0], e, xv, sp, mn);
-          mp[e0] = mn;
+          dl = worker_update<WD>(__ldcs(gp + e0), MU0 ? 0.0f : mp[e0], e, xv, sp, mn);
+          if (!MU0) mp[e0] = mn;
           if (WRITE_D) dp[e0] = dl;
           if (SIGN) lane_add(acc, dl);
         }

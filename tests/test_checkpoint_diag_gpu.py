@@ -12,14 +12,15 @@ pytestmark = pytest.mark.gpu
 SIZES = [33, 4096, 5000, 700, 3 * 4096]
 
 
+@pytest.mark.parametrize("mu", [0.9, 0.0])
 @pytest.mark.parametrize("comp,p,K", [(so.SIGN, 1, 4), (so.SIGN, 3, 3), (so.TOPK, 2, 4), (so.TOPK, 1, 3), (so.SIGN, 0, 2)])
-def test_resume_continues_bit_for_bit(comp, p, K):
+def test_resume_continues_bit_for_bit(comp, p, K, mu):
     """Save after 5 steps, restore into a fresh handle (different x0), continue: same bits as the oracle."""
     import torch
     d = sum(SIZES)
     scales = synth.tensor_scales(7, len(SIZES), -4.0, -1.0)
     x0 = synth.x0_numpy(7, d)
-    kw = dict(compressor=comp, avg_period=p, momentum=0.9, weight_decay=1e-4, topk_num=1, topk_den=20)
+    kw = dict(compressor=comp, avg_period=p, momentum=mu, weight_decay=1e-4, topk_num=1, topk_den=20)
     orc = so.Oracle(K, SIZES, x0, threads=4, **kw)
     a = sb.Sae(K, SIZES, torch.from_numpy(x0).cuda(), **kw)
     lrs = [0.1, 0.1, 0.05, 0.1, 0.2, 0.1, 0.05, 0.1, 0.1]

@@ -336,3 +336,27 @@ def test_blockwise_sign(block, p):
     sizes = configs.blockwise_sizes([3 * 4096 + 17, 4096, 5, 20000, 8192], block)
     assert sum(sizes) == 3 * 4096 + 17 + 4096 + 5 + 20000 + 8192
     run_pair(4, sizes, so.SIGN, 6, p=p, lrs=[0.1, 0.05])
+
+
+@pytest.mark.parametrize("comp", [so.SIGN, so.TOPK, so.IDENTITY])
+@pytest.mark.parametrize("p,lam,mode", [(0, 0.0, so.SAEF), (3, 1e-4, so.SAEF), (2, 1e-4, so.EF), (1, 0.0, so.SAEF)])
+def test_momentum_constant_zero(comp, p, lam, mode):
+    """mu = 0 (the SGD / SignSGD variants of Section 5).  For p != 1 the library keeps no momentum rows at all
+    (m^(k) is the step's gradient term); p = 1 goes through the regular paths.  Same bits either way."""
+    run_pair(3, RAGGED, comp, 7, p=p, mu=0.0, lam=lam, mode=mode, num=1, den=20, outliers=(66, 100.0), seed=4,
+             lrs=[0.1, 0.05])
+
+
+def test_momentum_getter_is_refused_without_momentum_rows():
+    import torch
+    x0 = torch.zeros(sum(RAGGED), device="cuda")
+    a = sb.Sae(2, RAGGED, x0, momentum=0.0, avg_period=0)
+    assert not a.keeps_momentum
+    with pytest.raises(sb.SaeError):
+        a.get_state(sb.STATE_MOMENTUM, 0)
+    a.get_state(sb.STATE_WORKER_ERROR, 0)
+    a.close()
+    b = sb.Sae(2, RAGGED, x0, momentum=0.0, avg_period=1)       # p = 1 keeps them (the folded averaging reads them)
+    assert b.keeps_momentum
+    b.get_state(sb.STATE_MOMENTUM, 0)
+    b.close()
