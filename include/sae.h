@@ -210,6 +210,13 @@ int64_t sae_kernel_launches(const sae_handle *h);
  *   sae_step_begin    worker lines of iteration t for the local workers: grads_local is [num_local][d].
  *   sae_step_end      server lines, re-update and the pre-step of iteration t+1.
  *
+ * Errors: SAE_ERR_INVALID_ARG for a null pointer, a compressor other than scaled sign, a worker range outside
+ * 0..K-1, a blob that is too short / foreign / describes another parameter list / names rows that are already
+ * attached, sae_step_begin before every worker's rows are attached or while a step is open, sae_step_end
+ * without an open step, sae_shard_attach / sae_shard_detach / checkpoint calls while a step is open;
+ * SAE_ERR_CUDA when mapping a peer's buffer fails (sae_last_cuda_error has the code).  Device-detected
+ * errors (RANGE, TIMEOUT) are sticky and reported by sae_sync, as for sae_step.
+ *
  * Ordering is the caller's duty (a host barrier after synchronising the streams, or a collective that is
  * stream-ordered on every shard): every shard's sae_step_begin work must be complete before any shard's
  * sae_step_end work starts (the messages are read remotely), and every shard's sae_step_end work before
