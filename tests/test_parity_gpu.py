@@ -360,3 +360,48 @@ def test_momentum_getter_is_refused_without_momentum_rows():
     assert b.keeps_momentum
     b.get_state(sb.STATE_MOMENTUM, 0)
     b.close()
+
+
+def test_maximum_worker_count():
+    """K = 1024, the largest the library accepts (and 1025 is refused)."""
+    import torch
+    run_pair(1024, [33, 700], so.SIGN, 3, p=2, seed=5)
+    run_pair(1024, [33, 700], so.TOPK, 2, p=0, num=1, den=10, seed=5)
+    with pytest.raises(sb.SaeError):
+        sb.Sae(1025, [33], torch.zeros(33, device="cuda"))
+
+
+def test_maximum_tensor_size():
+    """One tensor of 2^30 elements (the largest allowed: 262 144 tiles, the limit of the L1 record's headroom),
+    one worker, single-way compression.  Too large for the CPU oracle to hold comfortably, so the step is
+    checked against what Eq. 2 and Algorithm 1 fix for it: with K = 1, zero initial state and no server
+    compression, Delta = lr * g, scale = mean |Delta| (within one fp32 rounding of the exactly rounded mean),
+    bit i = (Delta_i >= 0), x_1 = x_0 - (+-scale), e^(1) = Delta - (+-scale)."""
+    import torch
+    n = 1 << 30
+    gen = torch.Generator(device="cuda").manual_seed(7)
+    g = torch.empty(1, n, device="cuda").normal_(0.0, 1e-2, generator=gen)
+    x0 = torch.zeros(n, device="cuda")
+    with pytest.raises(sb.SaeError):
+        sb.Sae(1, [n + 1], torch.zeros(n + 1, device="cuda"))          # above the limit
+    a = sb.Sae(1, [n], x0, compressor=sb.SIGN, server_compress=0, avg_period=0, momentum=0.9)
+    a.step(g, 0.5)
+    a.sync()
+    delta = g[0] * 0.5                                                 # fma(0.5, m, 0) with m = fma(0.9, 0, g) = g: exact
+    scale = a.get_state(sb.STATE_WORKER_SCALES, 0)
+    exact = float(delta.double().abs().sum().item()) / n               # fp64 sum of 2^30 terms: ~1e-13 relative
+    got = float(scale[0].item())
+    assert abs(got - exact) <= 2.0 ** -23 * exact, (got, exact)
+    words = a.get_state(sb.STATE_WORKER_WORDS, 0)
+    pos = delta >= 0
+    weights = (2 ** torch.arange(32, device="cuda", dtype=torch.int64))
+    exp_words = (pos.view(-1, 32).to(torch.int64) * weights).sum(dim=1)
+    assert torch.equal(words.to(torch.int64) & 0xFFFFFFFF, exp_words)
+    del exp_words, weights
+    code = torch.where(pos, scale[0], -scale[0])
+    x1 = a.get_params()
+    assert torch.equal(x1, x0 - code)
+    del x1
+    e1 = a.get_state(sb.STATE_WORKER_ERROR, 0)
+    assert torch.equal(e1, delta - code)
+    a.close()
