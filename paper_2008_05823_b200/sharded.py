@@ -25,9 +25,11 @@ class ShardedRun:
     """One rank of a sharded run.
 
     make_engine(worker_begin, num_local) -> object with shard_export() -> bytes, shard_attach(bytes),
-    step_begin(grads_local, lr), step_end(), close() and optionally shard_detach().  `barrier()` must
-    return only when every rank has reached it AND the device work each rank enqueued before it is complete
-    (default: synchronise the CUDA device, then torch.distributed.barrier)."""
+    step_begin(grads_local, lr), step_end(), close() and optionally shard_detach().  `barrier()` must order
+    the device work every rank enqueued before it ahead of the device work any rank enqueues after it.
+    Defaults: with the NCCL backend a one-element all-reduce on the current CUDA stream (stream-ordered on
+    every rank: its kernel starts after the rank's earlier work and ends only when every rank's has started;
+    the host does not wait); otherwise synchronise the device, then torch.distributed.barrier."""
 
     def __init__(self, num_workers: int, make_engine: Callable, group=None, barrier: Optional[Callable] = None):
         import torch.distributed as dist
@@ -38,6 +40,11 @@ class ShardedRun:
         self.num_workers = num_workers
         self.begin, self.count = worker_range(num_workers, self.world, self.rank)
         self.engine = make_engine(self.begin, self.count)
+        self._flag = None
+        if barrier is None and dist.get_backend(group) == "nccl":
+            import torch
+            self._flag = torch.zeros(1, device="cuda")
+            barrier = self._stream_barrier
         self._barrier = barrier if barrier is not None else self._default_barrier
         blobs: List[Optional[bytes]] = [None] * self.world
         dist.all_gather_object(blobs, self.engine.shard_export(), group=group)
@@ -45,6 +52,9 @@ class ShardedRun:
             self.engine.shard_attach(b)
         self._readers_pending = False         # peers may still be reading this rank's rows
         self._barrier()
+
+    def _stream_barrier(self):
+        self.dist.all_reduce(self._flag, group=self.group)
 
     def _default_barrier(self):
         import torch
@@ -64,7 +74,9 @@ class ShardedRun:
         self._readers_pending = True
 
     def finish(self):
-        """Waits until no peer reads this rank's rows any more (call before reading results)."""
+        """Orders everything after it behind every peer's reads of this rank's rows (call before reading
+        results or reusing buffers; with the stream-ordered barrier the host still has to synchronise the
+        stream before it looks at device memory)."""
         if self._readers_pending:
             self._barrier()
             self._readers_pending = False
@@ -73,8 +85,11 @@ class ShardedRun:
         """Orderly shutdown: every rank unmaps its peers' rows before any rank frees its own."""
         self.finish()
         if hasattr(self.engine, "shard_detach"):
-            self.engine.shard_detach()
+            self.engine.shard_detach()           # waits for this rank's stream, then unmaps
         self._barrier()
+        if self._flag is not None:
+            import torch
+            torch.cuda.synchronize()             # the stream-ordered barrier has actually completed
         self.engine.close()
 
 

@@ -161,3 +161,44 @@ def test_config2_fullsize_shards_equal_the_single_handle():
                     assert torch.equal(a.view(torch.int32), r.view(torch.int32)), f"p={p} state {which} worker {b + kl}"
             s.close()
         one.close()
+
+
+NCCL_WORKER = r"""
+import os, sys
+import numpy as np, torch, torch.distributed as dist
+sys.path.insert(0, {root!r}); sys.path.insert(0, os.path.join({root!r}, "tests"))
+from oracle import sae_oracle as so
+from paper_2008_05823_b200 import synth
+from paper_2008_05823_b200.sharded import sharded_sae
+os.environ.setdefault("MASTER_ADDR", "127.0.0.1"); os.environ.setdefault("MASTER_PORT", "29761")
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+sizes = [33, 4096, 5000]
+K, d = 3, sum(sizes)
+scales = synth.tensor_scales(1, len(sizes), -4.0, -1.0)
+x0 = synth.x0_numpy(1, d)
+orc = so.Oracle(K, sizes, x0, compressor=so.SIGN, avg_period=2, momentum=0.9)
+run = sharded_sae(K, sizes, torch.from_numpy(x0).cuda(), avg_period=2, momentum=0.9)
+assert run._flag is not None                      # the stream-ordered barrier is in use
+for t in range(4):
+    g = synth.grads_numpy(1, t, K, sizes, scales)
+    orc.step(g, 0.1)
+    run.step(torch.from_numpy(g).cuda(), 0.1)
+run.finish()
+torch.cuda.synchronize()
+assert np.array_equal(run.engine.get_params().cpu().numpy().view(np.uint32), orc.get(orc.X).view(np.uint32))
+run.close()
+dist.destroy_process_group()
+print("NCCL_OK")
+"""
+
+
+def test_stream_ordered_barrier_with_the_nccl_backend(tmp_path):
+    """World size 1 (this box has one GPU): the NCCL code path of the rank logic -- all-gather of the row
+    descriptions, the one-element all-reduce as the stream-ordered barrier, orderly shutdown."""
+    script = tmp_path / "nccl_worker.py"
+    script.write_text(NCCL_WORKER.format(root=ROOT))
+    res = subprocess.run([sys.executable, str(script)], cwd=ROOT, capture_output=True, text=True, timeout=600,
+                         env=dict(os.environ, OMP_NUM_THREADS="2"))
+    assert res.returncode == 0, (res.stdout[-1000:], res.stderr[-3000:])
+    assert "NCCL_OK" in res.stdout
