@@ -210,6 +210,15 @@ int64_t sae_kernel_launches(const sae_handle *h);
  *   sae_step_begin    worker lines of iteration t for the local workers: grads_local is [num_local][d].
  *   sae_step_end      server lines, re-update and the pre-step of iteration t+1.
  *
+ * Error averaging by all-reduce (the communication the paper names for it, Section 3.2: "ring all-reduce").
+ * sae_shard_set_avg_mode(h, 1) replaces the in-place pull of all K x d stored differences by a sum the
+ * caller all-reduces: when sae_avg_due(h) is 1 after sae_step_end, call sae_avg_local_sum(h, buf) (buf:
+ * device, sae_num_padded(h) floats; receives sum_k e^(k) over this shard's workers, k in order, in the
+ * library's padded layout), all-reduce buf over the shards with SUM, then sae_avg_set(h, buf) on every
+ * shard (ebar = buf / K).  This moves 2 d floats per shard instead of K d, but the order of the all-reduce's
+ * additions is the library's, not k = 0..K-1: the averaged error then agrees with Algorithm 1 to fp32
+ * rounding, not bit for bit (with one shard it is exact).  sae_step_begin is refused while the sum is owed.
+ *
  * Errors: SAE_ERR_INVALID_ARG for a null pointer, a compressor other than scaled sign, a worker range outside
  * 0..K-1, a blob that is too short / foreign / describes another parameter list / names rows that are already
  * attached, sae_step_begin before every worker's rows are attached or while a step is open, sae_step_end
@@ -231,6 +240,11 @@ int sae_shard_attach(sae_handle *h, const void *blob_host, size_t bytes);
 int sae_shard_detach(sae_handle *h);
 int sae_step_begin(sae_handle *h, const float *grads_local, float lr);
 int sae_step_end(sae_handle *h);
+int sae_shard_set_avg_mode(sae_handle *h, int32_t external_sum);
+int sae_avg_due(const sae_handle *h);
+int64_t sae_num_padded(const sae_handle *h);
+int sae_avg_local_sum(sae_handle *h, float *sum_padded);
+int sae_avg_set(sae_handle *h, const float *sum_padded);
 
 /* Frees everything the handle owns (synchronises first). NULL is allowed. */
 void sae_destroy(sae_handle *h);

@@ -25,7 +25,8 @@ EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_p
            "sae_get_kernel_times", "sae_kernel_name", "sae_kernel_launches", "sae_destroy", "sae_strerror",
            "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements", "sae_state_bytes",
            "sae_save_state", "sae_load_state", "sae_get_mismatch", "sae_init_shard", "sae_shard_export",
-           "sae_shard_attach", "sae_shard_detach", "sae_step_begin", "sae_step_end"]
+           "sae_shard_attach", "sae_shard_detach", "sae_step_begin", "sae_step_end", "sae_shard_set_avg_mode", "sae_avg_due",
+           "sae_num_padded", "sae_avg_local_sum", "sae_avg_set"]
 
 SHARD_BLOB_BYTES = 512
 
@@ -89,6 +90,12 @@ def lib():
         L.sae_shard_detach.argtypes = [vp]
         L.sae_step_begin.argtypes = [vp, vp, f32]
         L.sae_step_end.argtypes = [vp]
+        L.sae_shard_set_avg_mode.argtypes = [vp, i32]
+        L.sae_avg_due.argtypes = [vp]
+        L.sae_num_padded.argtypes = [vp]
+        L.sae_num_padded.restype = i64
+        L.sae_avg_local_sum.argtypes = [vp, vp]
+        L.sae_avg_set.argtypes = [vp, vp]
         L.sae_sign_compress_noalloc.argtypes = [vp, i64, vp, vp, vp, vp]
         L.sae_noalloc_max_elements.argtypes = []
         L.sae_noalloc_max_elements.restype = i64
@@ -182,6 +189,23 @@ class Sae:
 
     def step_end(self):
         _check(lib().sae_step_end(self.h), "sae_step_end", self.h)
+
+    def shard_set_avg_mode(self, external_sum):
+        _check(lib().sae_shard_set_avg_mode(self.h, 1 if external_sum else 0), "sae_shard_set_avg_mode", self.h)
+
+    @property
+    def avg_due(self):
+        return bool(lib().sae_avg_due(self.h))
+
+    def avg_local_sum(self, buf=None):
+        """sum_k e^(k) over this shard's workers into buf (padded layout, sae_num_padded floats)."""
+        if buf is None:
+            buf = self._vec(n=int(lib().sae_num_padded(self.h)))
+        _check(lib().sae_avg_local_sum(self.h, buf.data_ptr()), "sae_avg_local_sum", self.h)
+        return buf
+
+    def avg_set(self, buf):
+        _check(lib().sae_avg_set(self.h, buf.data_ptr()), "sae_avg_set", self.h)
 
     def step_host(self, grads_host, lr):
         t = self.torch

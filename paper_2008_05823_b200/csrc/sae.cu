@@ -80,6 +80,8 @@ struct sae_handle {
   Plan P_all;                       // the plan with K = K_total (server pass, averaging)
   int attached;                     // workers whose message rows are known
   int mid_step;                     // sae_step_begin done, sae_step_end due
+  int avg_external;                 // the averaging sum is all-reduced by the caller instead of pulled in k order
+  int avg_owed;                     // ... and is owed before the next sae_step_begin
   float lr_pending;
   std::vector<const u32*> h_word_rows;
   std::vector<const float*> h_scale_rows[2], h_d_rows;
@@ -743,8 +745,10 @@ int shard_end(sae_handle* h) {
   else LAUNCH(h, S_SERVER, (k_server_sign<false, true>), nblk, PA, sa, tpb);
   if (dc) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), PA.ntiles, PA, aa);
   else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), PA.ntiles, PA, aa);
-  if (avg_after) LAUNCH(h, S_APPLY, k_avg_pull, PA.ntiles, PA, h->d_d_rows, h->d_scale_rows[cur], h->ebar);
-  h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
+  if (avg_after && !h->avg_external)
+    LAUNCH(h, S_APPLY, k_avg_pull<false>, PA.ntiles, PA, h->d_d_rows, h->d_scale_rows[cur], h->ebar);
+  if (avg_after && h->avg_external) h->avg_owed = 1;     // the error stays "lazy" until sae_avg_set
+  h->esrc = (avg_after && !h->avg_external) ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
   h->last = cur; h->eta_prev = h->lr_pending; h->t += 1; h->mid_step = 0;
   return check_launch(h);
 }
@@ -835,9 +839,38 @@ int sae_shard_detach(sae_handle* h) {
   return SAE_OK;
 }
 
+int sae_shard_set_avg_mode(sae_handle* h, int32_t external_sum) {
+  if (!h || !h->shard || h->mid_step || h->avg_owed) return SAE_ERR_INVALID_ARG;
+  h->avg_external = external_sum ? 1 : 0;
+  return SAE_OK;
+}
+
+int sae_avg_due(const sae_handle* h) { return (h && h->avg_owed) ? 1 : 0; }
+int64_t sae_num_padded(const sae_handle* h) { return h ? h->P.dpad : -1; }
+
+int sae_avg_local_sum(sae_handle* h, float* sum_padded) {
+  if (!h || !sum_padded || !h->shard || !h->avg_owed || h->mid_step) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  // this shard's own rows, k in order: the table entries k0 .. k0+K-1 with the local plan (K = local workers)
+  LAUNCH(h, S_APPLY, k_avg_pull<true>, h->P.ntiles, h->P, h->d_d_rows + h->k0, h->d_scale_rows[h->last] + h->k0,
+         sum_padded);
+  return check_launch(h);
+}
+
+int sae_avg_set(sae_handle* h, const float* sum_padded) {
+  if (!h || !sum_padded || !h->shard || !h->avg_owed || h->mid_step) return SAE_ERR_INVALID_ARG;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return SAE_ERR_CUDA;
+  LAUNCH(h, S_APPLY, k_avg_set, h->P_all.ntiles, h->P_all, sum_padded, h->ebar);
+  h->esrc = ESRC_UNIFORM;
+  h->avg_owed = 0;
+  return check_launch(h);
+}
+
 int sae_step_begin(sae_handle* h, const float* grads_local, float lr) {
   if (!h || !grads_local || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
-  if (!h->shard || h->mid_step || h->attached != h->K_total) return SAE_ERR_INVALID_ARG;
+  if (!h->shard || h->mid_step || h->avg_owed || h->attached != h->K_total) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   return shard_begin(h, grads_local, lr);
@@ -941,7 +974,7 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
 int64_t sae_state_bytes(sae_handle* h) { return h ? (int64_t)ckpt_bytes(h) : -1; }
 
 int sae_save_state(sae_handle* h, void* out, size_t bytes) {
-  if (!h || !out || bytes < ckpt_bytes(h) || h->mid_step) return SAE_ERR_INVALID_ARG;
+  if (!h || !out || bytes < ckpt_bytes(h) || h->mid_step || h->avg_owed) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   CkptHeader hd;

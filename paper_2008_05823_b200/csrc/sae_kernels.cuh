@@ -345,6 +345,8 @@ __global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const
 // Sharded operation, error averaging (Algorithm 1, pre-step): ebar = (1/K) sum_k e^(k) in k order, with
 // e^(k) = D^(k) - C(D^(k)) formed from every owner's stored model differences and scales, read in place
 // through row tables (the same subtraction, order and division as the unsharded averaging in k_apply).
+// SUM_ONLY (rows = this shard's own workers): the undivided partial sum, for an all-reduce across shards.
+template <bool SUM_ONLY>
 __global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const* __restrict__ d_rows,
                                                        const float* const* __restrict__ scale_rows, float* ebar) {
   __shared__ float s_k[MAX_WORKERS];
@@ -367,18 +369,26 @@ __global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const
         b2 = __fadd_rn(b2, prev_error<ESRC_LAZY_SIGN>(v.z, s, 0u));
         b3 = __fadd_rn(b3, prev_error<ESRC_LAZY_SIGN>(v.w, s, 0u));
       }
-      st4(ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
+      if (SUM_ONLY) st4(ebar + pbase + i, make_float4(b0, b1, b2, b3));
+      else st4(ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
     }
   } else {
     for (int i = tid; i < ti.cnt; i += THREADS) {
       float b = 0.f;
       for (int k = 0; k < P.K; ++k) b = __fadd_rn(b, prev_error<ESRC_LAZY_SIGN>(s_row[k][pbase + i], s_k[k], 0u));
-      ebar[pbase + i] = div_by_k(P, b);
+      ebar[pbase + i] = SUM_ONLY ? b : div_by_k(P, b);
     }
   }
 }
 
 // ---------------------------------------------------------------------------------------------------
+// ebar = sum / K over the padded layout (the all-reduced sum of the shards' partial sums)
+__global__ void __launch_bounds__(THREADS) k_avg_set(Plan P, const float* __restrict__ sum, float* __restrict__ ebar) {
+  const TileInfo ti = tile_info(P, blockIdx.x);
+  const long long pbase = ti.poff + ti.t0;
+  for (int i = threadIdx.x; i < ti.cnt; i += THREADS) ebar[pbase + i] = div_by_k(P, sum[pbase + i]);
+}
+
 struct ApplyArgs {
   float* e_srv;            // [dpad] in: Delta_{t+1}, out: e_{t+1}
   float* x;                // [dpad]

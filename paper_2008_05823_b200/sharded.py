@@ -31,7 +31,8 @@ class ShardedRun:
     every rank: its kernel starts after the rank's earlier work and ends only when every rank's has started;
     the host does not wait); otherwise synchronise the device, then torch.distributed.barrier."""
 
-    def __init__(self, num_workers: int, make_engine: Callable, group=None, barrier: Optional[Callable] = None):
+    def __init__(self, num_workers: int, make_engine: Callable, group=None, barrier: Optional[Callable] = None,
+                 allreduce_average: bool = False):
         import torch.distributed as dist
         self.dist = dist
         self.group = group
@@ -51,6 +52,10 @@ class ShardedRun:
         for b in blobs:                       # rank order; includes this rank's own rows
             self.engine.shard_attach(b)
         self._readers_pending = False         # peers may still be reading this rank's rows
+        self.allreduce_average = allreduce_average
+        self._sum = None
+        if allreduce_average:
+            self.engine.shard_set_avg_mode(True)
         self._barrier()
 
     def _stream_barrier(self):
@@ -72,6 +77,12 @@ class ShardedRun:
         self._barrier()                       # every rank's messages are complete
         self.engine.step_end()
         self._readers_pending = True
+        if self.allreduce_average and self.engine.avg_due:
+            # Section 3.2: the local errors are averaged with an all-reduce (2 d floats per rank instead of
+            # reading all K d stored differences in place; the sum order is the collective's)
+            self._sum = self.engine.avg_local_sum(self._sum)
+            self.dist.all_reduce(self._sum, group=self.group)
+            self.engine.avg_set(self._sum)
 
     def finish(self):
         """Orders everything after it behind every peer's reads of this rank's rows (call before reading
@@ -93,11 +104,11 @@ class ShardedRun:
         self.engine.close()
 
 
-def sharded_sae(num_workers, tensor_sizes, x0, group=None, barrier=None, **kw) -> ShardedRun:
+def sharded_sae(num_workers, tensor_sizes, x0, group=None, barrier=None, allreduce_average=False, **kw) -> ShardedRun:
     """ShardedRun over the CUDA library: every rank passes the same num_workers, tensor_sizes, x0 and options."""
     from . import binding as sb
 
     def make(begin, count):
         return sb.Sae(num_workers, tensor_sizes, x0, compressor=sb.SIGN, shard=(begin, count), **kw)
 
-    return ShardedRun(num_workers, make, group=group, barrier=barrier)
+    return ShardedRun(num_workers, make, group=group, barrier=barrier, allreduce_average=allreduce_average)

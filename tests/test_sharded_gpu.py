@@ -202,3 +202,58 @@ def test_stream_ordered_barrier_with_the_nccl_backend(tmp_path):
                          env=dict(os.environ, OMP_NUM_THREADS="2"))
     assert res.returncode == 0, (res.stdout[-1000:], res.stderr[-3000:])
     assert "NCCL_OK" in res.stdout
+
+
+@pytest.mark.parametrize("world", [1, 2, 3])
+def test_error_averaging_by_allreduce(world):
+    """The all-reduce form of the error averaging (Section 3.2).  One shard: the sum is the shard's own ordered
+    sum, so everything stays bit-exact.  Several shards: the partial sums are added in another order than
+    k = 0..K-1, so the averaged error matches the oracle to fp32 rounding (and everything that does not yet
+    depend on it, bit for bit)."""
+    import torch
+    K, p = 5, 3
+    d = int(np.sum(SIZES))
+    scales = synth.tensor_scales(2, len(SIZES), -4.0, -1.0)
+    x0 = synth.x0_numpy(2, d)
+    kw = dict(compressor=so.SIGN, avg_period=p, momentum=0.9, weight_decay=1e-4)
+    orc = so.Oracle(K, SIZES, x0, threads=4, **kw)
+    ranges = [worker_range(K, world, r) for r in range(world)]
+    shards = [sb.Sae(K, SIZES, torch.from_numpy(x0).cuda(), shard=rg, **kw) for rg in ranges]
+    for s in shards:
+        for blob in [q.shard_export() for q in shards]:
+            s.shard_attach(blob)
+        s.shard_set_avg_mode(True)
+    steps = 6 if world == 1 else 2            # the first averaging is owed after step 2 ((t + 2) mod 3 = 0 at t = 1)
+    for t in range(steps):
+        g = synth.grads_numpy(2, t, K, SIZES, scales)
+        orc.step(g, 0.1)
+        gd = torch.from_numpy(g).cuda().view(K, d)
+        for s, (b, c) in zip(shards, ranges):
+            s.step_begin(gd[b:b + c].contiguous(), 0.1)
+        for s in shards:
+            s.step_end()
+        due = [s.avg_due for s in shards]
+        assert all(due) == any(due) and due[0] == ((t + 2) % p == 0)
+        if due[0]:
+            with pytest.raises(sb.SaeError):
+                shards[0].step_begin(gd[:ranges[0][1]].contiguous(), 0.1)      # refused while the sum is owed
+            total = None
+            for s in shards:                                                    # the "all-reduce", in rank order
+                part = s.avg_local_sum()
+                total = part if total is None else total + part
+            for s in shards:
+                s.avg_set(total)
+        for s, (b, c) in zip(shards, ranges):
+            s.sync()
+            got_x = s.get_params().cpu().numpy()
+            got_e = s.get_state(sb.STATE_WORKER_ERROR, 0).cpu().numpy()
+            if world == 1:
+                assert_same(f"t={t + 1} x", got_x, orc.get(orc.X))
+                assert_same(f"t={t + 1} e", got_e, orc.get(orc.E, b))
+            else:
+                assert_same(f"t={t + 1} x", got_x, orc.get(orc.X))             # does not depend on the average yet
+                # a mean of K terms of mixed sign: a few roundings of the largest term, absolute
+                exp_e = orc.get(orc.E, b)
+                np.testing.assert_allclose(got_e, exp_e, rtol=2e-6, atol=2.0 ** -22 * float(np.abs(exp_e).max()))
+    for s in shards:
+        s.close()
