@@ -256,7 +256,6 @@ void launch_apply(sae_handle* h, int avg, const ApplyArgs& aa) {
   else LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_RECOMPUTE>), h->P.ntiles, h->P, aa);
 }
 
-constexpr size_t kFusedSmem = sizeof(FwSmem) + 128;
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time dependency on libcuda).
 PFN_cuTensorMapEncodeTiled tensor_map_encoder() {
@@ -271,13 +270,13 @@ PFN_cuTensorMapEncodeTiled tensor_map_encoder() {
   return fn;
 }
 
-// Row-major fp32 matrix [rows][inner] with the given row pitch, fetched in boxes of 256 x rows.
+// Row-major fp32 matrix [rows][inner] with the given row pitch, fetched in boxes of fw_box(rows) x rows.
 bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows, long long pitch_elems) {
   PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
   if (!enc || (reinterpret_cast<uintptr_t>(base) & 15) || ((pitch_elems * 4) & 15)) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 4};
-  cuuint32_t box[2] = {(cuuint32_t)FW_BOX, (cuuint32_t)rows};
+  cuuint32_t box[2] = {(cuuint32_t)fw_box(rows), (cuuint32_t)rows};
   cuuint32_t estr[2] = {1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -286,6 +285,8 @@ bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows
 
 template <int K, bool WD>
 void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, const CUtensorMap& tm_g) {
+  constexpr size_t kFusedSmem = sizeof(FwSmemT<K>) + 128;
+  static_assert(kFusedSmem <= 227 * 1024, "the ring must fit the shared memory of one block");
   static thread_local int configured_device = -1;
   if (configured_device != h->device) {
     cudaFuncSetAttribute(k_worker_fused<K, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);

@@ -11,10 +11,10 @@
 // The two are done by different warps: four "averager" warps run one tile ahead of sixteen "worker"
 // warps and hand each tile over through an mbarrier, so the averaging overlaps the worker lines.
 // One block handles a tile for ALL workers: the producer warp brings the tile of all K momentum rows in
-// with 2-D tensor-map TMA copies (one request per box of 256 elements x K rows -- per-row copies of
+// with 2-D tensor-map TMA copies (one request per box of up to 256 elements x K rows -- per-row copies of
 // 1-2 KB each were limited by the per-request cost), likewise the K gradient rows when the caller's
 // layout allows a tensor map (16-byte aligned base and row pitch), and the ebar tile with a 1-D bulk
-// copy; 3-stage ring, full/empty mbarriers.  The consumers touch global memory only to store.
+// copy; 3- or 6-stage ring (by K), full/empty mbarriers.  The consumers touch global memory only to store.
 // In phase B a consumer warp always works for the same worker(s), so it carries their L1 partials
 // across tiles and adds them to the (worker, tensor) records only when the tensor changes.
 // All waits are bounded (STATUS_TIMEOUT).
@@ -27,29 +27,35 @@ namespace sae {
 constexpr int FW_WARPS = 16;                       // worker warps (warps 0..15)
 constexpr int FW_AVG_WARPS = 4;                    // averager warps (warps 17..20); warp 16 is the producer
 constexpr int FW_THREADS = (FW_WARPS + 1 + FW_AVG_WARPS) * 32;
-#ifndef SAE_FW_STAGES
-#define SAE_FW_STAGES 3
-#endif
-constexpr int FW_STAGES = SAE_FW_STAGES;
 constexpr int FW_MAXTILE = 2048;
-constexpr int FW_BOX = 256;                        // inner extent of a TMA box (the hardware limit)
-#ifndef SAE_FW_MBUF
-#define SAE_FW_MBUF 8192
+constexpr int FW_MAXBOX = 256;                     // inner extent of a TMA box (the hardware limit)
+// From this many workers on, an item is half as large and the ring twice as deep (6 stages of 2 x 16 KB
+// instead of 3 of 2 x 32 KB): with few, large stages the copies in flight -- (stages - 1) x stage size --
+// do not cover the memory latency at full bandwidth.
+#ifndef SAE_FW_SPLIT_K
+#define SAE_FW_SPLIT_K 16
 #endif
-constexpr int FW_MBUF = SAE_FW_MBUF;                      // floats of momentum (and of gradient) per stage (32 KB each)
+constexpr bool fw_split(int K) { return K >= SAE_FW_SPLIT_K && K <= 16; }     // (K = 32 would need 512-byte box rows: slower)
+constexpr int fw_mbuf(int K) { return fw_split(K) ? 4096 : 8192; }   // floats of momentum (and gradient) per stage
+constexpr int fw_stages(int K) { return fw_split(K) ? 6 : 3; }
+constexpr int fw_tilef(int K) { return (fw_mbuf(K) / K) < FW_MAXTILE ? (fw_mbuf(K) / K) : FW_MAXTILE; }
+constexpr int fw_box(int K) { return fw_tilef(K) < FW_MAXBOX ? fw_tilef(K) : FW_MAXBOX; }
 
 template <int K>
 struct FwGeom {
-  static constexpr int TILEF = (FW_MBUF / K) < FW_MAXTILE ? (FW_MBUF / K) : FW_MAXTILE;   // elements per item
+  static constexpr int MBUF = fw_mbuf(K);
+  static constexpr int STAGES = fw_stages(K);
+  static constexpr int TILEF = fw_tilef(K);                   // elements per item
+  static constexpr int BOX = fw_box(K);                       // inner extent of the TMA boxes
   static constexpr int SUB = TILE / TILEF;                    // items per 4096-element plan tile
   static constexpr int ROWS_PER_WORKER = TILEF / 128;
   static constexpr int RPW = K * ROWS_PER_WORKER / FW_WARPS;  // 128-element rows per warp and item
   static constexpr int WPW = RPW > ROWS_PER_WORKER ? RPW / ROWS_PER_WORKER : 1;   // workers per warp
   static_assert(K >= 1 && K <= 32 && (K & (K - 1)) == 0, "power-of-two worker counts up to 32");
-  static constexpr int CHUNKS = TILEF / FW_BOX;               // TMA boxes per array and item
-  static_assert(RPW >= 1 && WPW <= 2 && CHUNKS >= 1, "geometry");
-  // position of element e of worker k inside a stage buffer: boxes of [K][256] one after the other
-  __device__ static __forceinline__ int idx(int k, int e) { return (e >> 8) * (K * FW_BOX) + k * FW_BOX + (e & 255); }
+  static constexpr int CHUNKS = TILEF / BOX;                  // TMA boxes per array and item
+  static_assert(RPW >= 1 && WPW <= 2 && CHUNKS >= 1 && BOX % 128 == 0, "geometry");
+  // position of element e of worker k inside a stage buffer: boxes of [K][BOX] one after the other
+  __device__ static __forceinline__ int idx(int k, int e) { return (e / BOX) * (K * BOX) + k * BOX + (e % BOX); }
 };
 
 // 2-D tiled TMA load of one box at element coordinates (x, y), completing on `bar`.
@@ -67,15 +73,17 @@ struct FwItem {
   int j, cnt, gvec;  // tensor, valid elements (0 = empty item), gradient tile fetched by TMA into the stage
 };
 
-struct FwSmem {
-  alignas(128) float m[FW_STAGES][FW_MBUF];
-  alignas(128) float g[FW_STAGES][FW_MBUF];
-  alignas(128) float e[FW_STAGES][FW_MAXTILE];
-  alignas(8) u64 full[FW_STAGES];
-  alignas(8) u64 empty[FW_STAGES];
-  alignas(8) u64 avgd[FW_STAGES];   // "ebar' of this stage is ready": one arrival per averager warp
-  FwItem item[FW_STAGES];
-  float sc[FW_STAGES][32];      // last step's scales of the item's tensor, one per worker
+template <int K>
+struct FwSmemT {
+  typedef FwGeom<K> G;
+  alignas(128) float m[G::STAGES][G::MBUF];
+  alignas(128) float g[G::STAGES][G::MBUF];
+  alignas(128) float e[G::STAGES][G::TILEF];
+  alignas(8) u64 full[G::STAGES];
+  alignas(8) u64 empty[G::STAGES];
+  alignas(8) u64 avgd[G::STAGES];   // "ebar' of this stage is ready": one arrival per averager warp
+  FwItem item[G::STAGES];
+  float sc[G::STAGES][32];      // last step's scales of the item's tensor, one per worker
 };
 
 struct FusedArgs {
@@ -116,7 +124,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
                                                                  const __grid_constant__ CUtensorMap tm_g) {
   typedef FwGeom<K> G;
   extern __shared__ unsigned char smem_raw[];
-  FwSmem& S = *reinterpret_cast<FwSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+  typedef FwSmemT<K> Smem;
+  constexpr int FW_STAGES = G::STAGES;
+  constexpr int FW_BOX = G::BOX;
+  Smem& S = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int s = 0; s < FW_STAGES; ++s) {
@@ -180,7 +191,8 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   if (warp > FW_WARPS) {
     // ---------------- averagers: ebar' = (1/K) sum_k ( fma(eta_prev, m_k, ebar) - C(.) ), k in order ----------------
     constexpr int NA = FW_AVG_WARPS * 32;
-    constexpr int EPT = G::TILEF / NA;               // elements per thread: 2, 4, 8 or 16
+    constexpr int EPT = G::TILEF / NA;               // elements per thread: 1, 2, 4, 8 or 16
+    static_assert(EPT >= 1, "an item has at least one element per averager thread");
     constexpr int V = EPT < 4 ? EPT : 4;             // handled in chunks of V consecutive elements
     constexpr int CH = EPT / V;
     const int ta = tid - (FW_WARPS + 1) * 32;

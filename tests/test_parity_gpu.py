@@ -405,3 +405,11 @@ def test_maximum_tensor_size():
     e1 = a.get_state(sb.STATE_WORKER_ERROR, 0)
     assert torch.equal(e1, delta - code)
     a.close()
+
+
+@pytest.mark.parametrize("K", [8, 16, 32])
+@pytest.mark.parametrize("lam", [0.0, 1e-4])
+def test_folded_averaging_pass_ring_geometries(K, lam):
+    """p = 1 with 8, 16 and 32 workers: the worker pass with the averaging folded in, in both of its ring
+    geometries (3 deep stages up to 8 workers, 6 shallow ones from 16 on), on ragged and on whole tiles."""
+    run_pair(K, [33, 4096, 5000, 700, 3 * 4096, 130], so.SIGN, 5, p=1, lam=lam, seed=6, lrs=[0.1, 0.05])
