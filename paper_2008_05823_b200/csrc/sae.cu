@@ -270,13 +270,13 @@ PFN_cuTensorMapEncodeTiled tensor_map_encoder() {
   return fn;
 }
 
-// Row-major fp32 matrix [rows][inner] with the given row pitch, fetched in boxes of fw_box(rows) x rows.
+// Row-major fp32 matrix [rows][inner] with the given row pitch, fetched in boxes of fw_box(rows) x fw_kh(rows).
 bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows, long long pitch_elems) {
   PFN_cuTensorMapEncodeTiled enc = tensor_map_encoder();
   if (!enc || (reinterpret_cast<uintptr_t>(base) & 15) || ((pitch_elems * 4) & 15)) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 4};
-  cuuint32_t box[2] = {(cuuint32_t)fw_box(rows), (cuuint32_t)rows};
+  cuuint32_t box[2] = {(cuuint32_t)fw_box(rows), (cuuint32_t)fw_kh(rows)};
   cuuint32_t estr[2] = {1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -35,27 +35,38 @@ constexpr int FW_MAXBOX = 256;                     // inner extent of a TMA box 
 #ifndef SAE_FW_SPLIT_K
 #define SAE_FW_SPLIT_K 16
 #endif
-constexpr bool fw_split(int K) { return K >= SAE_FW_SPLIT_K && K <= 16; }     // (K = 32 would need 512-byte box rows: slower)
+// K = 32: a stage of all 32 rows x 256 elements is 2 x 32 KB, so only three fit; the element range is
+// instead handled as two consecutive items of 16 workers each (boxes of 16 rows), which makes the stages
+// half as large without shortening the 1 KB box rows (512-byte rows were slower).
+#ifndef SAE_FW_HALVES32
+#define SAE_FW_HALVES32 2
+#endif
+constexpr int fw_halves(int K) { return K == 32 ? SAE_FW_HALVES32 : 1; }
+constexpr int fw_kh(int K) { return K / fw_halves(K); }                         // workers (box rows) per item
+constexpr bool fw_split(int K) { return (K >= SAE_FW_SPLIT_K && K <= 16) || fw_halves(K) > 1; }
 constexpr int fw_mbuf(int K) { return fw_split(K) ? 4096 : 8192; }   // floats of momentum (and gradient) per stage
 constexpr int fw_stages(int K) { return fw_split(K) ? 6 : 3; }
-constexpr int fw_tilef(int K) { return (fw_mbuf(K) / K) < FW_MAXTILE ? (fw_mbuf(K) / K) : FW_MAXTILE; }
+constexpr int fw_tilef(int K) { return (fw_mbuf(K) / fw_kh(K)) < FW_MAXTILE ? (fw_mbuf(K) / fw_kh(K)) : FW_MAXTILE; }
 constexpr int fw_box(int K) { return fw_tilef(K) < FW_MAXBOX ? fw_tilef(K) : FW_MAXBOX; }
 
 template <int K>
 struct FwGeom {
+  static constexpr int HALVES = fw_halves(K);                 // items per element range
+  static constexpr int KH = fw_kh(K);                         // workers per item
   static constexpr int MBUF = fw_mbuf(K);
   static constexpr int STAGES = fw_stages(K);
   static constexpr int TILEF = fw_tilef(K);                   // elements per item
   static constexpr int BOX = fw_box(K);                       // inner extent of the TMA boxes
-  static constexpr int SUB = TILE / TILEF;                    // items per 4096-element plan tile
+  static constexpr int SUB = TILE / TILEF;                    // element ranges per 4096-element plan tile
   static constexpr int ROWS_PER_WORKER = TILEF / 128;
-  static constexpr int RPW = K * ROWS_PER_WORKER / FW_WARPS;  // 128-element rows per warp and item
-  static constexpr int WPW = RPW > ROWS_PER_WORKER ? RPW / ROWS_PER_WORKER : 1;   // workers per warp
+  static constexpr int RPW = KH * ROWS_PER_WORKER / FW_WARPS; // 128-element rows per warp and item
+  static constexpr int WPW = RPW > ROWS_PER_WORKER ? RPW / ROWS_PER_WORKER : 1;   // workers per warp and item
+  static constexpr int NACC = WPW * HALVES;                   // workers a warp ever works for
   static_assert(K >= 1 && K <= 32 && (K & (K - 1)) == 0, "power-of-two worker counts up to 32");
   static constexpr int CHUNKS = TILEF / BOX;                  // TMA boxes per array and item
-  static_assert(RPW >= 1 && WPW <= 2 && CHUNKS >= 1 && BOX % 128 == 0, "geometry");
-  // position of element e of worker k inside a stage buffer: boxes of [K][BOX] one after the other
-  __device__ static __forceinline__ int idx(int k, int e) { return (e / BOX) * (K * BOX) + k * BOX + (e % BOX); }
+  static_assert(RPW >= 1 && NACC <= 2 && CHUNKS >= 1 && BOX % 128 == 0 && STAGES % HALVES == 0, "geometry");
+  // position of element e of the item's worker kl inside a stage buffer: boxes of [KH][BOX] one after the other
+  __device__ static __forceinline__ int idx(int kl, int e) { return (e / BOX) * (KH * BOX) + kl * BOX + (e % BOX); }
 };
 
 // 2-D tiled TMA load of one box at element coordinates (x, y), completing on `bar`.
@@ -71,6 +82,7 @@ struct FwItem {
   long long pbase;   // first element in the [dpad] arrays
   long long goff;    // first element inside a gradient row (caller layout)
   int j, cnt, gvec;  // tensor, valid elements (0 = empty item), gradient tile fetched by TMA into the stage
+  int h;             // which group of KH workers
 };
 
 template <int K>
@@ -103,7 +115,7 @@ template <int K>
 __device__ __forceinline__ FwItem fw_lookup(const Plan& P, int g_tma_ok, long long w, long long nitems) {
   typedef FwGeom<K> G;
   FwItem it;
-  it.pbase = 0; it.goff = 0; it.j = 0; it.cnt = 0; it.gvec = 0;
+  it.pbase = 0; it.goff = 0; it.j = 0; it.cnt = 0; it.gvec = 0; it.h = 0;
   if (w >= nitems) { it.cnt = -1; return it; }
   const int tile = (int)(w / G::SUB);
   const int sub = (int)(w - (long long)tile * G::SUB);
@@ -139,47 +151,49 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 
   if (warp == FW_WARPS) {
     // ---------------- producer ----------------
+    // nitems counts element ranges; each is issued as HALVES consecutive items (one per group of KH workers)
     const long long GR = gridDim.x;
     long long wb = blockIdx.x;
     FwItem nxt = fw_lookup<K>(P, A.g_tma_ok, wb + lane * GR, nitems);
-    for (int i0 = 0; wb < nitems; i0 += 32, wb += 32 * GR) {
+    for (int p0 = 0; wb < nitems; p0 += 32, wb += 32 * GR) {
       const FwItem cur = nxt;
       nxt = fw_lookup<K>(P, A.g_tma_ok, wb + (32 + lane) * GR, nitems);
       for (int l = 0; l < 32; ++l) {
-        // the item of lane l, broadcast so that the lanes can share the issue of its copies
+        // the range of lane l, broadcast so that the lanes can share the issue of its copies
         const int cnt = __shfl_sync(0xffffffffu, cur.cnt, l);
-        if (cnt < 0) break;                                   // past the last item (uniform)
+        if (cnt < 0) break;                                   // past the last range (uniform)
         const long long pbase = __shfl_sync(0xffffffffu, cur.pbase, l);
         const int j = __shfl_sync(0xffffffffu, cur.j, l);
-        float scale_k = 0.0f;
-        if (cnt > 0 && lane < K) scale_k = __ldg(A.scale_prev + (long long)lane * P.T + j);
-        const int i = i0 + l;
-        const int s = i % FW_STAGES;
-        int ok = 1;
-        if (lane == 0) {
-          if (i >= FW_STAGES && !mbar_wait(&S.empty[s], ((i / FW_STAGES) - 1) & 1)) {
-            atomicOr(A.status, STATUS_TIMEOUT);
-            ok = 0;
-          }
-        }
-        if (!__shfl_sync(0xffffffffu, ok, 0)) return;
-        if (lane == l) S.item[s] = cur;
-        if (lane < K) S.sc[s][lane] = scale_k;
-        __syncwarp();
-        if (cnt == 0) {
-          if (lane == 0) mbar_arrive(&S.full[s]);
-        } else {
-          const u32 ebytes = (u32)((cnt + 31) & ~31) * 4u;    // rows are padded to 32 elements
-          const int gtma = __shfl_sync(0xffffffffu, cur.gvec, l);
-          const long long goff = __shfl_sync(0xffffffffu, cur.goff, l);
+        const int gtma = __shfl_sync(0xffffffffu, cur.gvec, l);
+        const long long goff = __shfl_sync(0xffffffffu, cur.goff, l);
+#pragma unroll
+        for (int hh = 0; hh < G::HALVES; ++hh) {
+          float scale_k = 0.0f;
+          if (cnt > 0 && lane < G::KH) scale_k = __ldg(A.scale_prev + (long long)(hh * G::KH + lane) * P.T + j);
+          const int i = (p0 + l) * G::HALVES + hh;
+          const int s = i % FW_STAGES;
+          int ok = 1;
           if (lane == 0) {
+            if (i >= FW_STAGES && !mbar_wait(&S.empty[s], ((i / FW_STAGES) - 1) & 1)) {
+              atomicOr(A.status, STATUS_TIMEOUT);
+              ok = 0;
+            }
+          }
+          if (!__shfl_sync(0xffffffffu, ok, 0)) return;
+          if (lane == l) { FwItem t = cur; t.h = hh; S.item[s] = t; }
+          if (lane < G::KH) S.sc[s][lane] = scale_k;
+          __syncwarp();
+          if (cnt == 0) {
+            if (lane == 0) mbar_arrive(&S.full[s]);
+          } else if (lane == 0) {
+            const u32 ebytes = (hh == 0) ? (u32)((cnt + 31) & ~31) * 4u : 0u;    // rows are padded to 32 elements
             const int chunks = (cnt + FW_BOX - 1) / FW_BOX;
-            constexpr u32 BOXB = (u32)(K * FW_BOX * 4);
+            constexpr u32 BOXB = (u32)(G::KH * FW_BOX * 4);
             mbar_arrive_expect_tx(&S.full[s], ebytes + (u32)chunks * BOXB * (gtma ? 2u : 1u));
-            bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);
+            if (hh == 0) bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);  // the old ebar travels with the first group
             for (int c = 0; c < chunks; ++c) {
-              tma_load_2d(&S.m[s][c * K * FW_BOX], &tm_m, (int)pbase + c * FW_BOX, 0, &S.full[s]);
-              if (gtma) tma_load_2d(&S.g[s][c * K * FW_BOX], &tm_g, (int)goff + c * FW_BOX, 0, &S.full[s]);
+              tma_load_2d(&S.m[s][c * G::KH * FW_BOX], &tm_m, (int)pbase + c * FW_BOX, hh * G::KH, &S.full[s]);
+              if (gtma) tma_load_2d(&S.g[s][c * G::KH * FW_BOX], &tm_g, (int)goff + c * FW_BOX, hh * G::KH, &S.full[s]);
             }
           }
         }
@@ -190,14 +204,23 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 
   if (warp > FW_WARPS) {
     // ---------------- averagers: ebar' = (1/K) sum_k ( fma(eta_prev, m_k, ebar) - C(.) ), k in order ----------------
+    // With two groups of workers per range the partial sums are carried from the first item to the second
+    // (k = 0..KH-1, then KH..K-1: still one sequential sum), and ebar' is written into both stages.
     constexpr int NA = FW_AVG_WARPS * 32;
     constexpr int EPT = G::TILEF / NA;               // elements per thread: 1, 2, 4, 8 or 16
     static_assert(EPT >= 1, "an item has at least one element per averager thread");
     constexpr int V = EPT < 4 ? EPT : 4;             // handled in chunks of V consecutive elements
     constexpr int CH = EPT / V;
     const int ta = tid - (FW_WARPS + 1) * 32;
-    long long w = blockIdx.x;
-    for (int i = 0; w < nitems; ++i, w += gridDim.x) {
+    float eb[CH][V], a[CH][V];
+#pragma unroll
+    for (int c = 0; c < CH; ++c)
+#pragma unroll
+      for (int v = 0; v < V; ++v) { eb[c][v] = 0.0f; a[c][v] = 0.0f; }
+    for (int i = 0;; ++i) {
+      const long long w = blockIdx.x + (long long)(i / G::HALVES) * gridDim.x;
+      if (w >= nitems) break;
+      const int hh = i % G::HALVES;
       const int s = i % FW_STAGES;
       if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
         if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
@@ -206,50 +229,60 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       const FwItem it = S.item[s];
       if (it.cnt > 0) {
         const float* sm = S.m[s];
-        float* se = S.e[s];
+        const float* se0 = S.e[(i - hh) % FW_STAGES];       // the first group's stage holds the old ebar
         const float* sc = S.sc[s];
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           const int e0 = c * (NA * V) + ta * V;
           if (e0 < it.cnt) {
-            float eb[V], a[V];
+            if (hh == 0) {
 #pragma unroll
-            for (int v = 0; v < V; ++v) { eb[v] = se[e0 + v]; a[v] = 0.0f; }
+              for (int v = 0; v < V; ++v) { eb[c][v] = se0[e0 + v]; a[c][v] = 0.0f; }
+            }
 #pragma unroll
-            for (int k = 0; k < K; ++k) {
+            for (int k = 0; k < G::KH; ++k) {
               const float sk = sc[k];
 #pragma unroll
               for (int v = 0; v < V; ++v) {
-                const float dk = __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[v]);
-                a[v] = __fadd_rn(a[v], __fsub_rn(dk, sign_code(dk, sk)));
+                const float dk = __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[c][v]);
+                a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, sign_code(dk, sk)));
               }
             }
+            if (hh == G::HALVES - 1) {
 #pragma unroll
-            for (int v = 0; v < V; ++v) {
-              if (e0 + v < it.cnt) {
-                const float en = div_by_k(P, a[v]);
-                se[e0 + v] = en;
-                A.ebar[it.pbase + e0 + v] = en;
+              for (int v = 0; v < V; ++v) {
+                if (e0 + v < it.cnt) {
+                  const float en = div_by_k(P, a[c][v]);
+#pragma unroll
+                  for (int hq = 0; hq < G::HALVES; ++hq) S.e[(i - hh + hq) % FW_STAGES][e0 + v] = en;
+                  A.ebar[it.pbase + e0 + v] = en;
+                }
               }
             }
           }
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&S.avgd[s]);
+      if (hh == G::HALVES - 1 && lane == 0) {
+#pragma unroll
+        for (int hq = 0; hq < G::HALVES; ++hq) mbar_arrive(&S.avgd[(i - hh + hq) % FW_STAGES]);
+      }
     }
     return;
   }
 
   // ---------------- workers ----------------
-  LaneAcc acc[G::WPW];
+  // accumulator a belongs to worker (a / WPW) * KH + kl0 + (a % WPW)
+  LaneAcc acc[G::NACC];
 #pragma unroll
-  for (int a = 0; a < G::WPW; ++a) lane_acc_init(acc[a]);
+  for (int a = 0; a < G::NACC; ++a) lane_acc_init(acc[a]);
   int acc_j = -1;
   const int row0 = warp * G::RPW;                       // first row of this warp inside an item
-  const int k0 = row0 / G::ROWS_PER_WORKER;             // its (first) worker
-  long long w = blockIdx.x;
-  for (int i = 0; w < nitems; ++i, w += gridDim.x) {
+  const int kl0 = row0 / G::ROWS_PER_WORKER;            // its (first) worker inside the item's group
+  for (int i = 0;; ++i) {
+    const long long w = blockIdx.x + (long long)(i / G::HALVES) * gridDim.x;
+    if (w >= nitems) break;
+    const int hh = i % G::HALVES;
     const int s = i % FW_STAGES;
     if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
       if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
@@ -260,8 +293,9 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       if (it.j != acc_j) {
         if (acc_j >= 0) {
 #pragma unroll
-          for (int a = 0; a < G::WPW; ++a) {
-            warp_commit(acc[a], A.recs + (long long)(k0 + a) * P.T + acc_j, A.status);
+          for (int a = 0; a < G::NACC; ++a) {
+            const int kk = (a / G::WPW) * G::KH + kl0 + (a % G::WPW);
+            warp_commit(acc[a], A.recs + (long long)kk * P.T + acc_j, A.status);
             lane_acc_init(acc[a]);
           }
         }
@@ -270,7 +304,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       const float* sm = S.m[s];
       const float* sg = S.g[s];
       const float* se = S.e[s];
-      // ebar' of this tile comes from the averager warps
+      // ebar' of this range comes from the averager warps
       if (!mbar_wait(&S.avgd[s], (i / FW_STAGES) & 1)) {
         if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
         return;
@@ -279,11 +313,12 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 #pragma unroll
       for (int q = 0; q < G::RPW; ++q) {
         const int r = row0 + q;
-        const int k = r / G::ROWS_PER_WORKER, rr = r % G::ROWS_PER_WORKER;
-        const int a = (G::WPW == 1) ? 0 : (k - k0);
+        const int kl = r / G::ROWS_PER_WORKER, rr = r % G::ROWS_PER_WORKER;
+        const int k = hh * G::KH + kl;
+        const int a = hh * G::WPW + ((G::WPW == 1) ? 0 : (kl - kl0));
         float* mp = A.m + (long long)k * P.dpad + it.pbase;
         u32* wp = A.words + (long long)k * P.nwords + (it.pbase >> 5);
-        const int rbase = G::idx(k, rr * 128);                 // the row's position in the stage buffers
+        const int rbase = G::idx(kl, rr * 128);                // the row's position in the stage buffers
         if (it.gvec && rr * 128 + 128 <= it.cnt) {
           const int e0 = rr * 128 + lane * 4;
           const float4 Gq = *reinterpret_cast<const float4*>(sg + rbase + lane * 4);
@@ -297,9 +332,8 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           dl.z = worker_update<WD>(Gq.z, M.z, E.z, X.z, sp, mn.z);
           dl.w = worker_update<WD>(Gq.w, M.w, E.w, X.w, sp, mn.w);
           st4(mp + e0, mn);
-          if (G::WPW == 1) lane_add4(acc[0], dl);
-          else if (a == 0) lane_add4(acc[0], dl);
-          else lane_add4(acc[G::WPW - 1], dl);
+          if (G::NACC == 1 || a == 0) lane_add4(acc[0], dl);
+          else lane_add4(acc[G::NACC - 1], dl);
           const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
           if ((lane & 7) == 0) wp[e0 >> 5] = wd;
         } else if (rr * 128 < it.cnt) {
@@ -316,9 +350,8 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
               float mn;
               dl = worker_update<WD>(gv, sm[rbase + c * 32 + lane], se[e], xv, sp, mn);
               mp[e] = mn;
-              if (G::WPW == 1) lane_add(acc[0], dl);
-              else if (a == 0) lane_add(acc[0], dl);
-              else lane_add(acc[G::WPW - 1], dl);
+              if (G::NACC == 1 || a == 0) lane_add(acc[0], dl);
+              else lane_add(acc[G::NACC - 1], dl);
             }
             const u32 wd = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
             if (lane == 0 && (rr * 128 + c * 32) < it.cnt) wp[(rr * 128 + c * 32) >> 5] = wd;
@@ -331,7 +364,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   }
   if (acc_j >= 0) {
 #pragma unroll
-    for (int a = 0; a < G::WPW; ++a) warp_commit(acc[a], A.recs + (long long)(k0 + a) * P.T + acc_j, A.status);
+    for (int a = 0; a < G::NACC; ++a) {
+      const int kk = (a / G::WPW) * G::KH + kl0 + (a % G::WPW);
+      warp_commit(acc[a], A.recs + (long long)kk * P.T + acc_j, A.status);
+    }
   }
 }
 
