@@ -316,7 +316,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", type=int, default=4, help="index into BASELINE.json configs (default: the largest)")
+    ap.add_argument("--workload", type=int, default=4, help="index of the benchmark configuration, 0..4 (default: the largest)")
     ap.add_argument("--avg-period", type=int, default=1,
                     help="error-averaging period p (1 = average inside every step; 0 = never)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
