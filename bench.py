@@ -290,7 +290,10 @@ def run_sharded(args, w, p, rank, local_rank, world):
     roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": None, "algorithmic_bytes_per_launch": worker_bytes,
                 "ms_per_launch": wk_ms, "peak_source": peak_source, "kernels": kernels,
-                "exchange_bytes_per_rank_per_step": (K - count) * (w.num_tensors * 4 + ((d + 31) // 32) * 4)}
+                # what a rank reads from its peers per step (1 bit per element + 1 scale per tensor and
+                # worker), against the ring all-reduce of fp32 model differences it replaces
+                "exchange_bytes_per_rank_per_step": (K - count) * (w.num_tensors * 4 + ((d + 31) // 32) * 4),
+                "fp32_ring_allreduce_bytes_per_rank_per_step": (2 * 4 * d * (world - 1)) // world}
     if world > 1:
         run.close()
     else:
