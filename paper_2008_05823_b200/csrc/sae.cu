@@ -48,6 +48,8 @@ struct sae_handle {
   float *scale[2], *scale_srv;
   u32 *tau[2], *tau_srv;
   L1Record *recs, *recs_srv;
+  L1Record* recs_srv_alt;  // second server-record buffer (inline_fin: the two alternate with the step parity)
+  int inline_fin;          // small problem: the server pass forms the worker scales itself (one launch fewer)
   u32 *hist;
   SelectState* sel;
   // Top-K candidate windows: key lists, per-tensor region offsets / capacities, cursors, fallback flags
@@ -163,7 +165,7 @@ cudaError_t dalloc(T** p, size_t count) {
 void free_all(sae_handle* h) {
   void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->ebar_alt, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
-                  h->tau_srv, h->recs, h->recs_srv, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
+                  h->tau_srv, h->recs, h->recs_srv, h->recs_srv_alt, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -335,12 +337,17 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   wa.cand = cand_args(h, false);
   ServerArgs sa;
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
-  sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status;
+  // inline_fin: step t accumulates the server's L1 into one buffer while the apply kernel clears the other
+  L1Record* const recs_srv_now = (h->inline_fin && cur) ? h->recs_srv_alt : h->recs_srv;
+  L1Record* const recs_srv_next = (h->inline_fin && !cur) ? h->recs_srv_alt : h->recs_srv;
+  sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = recs_srv_now; sa.status = h->status;
+  sa.word_rows = nullptr; sa.scale_rows = nullptr; sa.recs = h->recs; sa.scale_out = h->scale[cur];
   sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = ebar_now(h);
   sa.m = h->m; sa.ebar_in = ebar_now(h); sa.eta = lr;
   ApplyArgs aa;
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = ebar_now(h); aa.m = h->m; aa.D = h->D;
-  aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv; aa.tau_cur = h->tau[cur];
+  aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = recs_srv_now; aa.tau_cur = h->tau[cur];
+  aa.recs_clear = h->inline_fin ? h->recs : nullptr; aa.recs_srv_clear = recs_srv_next;
   aa.tau_srv = h->tau_srv;
   aa.mask_srv = h->mask_srv; aa.eta = lr;
 
@@ -363,12 +370,16 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
-    LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
-           h->scale[cur], h->recs_srv);
+    if (!h->inline_fin)
+      LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
+             h->scale[cur], h->recs_srv);
     // consecutive tiles per block: enough blocks to fill the device several times over, at most 8 tiles each
     const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
     const int nblk = (P.ntiles + tpb - 1) / tpb;
-    if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
+    if (h->inline_fin) {
+      if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true>), nblk, P, sa, tpb);
+      else LAUNCH(h, S_SERVER, (k_server_sign<false, false, true>), nblk, P, sa, tpb);
+    } else if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
     else LAUNCH(h, S_SERVER, k_server_sign<false>, nblk, P, sa, tpb);
     const int avg = (avg_after && !defer_avg) ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
     if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
@@ -626,6 +637,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->scale[0], KT); ALLOC0(h->scale[1], KT); ALLOC0(h->scale_srv, T);
   ALLOC0(h->tau[0], KT); ALLOC0(h->tau[1], KT); ALLOC0(h->tau_srv, T);
   ALLOC0(h->recs, sign ? KT : 0); ALLOC0(h->recs_srv, sign ? T : 0);
+  // latency-bound sizes (the whole K x d state fits L2 several times over): one launch fewer per step
+  h->inline_fin = (sign && !shard && (long long)K * dpad <= (1ll << 24)) ? 1 : 0;
+  if (h->inline_fin) ALLOC0(h->recs_srv_alt, T);
   ALLOC0(h->hist, topk ? KT * HIST_BINS : 0);
   ALLOC0(h->sel, topk ? KT : 0);
   std::vector<long long> cand_off(T, 0);
@@ -1015,6 +1029,11 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
     q += (s.bytes + 255) / 256 * 256;
   }
   h->t = hd.t; h->esrc = hd.esrc; h->last = hd.last; h->eta_prev = hd.eta_prev;
+  if (h->inline_fin) {       // the L1 records are transient, but nothing else clears them before the next step
+    SAE_CUDA(h, cudaMemsetAsync(h->recs, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
+    SAE_CUDA(h, cudaMemsetAsync(h->recs_srv, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
+    SAE_CUDA(h, cudaMemsetAsync(h->recs_srv_alt, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
+  }
   return SAE_OK;
 }
 

@@ -76,6 +76,9 @@ struct ServerArgs {
   // sharded operation: worker k's message lives with its owner (possibly another GPU's memory, read in place)
   const u32* const* word_rows;     // [K] -> worker k's [nwords] sign words
   const float* const* scale_rows;  // [K] -> worker k's [T] scales of this step
+  // small problems: the scales are formed here from the workers' exact L1 records (no separate launch)
+  const L1Record* recs;            // [K][T]
+  float* scale_out;                // [K][T] this step's scales, written by the block that holds a tensor's first tile
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -110,7 +113,9 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
   return r;
 }
 
-template <bool DC, bool TABLE = false>
+// FIN (small, latency-bound problems): the worker scales are not read but formed here from the exact L1
+// records, which saves the launch of k_finalize_scales; the records are then cleared by k_apply.
+template <bool DC, bool TABLE = false, bool FIN = false>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
   __shared__ const u32* s_row[TABLE ? MAX_WORKERS : 1];
@@ -128,8 +133,16 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
     if (ti.j != cur_j) {
       if (DC && cur_j >= 0) { warp_commit(acc, A.recs_srv + cur_j, A.status); lane_acc_init(acc); }
       __syncthreads();                            // the previous tensor's scales are no longer read
-      for (int k = tid; k < P.K; k += THREADS)
-        s_k[k] = TABLE ? A.scale_rows[k][ti.j] : A.scale_cur[(long long)k * P.T + ti.j];
+      for (int k = tid; k < P.K; k += THREADS) {
+        if (FIN) {
+          const L1Record r = A.recs[(long long)k * P.T + ti.j];
+          const float s = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
+          s_k[k] = s;
+          if (ti.t0 == 0) A.scale_out[(long long)k * P.T + ti.j] = s;
+        } else {
+          s_k[k] = TABLE ? A.scale_rows[k][ti.j] : A.scale_cur[(long long)k * P.T + ti.j];
+        }
+      }
       __syncthreads();
       cur_j = ti.j;
     }
@@ -401,6 +414,9 @@ struct ApplyArgs {
   const u32* tau_cur;      // [K][T]
   const u32* tau_srv;      // [T]
   u32* mask_srv;           // [nwords] Top-K: server selection of this step
+  // small problems (no k_finalize_scales launch): records to clear once the server pass has read them
+  L1Record* recs_clear;      // [K][T] the workers' records, or null
+  L1Record* recs_srv_clear;  // [T] the server records the NEXT step accumulates into (the other of two buffers)
   float eta;
 };
 
@@ -439,6 +455,13 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
       if (COMP == 2) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
     }
     __syncthreads();
+  }
+  if (A.recs_clear && ti.t0 == 0) {
+    for (int k = tid; k < P.K; k += THREADS) {
+      L1Record* r = A.recs_clear + (long long)k * P.T + ti.j;
+      r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0;
+    }
+    if (tid == 0) { L1Record* r = A.recs_srv_clear + ti.j; r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0; }
   }
   __shared__ float sh_s_srv;
   if (SRV == 1) {
