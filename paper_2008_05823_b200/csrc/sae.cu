@@ -26,8 +26,8 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after; const float* grads; float lr, eta_prev; };
-struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after; uint64_t stamp; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending; const float* grads; float lr, eta_prev; };
+struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after; uint64_t stamp; };
 
 }  // namespace
 
@@ -49,6 +49,9 @@ struct sae_handle {
   u32 *tau[2], *tau_srv;
   L1Record *recs, *recs_srv;
   L1Record* recs_srv_alt;  // second server-record buffer (inline_fin: the two alternate with the step parity)
+  int srv_pending;         // the last step's server lines (e = Delta - C(Delta), x -= C(Delta)) are still owed:
+                           // e_srv holds Delta, the server records hold its L1 sum; the next server pass
+                           // (or flush_server, before anything reads x or e) carries them out
   int inline_fin;          // small problem: the server pass forms the worker scales itself (one launch fewer)
   u32 *hist;
   SelectState* sel;
@@ -217,6 +220,18 @@ CandArgs cand_args(sae_handle* h, bool server) {
   return c;
 }
 
+// The server lines a step left pending, carried out now (getters, checkpoints, steps that need x or e).
+int flush_server(sae_handle* h) {
+  if (!h->srv_pending) return SAE_OK;
+  ApplyArgs aa;
+  memset(&aa, 0, sizeof(aa));
+  aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
+  if (h->cfg.server_compress) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), h->P.ntiles, h->P, aa);
+  else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), h->P.ntiles, h->P, aa);
+  h->srv_pending = 0;
+  return check_launch(h);
+}
+
 constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
 
 template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK, bool MU0 = false>
@@ -370,19 +385,36 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
+    // The server lines of this step can be left to the next step's server pass when nothing in between
+    // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
+#ifndef SAE_LAZY_SERVER
+#define SAE_LAZY_SERVER 1
+#endif
+    const bool lazy_ok = SAE_LAZY_SERVER && !h->inline_fin && !sp.wd;
+    if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
+    const bool pending = h->srv_pending != 0;
     if (!h->inline_fin)
       LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
-             h->scale[cur], h->recs_srv);
+             h->scale[cur], h->recs_srv, (pending && dc) ? h->scale_srv : nullptr);
+    sa.x = h->x; sa.scale_srv_prev = h->scale_srv;
     // consecutive tiles per block: enough blocks to fill the device several times over, at most 8 tiles each
     const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
     const int nblk = (P.ntiles + tpb - 1) / tpb;
     if (h->inline_fin) {
       if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true>), nblk, P, sa, tpb);
       else LAUNCH(h, S_SERVER, (k_server_sign<false, false, true>), nblk, P, sa, tpb);
+    } else if (pending) {
+      if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, true>), nblk, P, sa, tpb);
+      else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, true>), nblk, P, sa, tpb);
     } else if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
     else LAUNCH(h, S_SERVER, k_server_sign<false>, nblk, P, sa, tpb);
     const int avg = (avg_after && !defer_avg) ? (write_d ? AVG_FROM_D : AVG_RECOMPUTE) : AVG_NONE;
-    if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
+    if (lazy_ok && avg == AVG_NONE) {
+      h->srv_pending = 1;                       // this step's server lines wait for the next server pass
+    } else {
+      h->srv_pending = 0;
+      if (dc) launch_apply<1, 1>(h, avg, aa); else launch_apply<1, 0>(h, avg, aa);
+    }
     h->esrc = defer_avg ? ESRC_PENDING_AVG : (avg_after ? ESRC_UNIFORM : ESRC_LAZY_SIGN);
   } else if (c.compressor == SAE_COMPRESSOR_TOPK) {
     // p = 1 (previous error uniform, pre-step averages, every step): the model differences are not stored;
@@ -435,16 +467,16 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   if (!usable) return do_step_direct(h, grads, lr);
 
   StepGraphKey key;
-  key.esrc = h->esrc; key.last = h->last;
+  key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
-      h->esrc = e.esrc_after; h->last = e.last_after; h->eta_prev = lr; h->t += 1;
+      h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->eta_prev = lr; h->t += 1;
       e.stamp = ++h->graph_clock;
       h->graph_misses = 0;
       return SAE_OK;
@@ -465,7 +497,7 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   }
   StepGraph e;
   e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
-  e.esrc_after = h->esrc; e.last_after = h->last; e.stamp = ++h->graph_clock;
+  e.esrc_after = h->esrc; e.last_after = h->last; e.pending_after = h->srv_pending; e.stamp = ++h->graph_clock;
   ce = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
   if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); return SAE_ERR_CUDA; }
@@ -497,6 +529,7 @@ ExportArgs export_args(sae_handle* h, int what, int k, bool need_error) {
 }
 
 int export_vec(sae_handle* h, int what, int k, float* out) {
+  if (what != EXP_M) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }     // x and e must be up to date
   const ExportArgs ea = export_args(h, what, k, what == EXP_WERR || what == EXP_STEP_AHEAD);
   LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
   return check_launch(h);
@@ -735,7 +768,7 @@ int shard_begin(sae_handle* h, const float* grads, float lr) {
   if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
   else launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
   LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
-         h->scale[cur], h->recs_srv);
+         h->scale[cur], h->recs_srv, (float*)nullptr);
   h->mid_step = 1; h->lr_pending = lr;
   return check_launch(h);
 }
@@ -952,6 +985,7 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
   if (per_worker && (worker < 0 || worker >= P.K)) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
+  if (which == SAE_STATE_SERVER_SCALES) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
   const bool sign = h->cfg.compressor == SAE_COMPRESSOR_SIGN, topk = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
   const size_t vec = sizeof(float) * (size_t)P.d, tb = sizeof(float) * (size_t)P.T, wb = sizeof(u32) * (size_t)P.nwords;
   const void* src = nullptr; size_t need = 0;
@@ -992,6 +1026,7 @@ int sae_save_state(sae_handle* h, void* out, size_t bytes) {
   if (!h || !out || bytes < ckpt_bytes(h) || h->mid_step || h->avg_owed) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
+  { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
   CkptHeader hd;
   memset(&hd, 0, sizeof(hd));
   hd.magic = kCkptMagic; hd.K = h->P.K; hd.T = h->P.T; hd.compressor = h->cfg.compressor;
@@ -1029,6 +1064,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
     q += (s.bytes + 255) / 256 * 256;
   }
   h->t = hd.t; h->esrc = hd.esrc; h->last = hd.last; h->eta_prev = hd.eta_prev;
+  h->srv_pending = 0;        // a checkpoint is taken with the server lines carried out
   if (h->inline_fin) {       // the L1 records are transient, but nothing else clears them before the next step
     SAE_CUDA(h, cudaMemsetAsync(h->recs, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
     SAE_CUDA(h, cudaMemsetAsync(h->recs_srv, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
@@ -1041,6 +1077,7 @@ int sae_get_mismatch(sae_handle* h, double* out_host) {
   if (!h || !out_host || h->shard) return SAE_ERR_INVALID_ARG;     // needs every worker's error in one place
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
+  { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
   if (!h->mismatch) SAE_CUDA(h, dalloc(&h->mismatch, 2));
   SAE_CUDA(h, cudaMemsetAsync(h->mismatch, 0, 2 * sizeof(double), h->stream));
   const ExportArgs ea = export_args(h, EXP_WERR, 0, true);

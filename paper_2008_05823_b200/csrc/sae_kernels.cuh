@@ -79,6 +79,10 @@ struct ServerArgs {
   // small problems: the scales are formed here from the workers' exact L1 records (no separate launch)
   const L1Record* recs;            // [K][T]
   float* scale_out;                // [K][T] this step's scales, written by the block that holds a tensor's first tile
+  // deferred server update of the previous step (LAZY): e_srv still holds that step's Delta and x is not yet
+  // re-updated; both are brought up to date here, element by element, before this step's Delta is formed
+  float* x;                        // [dpad]
+  const float* scale_srv_prev;     // [T] server scales of the previous step (double-way)
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -115,9 +119,14 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
 
 // FIN (small, latency-bound problems): the worker scales are not read but formed here from the exact L1
 // records, which saves the launch of k_finalize_scales; the records are then cleared by k_apply.
-template <bool DC, bool TABLE = false, bool FIN = false>
+// LAZY: the previous step left its server lines pending (e = Delta - C(Delta), x = x - C(Delta): the work of
+// k_apply); they are carried out here on the fly -- the same two subtractions per parameter -- so that the
+// server error and the parameters make one trip through memory per step instead of two.  This pass has
+// the memory bandwidth to spare (it is bound by instruction issue).
+template <bool DC, bool TABLE = false, bool FIN = false, bool LAZY = false>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
+  __shared__ float sh_s_old;
   __shared__ const u32* s_row[TABLE ? MAX_WORKERS : 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (TABLE) {
@@ -143,11 +152,14 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
           s_k[k] = TABLE ? A.scale_rows[k][ti.j] : A.scale_cur[(long long)k * P.T + ti.j];
         }
       }
+      if (LAZY && DC && tid == 0) sh_s_old = A.scale_srv_prev[ti.j];
       __syncthreads();
       cur_j = ti.j;
     }
     const long long pbase = ti.poff + ti.t0;
     float* ep = A.e_srv + pbase;
+    float* xp = A.x + pbase;                       // (LAZY only)
+    const float s_old = (LAZY && DC) ? sh_s_old : 0.0f;
     const u32* __restrict__ wp = A.words + (pbase >> 5);
     u32* wsp = A.words_srv + (pbase >> 5);
 
@@ -204,6 +216,18 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         unpack2(a2[2 * q + 1], a3, a4);
         float4 e;
         if constexpr (DC) e = ld4(ep + i + 4 * q); else e = ev[q];
+        if constexpr (LAZY) {
+          // e holds the previous step's Delta: C(Delta) is its scaled sign (double-way) or Delta itself
+          float4 xv = ld4(xp + i + 4 * q);
+          float4 cs;
+          cs.x = DC ? sign_code(e.x, s_old) : e.x; cs.y = DC ? sign_code(e.y, s_old) : e.y;
+          cs.z = DC ? sign_code(e.z, s_old) : e.z; cs.w = DC ? sign_code(e.w, s_old) : e.w;
+          xv.x = __fsub_rn(xv.x, cs.x); xv.y = __fsub_rn(xv.y, cs.y);
+          xv.z = __fsub_rn(xv.z, cs.z); xv.w = __fsub_rn(xv.w, cs.w);
+          st4(xp + i + 4 * q, xv);
+          e.x = __fsub_rn(e.x, cs.x); e.y = __fsub_rn(e.y, cs.y);
+          e.z = __fsub_rn(e.z, cs.z); e.w = __fsub_rn(e.w, cs.w);
+        }
         float4 ds;
         ds.x = __fadd_rn(e.x, div_by_k(P, a0));
         ds.y = __fadd_rn(e.y, div_by_k(P, a1));
@@ -234,7 +258,13 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
             const float s = s_k[k];
             a = __fadd_rn(a, (w & 1u) ? s : -s);
           }
-          ds = __fadd_rn(ep[i], div_by_k(P, a));
+          float eo = ep[i];
+          if (LAZY) {
+            const float cs = DC ? sign_code(eo, s_old) : eo;
+            xp[i] = __fsub_rn(xp[i], cs);
+            eo = __fsub_rn(eo, cs);
+          }
+          ds = __fadd_rn(eo, div_by_k(P, a));
           ep[i] = ds;
           if (DC) lane_add(acc, ds);
         }
@@ -342,8 +372,11 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
 // Between the worker pass and the server pass: one thread per (worker, tensor) record turns the exact
 // L1 sum into the scale and clears the record; T more threads clear the server records, which the
 // previous step's apply kernel has finished reading.
+// scale_srv_pending != null: the previous step's server lines are still pending, so its server scales are
+// formed here from the server records before those are cleared (the server pass that follows needs them).
 __global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const int* __restrict__ n, L1Record* recs,
-                                                              float* __restrict__ scale_cur, L1Record* recs_srv) {
+                                                              float* __restrict__ scale_cur, L1Record* recs_srv,
+                                                              float* scale_srv_pending) {
   const int q = blockIdx.x * THREADS + threadIdx.x;
   if (q < K * T) {
     L1Record r = recs[q];
@@ -351,6 +384,7 @@ __global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const
     scale_cur[q] = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], n[q % T]);
   } else if (q < K * T + T) {
     L1Record* r = recs_srv + (q - K * T);
+    if (scale_srv_pending) scale_srv_pending[q - K * T] = scale_from_limbs(r->limb[0], r->limb[1], r->limb[2], n[q - K * T]);
     r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0;
   }
 }
