@@ -413,3 +413,41 @@ def test_folded_averaging_pass_ring_geometries(K, lam):
     """p = 1 with 8, 16 and 32 workers: the worker pass with the averaging folded in, in both of its ring
     geometries (3 deep stages up to 8 workers, 6 shallow ones from 16 on), on ragged and on whole tiles."""
     run_pair(K, [33, 4096, 5000, 700, 3 * 4096, 130], so.SIGN, 5, p=1, lam=lam, seed=6, lrs=[0.1, 0.05])
+
+
+@pytest.mark.parametrize("K,p", [(2, 0), (3, 1), (4, 1), (4, 3), (16, 1), (5, 2)])
+@pytest.mark.parametrize("dc", [0, 1])
+def test_steps_without_getters_in_between(K, p, dc):
+    """With no getter between steps the server lines of a step are left pending and carried out inside the
+    next step's server pass; the state is looked at only every fourth step here (and each look forces the
+    pending lines), so both forms of the server pass and the switch between them are exercised."""
+    run_pair(K, RAGGED, so.SIGN, 13, p=p, dc=dc, seed=8, lrs=[0.1, 0.05, 0.2], every=4)
+
+
+def test_pending_server_lines_survive_a_checkpoint_and_a_side_stream():
+    import torch
+    d = int(np.sum(RAGGED))
+    scales = synth.tensor_scales(9, len(RAGGED), -4.0, -1.0)
+    x0 = synth.x0_numpy(9, d)
+    kw = dict(compressor=so.SIGN, avg_period=3, momentum=0.9)
+    orc = so.Oracle(4, RAGGED, x0, threads=4, **kw)
+    with torch.cuda.stream(torch.cuda.Stream()):          # graph replay: the pending flag is part of the graph key
+        a = sb.Sae(4, RAGGED, torch.from_numpy(x0).cuda(), **kw)
+        gs = [torch.from_numpy(synth.grads_numpy(9, t, 4, RAGGED, scales)).cuda() for t in range(12)]
+        for t in range(7):
+            orc.step(gs[t].cpu().numpy(), 0.1)
+            a.step(gs[t], 0.1)
+        blob = a.save_state()                             # taken with a step's server lines pending
+        b = sb.Sae(4, RAGGED, torch.zeros(d, device="cuda"), **kw)
+        b.load_state(blob)
+        for t in range(7, 12):
+            orc.step(gs[t].cpu().numpy(), 0.1)
+            a.step(gs[t], 0.1)
+            b.step(gs[t], 0.1)
+        compare_state(a, orc, so.SIGN, tag="continued")
+        compare_state(b, orc, so.SIGN, tag="restored")
+        compare_server_messages(a, orc, so.SIGN, 1, tag="continued")
+        compare_server_messages(b, orc, so.SIGN, 1, tag="restored")
+        a.close()
+        b.close()
+    torch.cuda.synchronize()

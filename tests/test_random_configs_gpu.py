@@ -51,8 +51,9 @@ def test_random_configuration(case):
         lr = c["lrs"][t % 3]
         orc.step(g, lr)
         gpu.step(torch.from_numpy(g).cuda(), lr)
-        compare_state(gpu, orc, c["comp"], tag=f"case {case} {c} t={t + 1}")
-        compare_server_messages(gpu, orc, c["comp"], c["dc"], tag=f"case {case} t={t + 1}")
+        if case % 2 == 0 or t in (1, 4):      # odd cases: no getter between most steps (pending server lines)
+            compare_state(gpu, orc, c["comp"], tag=f"case {case} {c} t={t + 1}")
+            compare_server_messages(gpu, orc, c["comp"], c["dc"], tag=f"case {case} t={t + 1}")
     assert not orc.range_flag
     gpu.close()
 
