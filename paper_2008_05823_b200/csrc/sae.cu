@@ -221,12 +221,20 @@ CandArgs cand_args(sae_handle* h, bool server) {
 }
 
 // The server lines a step left pending, carried out now (getters, checkpoints, steps that need x or e).
+#ifndef SAE_LAZY_SERVER
+#define SAE_LAZY_SERVER 1        // 0: every step runs its own apply kernel
+#endif
 int flush_server(sae_handle* h) {
   if (!h->srv_pending) return SAE_OK;
   ApplyArgs aa;
   memset(&aa, 0, sizeof(aa));
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
-  if (h->cfg.server_compress) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), h->P.ntiles, h->P, aa);
+  aa.tau_srv = h->tau_srv; aa.mask_srv = h->mask_srv;
+  const bool dcs = h->cfg.server_compress != 0;
+  if (h->cfg.compressor == SAE_COMPRESSOR_TOPK) {
+    if (dcs) LAUNCH(h, S_APPLY, (k_apply<2, 2, AVG_NONE>), h->P.ntiles, h->P, aa);
+    else LAUNCH(h, S_APPLY, (k_apply<2, 0, AVG_NONE>), h->P.ntiles, h->P, aa);
+  } else if (dcs) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), h->P.ntiles, h->P, aa);
   else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), h->P.ntiles, h->P, aa);
   h->srv_pending = 0;
   return check_launch(h);
@@ -351,6 +359,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
   wa.cand = cand_args(h, false);
   ServerArgs sa;
+  memset(&sa, 0, sizeof(sa));
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
   // inline_fin: step t accumulates the server's L1 into one buffer while the apply kernel clears the other
   L1Record* const recs_srv_now = (h->inline_fin && cur) ? h->recs_srv_alt : h->recs_srv;
@@ -360,6 +369,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = ebar_now(h);
   sa.m = h->m; sa.ebar_in = ebar_now(h); sa.eta = lr;
   ApplyArgs aa;
+  memset(&aa, 0, sizeof(aa));
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = ebar_now(h); aa.m = h->m; aa.D = h->D;
   aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = recs_srv_now; aa.tau_cur = h->tau[cur];
   aa.recs_clear = h->inline_fin ? h->recs : nullptr; aa.recs_srv_clear = recs_srv_next;
@@ -387,9 +397,6 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     }
     // The server lines of this step can be left to the next step's server pass when nothing in between
     // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
-#ifndef SAE_LAZY_SERVER
-#define SAE_LAZY_SERVER 1
-#endif
     const bool lazy_ok = SAE_LAZY_SERVER && !h->inline_fin && !sp.wd;
     if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
     const bool pending = h->srv_pending != 0;
@@ -422,6 +429,11 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     const bool nod = h->topk_nod;
     if (nod && !(h->esrc == ESRC_UNIFORM && avg_after)) return SAE_ERR_INVALID_ARG;
     if (!nod && !h->D) return SAE_ERR_INVALID_ARG;
+    // the server lines wait for the next dense server pass unless the worker pass needs x (weight decay)
+    const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
+    if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
+    const int lsrv = h->srv_pending ? (dc ? 2 : 1) : 0;
+    sa.x = h->x; sa.mask_srv = h->mask_srv;
     DeltaSrc src = stored_rows(h->D);
     if (nod) { src.m = h->m; src.ebar = ebar_now(h); src.eta = lr; src.recompute = 1; }
     if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
@@ -429,13 +441,24 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
     topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
     // the averaged error (if the pre-step averages) comes out of the same pass over D as the server's sum
-    if (nod) {
-      sa.ebar = ebar_other(h);          // becomes the current one when `last` flips below
-      LAUNCH(h, S_SERVER, (k_server_dense<2, true, true>), P.ntiles, P, sa);
-    } else if (avg_after) LAUNCH(h, S_SERVER, (k_server_dense<2, true>), P.ntiles, P, sa);
-    else LAUNCH(h, S_SERVER, (k_server_dense<2, false>), P.ntiles, P, sa);
+    if (nod) sa.ebar = ebar_other(h);          // becomes the current one when `last` flips below
+#define SAE_DENSE(AVGF, RECF)                                                                              \
+    do {                                                                                                   \
+      if (lsrv == 0) LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 0>), P.ntiles, P, sa);             \
+      else if (lsrv == 1) LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 1>), P.ntiles, P, sa);        \
+      else LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 2>), P.ntiles, P, sa);                       \
+    } while (0)
+    if (nod) SAE_DENSE(true, true);
+    else if (avg_after) SAE_DENSE(true, false);
+    else SAE_DENSE(false, false);
+#undef SAE_DENSE
     if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
-    if (dc) launch_apply<2, 2>(h, AVG_NONE, aa); else launch_apply<2, 0>(h, AVG_NONE, aa);
+    if (lazy_ok) {
+      h->srv_pending = 1;
+    } else {
+      h->srv_pending = 0;
+      if (dc) launch_apply<2, 2>(h, AVG_NONE, aa); else launch_apply<2, 0>(h, AVG_NONE, aa);
+    }
     h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
   } else {
     // identity: every error stays exactly zero, so e^(k) is the (all-zero) uniform vector forever
@@ -985,7 +1008,10 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
   if (per_worker && (worker < 0 || worker >= P.K)) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
-  if (which == SAE_STATE_SERVER_SCALES) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
+  if (which == SAE_STATE_SERVER_SCALES || which == SAE_STATE_SERVER_MASK) {
+    int rcf = flush_server(h);
+    if (rcf != SAE_OK) return rcf;
+  }
   const bool sign = h->cfg.compressor == SAE_COMPRESSOR_SIGN, topk = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
   const size_t vec = sizeof(float) * (size_t)P.d, tb = sizeof(float) * (size_t)P.T, wb = sizeof(u32) * (size_t)P.nwords;
   const void* src = nullptr; size_t need = 0;

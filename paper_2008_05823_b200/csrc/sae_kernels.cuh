@@ -83,6 +83,7 @@ struct ServerArgs {
   // re-updated; both are brought up to date here, element by element, before this step's Delta is formed
   float* x;                        // [dpad]
   const float* scale_srv_prev;     // [T] server scales of the previous step (double-way)
+  u32* mask_srv;                   // [nwords] Top-K: the server's selection of the previous step (written when pending)
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -286,7 +287,10 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 // RECOMP (Top-K with p = 1: the previous error is uniform and the pre-step averages, every step): the worker
 // pass did not store D^(k); it is recomputed here from m^(k) and the previous uniform error with the fused
 // operation that formed it, so the step moves 4 bytes per worker-element less.
-template <int COMP, bool AVG, bool RECOMP = false>
+// LSRV != 0 (Top-K): the previous step left its server lines pending -- e = Delta - C(Delta), x = x - C(Delta)
+// and the server's selection words; they are carried out here on the fly with last step's server threshold
+// (LSRV 2) or with C = identity (LSRV 1, single-way), the same operations the apply kernel would have done.
+template <int COMP, bool AVG, bool RECOMP = false, int LSRV = 0>
 __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
@@ -303,11 +307,28 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   float* ep = A.e_srv + pbase;
   const float* __restrict__ dp = (RECOMP ? A.m : A.D) + pbase;
   const float* __restrict__ eo = A.ebar_in + pbase;      // read only when RECOMP
+  float* xp = A.x + pbase;                               // (LSRV only)
+  u32* mwp = A.mask_srv + (pbase >> 5);                  // (LSRV 2 only)
+  const u32 t_old = (LSRV == 2) ? A.tau_srv_prev[ti.j] : 0u;
+  const int lane = tid & 31, warp = tid >> 5;
   if (ti.cnt == TILE) {
 #pragma unroll 2
     for (int it = 0; it < VEC_ITERS; ++it) {
       const int i = it * (THREADS * 4) + tid * 4;
-      const float4 e = ld4(ep + i);
+      float4 e = ld4(ep + i);
+      if (LSRV != 0) {
+        float4 xv = ld4(xp + i);
+        const bool q0 = LSRV == 1 || topk_selected(e.x, t_old), q1 = LSRV == 1 || topk_selected(e.y, t_old);
+        const bool q2 = LSRV == 1 || topk_selected(e.z, t_old), q3 = LSRV == 1 || topk_selected(e.w, t_old);
+        const float c0 = q0 ? e.x : 0.0f, c1 = q1 ? e.y : 0.0f, c2 = q2 ? e.z : 0.0f, c3 = q3 ? e.w : 0.0f;
+        xv.x = __fsub_rn(xv.x, c0); xv.y = __fsub_rn(xv.y, c1); xv.z = __fsub_rn(xv.z, c2); xv.w = __fsub_rn(xv.w, c3);
+        st4(xp + i, xv);
+        e.x = __fsub_rn(e.x, c0); e.y = __fsub_rn(e.y, c1); e.z = __fsub_rn(e.z, c2); e.w = __fsub_rn(e.w, c3);
+        if (LSRV == 2) {
+          const u32 w = pack_row4(q0, q1, q2, q3);
+          if ((lane & 7) == 0) mwp[i >> 5] = w;
+        }
+      }
       float4 eold = make_float4(0.f, 0.f, 0.f, 0.f);
       if (RECOMP) eold = ld4(eo + i);
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -346,19 +367,31 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
     for (int r = 0; r < ROWS; ++r) {
       const int i = r * THREADS + tid;
       float ds = 0.0f;
+      bool qs = false;
       if (i < ti.cnt) {
         float a = 0.f, b = 0.f;
-        const float eold = RECOMP ? eo[i] : 0.0f;
+        const float ebo = RECOMP ? eo[i] : 0.0f;
         for (int k = 0; k < P.K; ++k) {
           float v = dp[(long long)k * P.dpad + i];
-          if (RECOMP) v = __fmaf_rn(A.eta, v, eold);
+          if (RECOMP) v = __fmaf_rn(A.eta, v, ebo);
           const float c = (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f;
           a = __fadd_rn(a, c);
           if (AVG) b = __fadd_rn(b, __fsub_rn(v, c));
         }
         if (AVG) A.ebar[pbase + i] = div_by_k(P, b);
-        ds = __fadd_rn(ep[i], div_by_k(P, a));
+        float eold = ep[i];
+        if (LSRV != 0) {
+          qs = LSRV == 1 || topk_selected(eold, t_old);
+          const float cs = qs ? eold : 0.0f;
+          xp[i] = __fsub_rn(xp[i], cs);
+          eold = __fsub_rn(eold, cs);
+        }
+        ds = __fadd_rn(eold, div_by_k(P, a));
         ep[i] = ds;
+      }
+      if (LSRV == 2) {
+        const u32 w = __ballot_sync(0xffffffffu, qs);
+        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) mwp[(r * THREADS + warp * 32) >> 5] = w;
       }
       if (COMP == 2 && lo != NO_GUESS) {
         if (stg.n > CAND_STAGE - 32) stage_flush(stg, A.cand_srv, 0, ti.j);
