@@ -415,13 +415,15 @@ def test_folded_averaging_pass_ring_geometries(K, lam):
     run_pair(K, [33, 4096, 5000, 700, 3 * 4096, 130], so.SIGN, 5, p=1, lam=lam, seed=6, lrs=[0.1, 0.05])
 
 
+@pytest.mark.parametrize("comp", [so.SIGN, so.TOPK])
 @pytest.mark.parametrize("K,p", [(2, 0), (3, 1), (4, 1), (4, 3), (16, 1), (5, 2)])
 @pytest.mark.parametrize("dc", [0, 1])
-def test_steps_without_getters_in_between(K, p, dc):
+def test_steps_without_getters_in_between(K, p, dc, comp):
     """With no getter between steps the server lines of a step are left pending and carried out inside the
     next step's server pass; the state is looked at only every fourth step here (and each look forces the
     pending lines), so both forms of the server pass and the switch between them are exercised."""
-    run_pair(K, RAGGED, so.SIGN, 13, p=p, dc=dc, seed=8, lrs=[0.1, 0.05, 0.2], every=4)
+    run_pair(K, RAGGED, comp, 13, p=p, dc=dc, seed=8, lrs=[0.1, 0.05, 0.2], every=4, num=1, den=20,
+             outliers=(66, 100.0))
 
 
 def test_pending_server_lines_survive_a_checkpoint_and_a_side_stream():
