@@ -214,8 +214,8 @@ def run_sharded(args, w, p, rank, local_rank, world):
     from paper_2008_05823_b200 import configs, synth
     from paper_2008_05823_b200.sharded import sharded_sae, worker_range
 
-    if w.compressor != configs.SIGN:
-        raise SystemExit("--sharded: scaled sign only")
+    if w.compressor == configs.IDENTITY:
+        raise SystemExit("--sharded: scaled sign or Top-K")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -238,15 +238,15 @@ def run_sharded(args, w, p, rank, local_rank, world):
         g = torch.empty(count, d, device=dev)
         gen.grads(g, count, args.seed + 1000 * rank, t, w.outlier_per_65536, w.outlier_mult)   # timing only
         grads.append(g)
-    kw = dict(server_compress=w.server_compress, mode=w.mode, avg_period=p, momentum=w.momentum,
-              weight_decay=w.weight_decay)
+    kw = dict(compressor=w.compressor, server_compress=w.server_compress, mode=w.mode, avg_period=p,
+              momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num, topk_den=w.topk_den)
     if world > 1:
         run = sharded_sae(K, w.tensor_sizes, x0, **kw)
         eng = run.engine
         step = lambda g: run.step(g, w.lr)
         finish = run.finish
     else:
-        eng = sb.Sae(K, w.tensor_sizes, x0, compressor=sb.SIGN, shard=(0, K), **kw)
+        eng = sb.Sae(K, w.tensor_sizes, x0, shard=(0, K), **kw)
         eng.shard_attach(eng.shard_export())
 
         def step(g):                       # one stream: begin is ordered before end, end before the next begin
@@ -303,7 +303,8 @@ def run_sharded(args, w, p, rank, local_rank, world):
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": w.name + "_sharded", "num_workers": K, "workers_per_rank": count, "d": d,
-                           "num_tensors": w.num_tensors, "compressor": "scaled_sign", "avg_period": p,
+                           "num_tensors": w.num_tensors,
+                           "compressor": {1: "scaled_sign", 2: "topk"}[w.compressor], "avg_period": p,
                            "parallelism": f"sharded: {K} workers over {world} rank(s); every rank's server pass reads "
                                           "all messages in place through row tables",
                            "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient "

@@ -186,7 +186,7 @@ int64_t sae_kernel_launches(const sae_handle *h);
 
 /*
  * Sharded operation: the K workers of Algorithm 1 spread over several handles ("shards": one per GPU /
- * process), scaled-sign compressor.  A shard owns workers worker_begin .. worker_begin+num_local_workers-1:
+ * process), scaled-sign or Top-K compressor.  A shard owns workers worker_begin .. worker_begin+num_local_workers-1:
  * their momentum, error and message rows live in its memory.  The server lines ("Server: receive ...,
  * send C(Delta)") are replicated: every shard keeps x and the server error e and computes the same bits,
  * because it reads all K messages (1 scale per tensor + 1 bit per element per worker, Eq. 2) in k order.
@@ -196,8 +196,12 @@ int64_t sae_kernel_launches(const sae_handle *h);
  * kernel.  Error averaging (pre-step, every p iterations) likewise reads the owners' stored model
  * differences in place.
  *
- *   sae_init_shard    cfg->num_workers is K of the whole job; otherwise as sae_init (compressor must be
- *                     SAE_COMPRESSOR_SIGN).  Worker indices of the getters are LOCAL (0 .. num_local-1).
+ *   sae_init_shard    cfg->num_workers is K of the whole job; otherwise as sae_init (the identity compressor
+ *                     is not sharded).  Worker indices of the getters are LOCAL (0 .. num_local-1).
+ *                     Top-K: a worker's message is the list of its selected (index, value) entries (Section
+ *                     3.1), compacted by its owner once the thresholds are known; every shard adds all K lists
+ *                     in k order, reading them in place (an unselected entry contributes an exact zero, so the
+ *                     ordered sum over the selecting workers is the full ordered sum).
  *   sae_shard_export  writes SAE_SHARD_BLOB_BYTES bytes (HOST) describing where this shard's rows live: raw
  *                     pointers for handles of the same process, CUDA IPC handles for other processes.
  *   sae_shard_attach  makes the rows of one exported blob (any shard's, including this handle's own) known
@@ -219,7 +223,7 @@ int64_t sae_kernel_launches(const sae_handle *h);
  * additions is the library's, not k = 0..K-1: the averaged error then agrees with Algorithm 1 to fp32
  * rounding, not bit for bit (with one shard it is exact).  sae_step_begin is refused while the sum is owed.
  *
- * Errors: SAE_ERR_INVALID_ARG for a null pointer, a compressor other than scaled sign, a worker range outside
+ * Errors: SAE_ERR_INVALID_ARG for a null pointer, the identity compressor, a worker range outside
  * 0..K-1, a blob that is too short / foreign / describes another parameter list / names rows that are already
  * attached, sae_step_begin before every worker's rows are attached or while a step is open, sae_step_end
  * without an open step, sae_shard_attach / sae_shard_detach / checkpoint calls while a step is open;
@@ -232,7 +236,7 @@ int64_t sae_kernel_launches(const sae_handle *h);
  * any shard's next sae_step_begin (which overwrites them).  Shards of one process on one stream need
  * nothing: stream order already gives both.  sae_step and sae_step_host refuse a sharded handle.
  */
-#define SAE_SHARD_BLOB_BYTES 512
+#define SAE_SHARD_BLOB_BYTES 1024
 int sae_init_shard(const sae_config *cfg, int32_t worker_begin, int32_t num_local_workers, const float *x0,
                    sae_handle **out);
 int sae_shard_export(sae_handle *h, void *blob_host, size_t bytes);

@@ -28,7 +28,7 @@ EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_p
            "sae_shard_attach", "sae_shard_detach", "sae_step_begin", "sae_step_end", "sae_shard_set_avg_mode", "sae_avg_due",
            "sae_num_padded", "sae_avg_local_sum", "sae_avg_set"]
 
-SHARD_BLOB_BYTES = 512
+SHARD_BLOB_BYTES = 1024
 
 
 class SaeConfig(C.Structure):

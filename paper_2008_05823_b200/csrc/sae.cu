@@ -4,6 +4,7 @@
 #include "sae_kernels.cuh"
 #include "sae_worker_tma.cuh"
 #include "sae_worker_fused.cuh"
+#include "sae_shard_topk.cuh"
 
 #include <cuda.h>
 #include <cudaTypedefs.h>
@@ -93,6 +94,15 @@ struct sae_handle {
   const u32** d_word_rows;
   const float** d_scale_rows[2];
   const float** d_d_rows;
+  // sharded Top-K: the local workers' messages (lists of selected entries) and the tables over all workers
+  unsigned long long* msg_entries;  // [K_loc][cand_stride]
+  u32* msg_count;                   // [K_loc][T]
+  float* agg_acc;                   // [dpad] scratch of the ordered sparse sum, zero between uses
+  std::vector<const unsigned long long*> h_entry_rows;
+  std::vector<const u32*> h_count_rows, h_tau_rows[2];
+  const unsigned long long** d_entry_rows;
+  const u32** d_count_rows;
+  const u32** d_tau_rows[2];
   std::vector<void*> ipc_opened;    // mappings of other processes' buffers, closed by sae_destroy
   // cached step graphs
   int graphs_enabled, graph_misses;
@@ -172,7 +182,9 @@ void free_all(sae_handle* h) {
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
-  void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows};
+  void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows,
+                  (void*)h->d_entry_rows, (void*)h->d_count_rows, (void*)h->d_tau_rows[0], (void*)h->d_tau_rows[1],
+                  (void*)h->msg_entries, (void*)h->msg_count, (void*)h->agg_acc};
   for (void* p : tabs) if (p) cudaFree(p);
   for (void* p : h->ipc_opened) cudaIpcCloseMemHandle(p);
   if (h->status_host) cudaFreeHost(h->status_host);
@@ -620,7 +632,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
     return SAE_ERR_INVALID_ARG;
   if (cfg->device < 0) return SAE_ERR_INVALID_ARG;
   if (k0 < 0 || K_loc < 1 || k0 + K_loc > cfg->num_workers) return SAE_ERR_INVALID_ARG;
-  if (shard && cfg->compressor != SAE_COMPRESSOR_SIGN) return SAE_ERR_INVALID_ARG;
+  if (shard && cfg->compressor == SAE_COMPRESSOR_IDENTITY) return SAE_ERR_INVALID_ARG;
   const int T = cfg->num_tensors, K = K_loc;          // K: worker rows held by this handle
   long long d = 0, dpad = 0, ntiles = 0;
   for (int j = 0; j < T; ++j) {
@@ -666,7 +678,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
     }
   }
   const bool sign = cfg->compressor == SAE_COMPRESSOR_SIGN, topk = cfg->compressor == SAE_COMPRESSOR_TOPK;
-  h->topk_nod = (topk && cfg->avg_period == 1) ? 1 : 0;
+  h->topk_nod = (!shard && topk && cfg->avg_period == 1) ? 1 : 0;      // (a shard always stores its differences)
   h->mu0 = (cfg->momentum == 0.0f && cfg->avg_period != 1) ? 1 : 0;
   const bool need_D = shard || !((sign || topk) && cfg->avg_period == 1);
   const long long nwords = dpad / 32;
@@ -754,6 +766,20 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
     if (e == cudaSuccess) e = dalloc(&h->d_scale_rows[0], Kt);
     if (e == cudaSuccess) e = dalloc(&h->d_scale_rows[1], Kt);
     if (e == cudaSuccess) e = dalloc(&h->d_d_rows, Kt);
+    if (topk) {
+      h->h_entry_rows.assign(Kt, nullptr); h->h_count_rows.assign(Kt, nullptr);
+      h->h_tau_rows[0].assign(Kt, nullptr); h->h_tau_rows[1].assign(Kt, nullptr);
+      if (e == cudaSuccess) e = dalloc(&h->d_entry_rows, Kt);
+      if (e == cudaSuccess) e = dalloc(&h->d_count_rows, Kt);
+      if (e == cudaSuccess) e = dalloc(&h->d_tau_rows[0], Kt);
+      if (e == cudaSuccess) e = dalloc(&h->d_tau_rows[1], Kt);
+      if (e == cudaSuccess) e = dalloc(&h->msg_entries, (size_t)K * (size_t)h->cand_stride);
+      if (e == cudaSuccess) e = dalloc(&h->msg_count, KT);
+      if (e == cudaSuccess) e = dalloc(&h->agg_acc, (size_t)dpad);
+      if (e == cudaSuccess) e = cudaMemsetAsync(h->msg_count, 0, KT * sizeof(u32), h->stream);
+      if (e == cudaSuccess) e = cudaMemsetAsync(h->agg_acc, 0, (size_t)dpad * sizeof(float), h->stream);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    }
     if (e != cudaSuccess) { h->last_cuda_error = (int)e; g_init_cuda_error = (int)e; cudaGetLastError(); rc = SAE_ERR_NOMEM; }
   }
   if (rc != SAE_OK) { free_all(h); delete h; return rc; }
@@ -769,10 +795,13 @@ struct ShardBlob {
   uint64_t magic;
   int32_t pid, device, worker_begin, num_local, T, pad;
   int64_t nwords, dpad;
-  void* raw[4];                       // words, scale[0], scale[1], D
-  cudaIpcMemHandle_t ipc[4];
+  int32_t compressor, pad2;
+  int64_t cand_stride;
+  void* raw[8];                       // words, scale[0], scale[1], D | Top-K: entries, counts, tau[0], tau[1]
+  cudaIpcMemHandle_t ipc[8];
 };
-constexpr uint64_t kShardMagic = 0x5341455F53484431ull;   // "SAE_SHD1"
+constexpr int kShardBufs = 8;
+constexpr uint64_t kShardMagic = 0x5341455F53484432ull;   // "SAE_SHD2"
 static_assert(sizeof(ShardBlob) <= SAE_SHARD_BLOB_BYTES, "blob must fit the documented size");
 
 int shard_begin(sae_handle* h, const float* grads, float lr) {
@@ -787,6 +816,19 @@ int shard_begin(sae_handle* h, const float* grads, float lr) {
   wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
   wa.cand = cand_args(h, false);
+  if (c.compressor == SAE_COMPRESSOR_TOPK) {
+    // worker lines, the local workers' thresholds, then their messages: the lists of selected entries
+    SAE_CUDA(h, cudaMemsetAsync(h->msg_count, 0, sizeof(u32) * (size_t)P.K * P.T, h->stream));
+    if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
+    else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
+    topk_thresholds(h, stored_rows(h->D), P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+    SparseMsgArgs ma;
+    ma.D = h->D; ma.tau = h->tau[cur]; ma.entries = h->msg_entries; ma.off = h->d_cand_off; ma.cap = h->d_cand_cap;
+    ma.stride = h->cand_stride; ma.count = h->msg_count;
+    LAUNCH(h, S_TOPK_SELECT, k_topk_compact, (long long)P.ntiles * P.K, P, ma);
+    h->mid_step = 1; h->lr_pending = lr;
+    return check_launch(h);
+  }
   // the model differences are always stored: the averaging reads them from every owner
   if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
   else launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
@@ -810,6 +852,30 @@ int shard_end(sae_handle* h) {
   memset(&aa, 0, sizeof(aa));
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
   aa.eta = h->lr_pending;
+  if (c.compressor == SAE_COMPRESSOR_TOPK) {
+    // the ordered worker-axis sum from every owner's list of selected entries, then the server lines
+    SparseAggArgs ga;
+    ga.e_srv = h->e_srv; ga.acc = h->agg_acc; ga.entry_rows = h->d_entry_rows; ga.count_rows = h->d_count_rows;
+    ga.d_rows = h->d_d_rows; ga.tau_rows = h->d_tau_rows[cur]; ga.off = h->d_cand_off; ga.cap = h->d_cand_cap;
+    {
+      LaunchScope ls(h, S_SERVER);
+      k_topk_sparse_aggregate<<<(unsigned)((PA.ntiles + AGG_TILES - 1) / AGG_TILES), AGG_THREADS, 0, h->stream>>>(PA, ga);
+    }
+    aa.tau_srv = h->tau_srv; aa.mask_srv = h->mask_srv;
+    if (dc) {
+      LAUNCH(h, S_SERVER, k_server_candidates, PA.ntiles, PA, h->e_srv, cand_args(h, true), h->tau_srv);
+      topk_thresholds(h, stored_rows(h->e_srv), 1, cand_args(h, true), h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
+      LAUNCH(h, S_APPLY, (k_apply<2, 2, AVG_NONE>), PA.ntiles, PA, aa);
+    } else {
+      LAUNCH(h, S_APPLY, (k_apply<2, 0, AVG_NONE>), PA.ntiles, PA, aa);
+    }
+    if (avg_after && !h->avg_external)
+      LAUNCH(h, S_APPLY, (k_avg_pull<false, 2>), PA.ntiles, PA, h->d_d_rows, (const void* const*)h->d_tau_rows[cur], h->ebar);
+    if (avg_after && h->avg_external) h->avg_owed = 1;
+    h->esrc = (avg_after && !h->avg_external) ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
+    h->last = cur; h->eta_prev = h->lr_pending; h->t += 1; h->mid_step = 0;
+    return check_launch(h);
+  }
   const int tpb = std::max(1, std::min(8, PA.ntiles / (h->num_sms * 16)));
   const int nblk = (PA.ntiles + tpb - 1) / tpb;
   if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, true>), nblk, PA, sa, tpb);
@@ -817,7 +883,7 @@ int shard_end(sae_handle* h) {
   if (dc) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), PA.ntiles, PA, aa);
   else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), PA.ntiles, PA, aa);
   if (avg_after && !h->avg_external)
-    LAUNCH(h, S_APPLY, k_avg_pull<false>, PA.ntiles, PA, h->d_d_rows, h->d_scale_rows[cur], h->ebar);
+    LAUNCH(h, S_APPLY, (k_avg_pull<false, 1>), PA.ntiles, PA, h->d_d_rows, (const void* const*)h->d_scale_rows[cur], h->ebar);
   if (avg_after && h->avg_external) h->avg_owed = 1;     // the error stays "lazy" until sae_avg_set
   h->esrc = (avg_after && !h->avg_external) ? ESRC_UNIFORM : ESRC_LAZY_SIGN;
   h->last = cur; h->eta_prev = h->lr_pending; h->t += 1; h->mid_step = 0;
@@ -849,8 +915,11 @@ int sae_shard_export(sae_handle* h, void* blob_host, size_t bytes) {
   memset(&b, 0, sizeof(b));
   b.magic = kShardMagic; b.pid = (int32_t)getpid(); b.device = h->device; b.worker_begin = h->k0; b.num_local = h->P.K;
   b.T = h->P.T; b.nwords = h->P.nwords; b.dpad = h->P.dpad;
+  b.compressor = h->cfg.compressor; b.cand_stride = h->cand_stride;
   b.raw[0] = h->words; b.raw[1] = h->scale[0]; b.raw[2] = h->scale[1]; b.raw[3] = h->D;
-  for (int q = 0; q < 4; ++q) SAE_CUDA(h, cudaIpcGetMemHandle(&b.ipc[q], b.raw[q]));
+  b.raw[4] = h->msg_entries; b.raw[5] = h->msg_count; b.raw[6] = h->tau[0]; b.raw[7] = h->tau[1];
+  for (int q = 0; q < kShardBufs; ++q)
+    if (b.raw[q]) SAE_CUDA(h, cudaIpcGetMemHandle(&b.ipc[q], b.raw[q]));
   memset(blob_host, 0, SAE_SHARD_BLOB_BYTES);
   memcpy(blob_host, &b, sizeof(b));
   return SAE_OK;
@@ -863,25 +932,35 @@ int sae_shard_attach(sae_handle* h, const void* blob_host, size_t bytes) {
   ShardBlob b;
   memcpy(&b, blob_host, sizeof(b));
   if (b.magic != kShardMagic || b.T != h->P.T || b.nwords != h->P.nwords || b.dpad != h->P.dpad || b.worker_begin < 0 ||
-      b.num_local < 1 || b.worker_begin + b.num_local > h->K_total)
+      b.num_local < 1 || b.worker_begin + b.num_local > h->K_total || b.compressor != h->cfg.compressor ||
+      b.cand_stride != h->cand_stride)
     return SAE_ERR_INVALID_ARG;
   for (int q = 0; q < b.num_local; ++q)
     if (h->h_word_rows[(size_t)b.worker_begin + q]) return SAE_ERR_INVALID_ARG;      // rows already attached
-  void* base[4];
+  void* base[kShardBufs];
   if (b.pid == (int32_t)getpid()) {
-    for (int q = 0; q < 4; ++q) base[q] = b.raw[q];
+    for (int q = 0; q < kShardBufs; ++q) base[q] = b.raw[q];
   } else {
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < kShardBufs; ++q) {
+      base[q] = nullptr;
+      if (!b.raw[q]) continue;
       SAE_CUDA(h, cudaIpcOpenMemHandle(&base[q], b.ipc[q], cudaIpcMemLazyEnablePeerAccess));
       h->ipc_opened.push_back(base[q]);
     }
   }
+  const bool topk_rows = h->cfg.compressor == SAE_COMPRESSOR_TOPK;
   for (int q = 0; q < b.num_local; ++q) {
     const size_t k = (size_t)b.worker_begin + q;
     h->h_word_rows[k] = (const u32*)base[0] + (size_t)q * b.nwords;
     h->h_scale_rows[0][k] = (const float*)base[1] + (size_t)q * b.T;
     h->h_scale_rows[1][k] = (const float*)base[2] + (size_t)q * b.T;
     h->h_d_rows[k] = (const float*)base[3] + (size_t)q * b.dpad;
+    if (topk_rows) {
+      h->h_entry_rows[k] = (const unsigned long long*)base[4] + (size_t)q * (size_t)b.cand_stride;
+      h->h_count_rows[k] = (const u32*)base[5] + (size_t)q * b.T;
+      h->h_tau_rows[0][k] = (const u32*)base[6] + (size_t)q * b.T;
+      h->h_tau_rows[1][k] = (const u32*)base[7] + (size_t)q * b.T;
+    }
   }
   h->attached += b.num_local;
   if (h->attached == h->K_total) {
@@ -890,6 +969,12 @@ int sae_shard_attach(sae_handle* h, const void* blob_host, size_t bytes) {
     SAE_CUDA(h, cudaMemcpyAsync(h->d_scale_rows[0], h->h_scale_rows[0].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
     SAE_CUDA(h, cudaMemcpyAsync(h->d_scale_rows[1], h->h_scale_rows[1].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
     SAE_CUDA(h, cudaMemcpyAsync(h->d_d_rows, h->h_d_rows.data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    if (topk_rows) {
+      SAE_CUDA(h, cudaMemcpyAsync(h->d_entry_rows, h->h_entry_rows.data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+      SAE_CUDA(h, cudaMemcpyAsync(h->d_count_rows, h->h_count_rows.data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+      SAE_CUDA(h, cudaMemcpyAsync(h->d_tau_rows[0], h->h_tau_rows[0].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+      SAE_CUDA(h, cudaMemcpyAsync(h->d_tau_rows[1], h->h_tau_rows[1].data(), Kt * sizeof(void*), cudaMemcpyHostToDevice, h->stream));
+    }
     SAE_CUDA(h, cudaStreamSynchronize(h->stream));
   }
   return SAE_OK;
@@ -906,6 +991,10 @@ int sae_shard_detach(sae_handle* h) {
   for (auto& r : h->h_d_rows) r = nullptr;
   for (auto& r : h->h_scale_rows[0]) r = nullptr;
   for (auto& r : h->h_scale_rows[1]) r = nullptr;
+  for (auto& r : h->h_entry_rows) r = nullptr;
+  for (auto& r : h->h_count_rows) r = nullptr;
+  for (auto& r : h->h_tau_rows[0]) r = nullptr;
+  for (auto& r : h->h_tau_rows[1]) r = nullptr;
   h->attached = 0;
   return SAE_OK;
 }
@@ -924,8 +1013,12 @@ int sae_avg_local_sum(sae_handle* h, float* sum_padded) {
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
   // this shard's own rows, k in order: the table entries k0 .. k0+K-1 with the local plan (K = local workers)
-  LAUNCH(h, S_APPLY, k_avg_pull<true>, h->P.ntiles, h->P, h->d_d_rows + h->k0, h->d_scale_rows[h->last] + h->k0,
-         sum_padded);
+  if (h->cfg.compressor == SAE_COMPRESSOR_TOPK)
+    LAUNCH(h, S_APPLY, (k_avg_pull<true, 2>), h->P.ntiles, h->P, h->d_d_rows + h->k0,
+           (const void* const*)(h->d_tau_rows[h->last] + h->k0), sum_padded);
+  else
+    LAUNCH(h, S_APPLY, (k_avg_pull<true, 1>), h->P.ntiles, h->P, h->d_d_rows + h->k0,
+           (const void* const*)(h->d_scale_rows[h->last] + h->k0), sum_padded);
   return check_launch(h);
 }
 

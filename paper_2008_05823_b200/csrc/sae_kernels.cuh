@@ -426,14 +426,21 @@ __global__ void __launch_bounds__(THREADS) k_finalize_scales(int K, int T, const
 // e^(k) = D^(k) - C(D^(k)) formed from every owner's stored model differences and scales, read in place
 // through row tables (the same subtraction, order and division as the unsharded averaging in k_apply).
 // SUM_ONLY (rows = this shard's own workers): the undivided partial sum, for an all-reduce across shards.
-template <bool SUM_ONLY>
+// COMP 1: aux_rows[k] -> worker k's [T] scales (float); COMP 2: -> its [T] Top-K thresholds (u32).
+template <bool SUM_ONLY, int COMP = 1>
 __global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const* __restrict__ d_rows,
-                                                       const float* const* __restrict__ scale_rows, float* ebar) {
+                                                       const void* const* __restrict__ aux_rows, float* ebar) {
+  constexpr int ES = (COMP == 1) ? ESRC_LAZY_SIGN : ESRC_LAZY_TOPK;
   __shared__ float s_k[MAX_WORKERS];
+  __shared__ u32 t_k[MAX_WORKERS];
   __shared__ const float* s_row[MAX_WORKERS];
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
-  for (int k = tid; k < P.K; k += THREADS) { s_k[k] = scale_rows[k][ti.j]; s_row[k] = d_rows[k]; }
+  for (int k = tid; k < P.K; k += THREADS) {
+    s_k[k] = (COMP == 1) ? reinterpret_cast<const float*>(aux_rows[k])[ti.j] : 0.0f;
+    t_k[k] = (COMP == 2) ? reinterpret_cast<const u32*>(aux_rows[k])[ti.j] : 0u;
+    s_row[k] = d_rows[k];
+  }
   __syncthreads();
   const long long pbase = ti.poff + ti.t0;
   if (ti.cnt == TILE) {
@@ -444,10 +451,11 @@ __global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const
       for (int k = 0; k < P.K; ++k) {
         const float4 v = ld4(s_row[k] + pbase + i);
         const float s = s_k[k];
-        b0 = __fadd_rn(b0, prev_error<ESRC_LAZY_SIGN>(v.x, s, 0u));
-        b1 = __fadd_rn(b1, prev_error<ESRC_LAZY_SIGN>(v.y, s, 0u));
-        b2 = __fadd_rn(b2, prev_error<ESRC_LAZY_SIGN>(v.z, s, 0u));
-        b3 = __fadd_rn(b3, prev_error<ESRC_LAZY_SIGN>(v.w, s, 0u));
+        const u32 t = t_k[k];
+        b0 = __fadd_rn(b0, prev_error<ES>(v.x, s, t));
+        b1 = __fadd_rn(b1, prev_error<ES>(v.y, s, t));
+        b2 = __fadd_rn(b2, prev_error<ES>(v.z, s, t));
+        b3 = __fadd_rn(b3, prev_error<ES>(v.w, s, t));
       }
       if (SUM_ONLY) st4(ebar + pbase + i, make_float4(b0, b1, b2, b3));
       else st4(ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
@@ -455,7 +463,7 @@ __global__ void __launch_bounds__(THREADS) k_avg_pull(Plan P, const float* const
   } else {
     for (int i = tid; i < ti.cnt; i += THREADS) {
       float b = 0.f;
-      for (int k = 0; k < P.K; ++k) b = __fadd_rn(b, prev_error<ESRC_LAZY_SIGN>(s_row[k][pbase + i], s_k[k], 0u));
+      for (int k = 0; k < P.K; ++k) b = __fadd_rn(b, prev_error<ES>(s_row[k][pbase + i], s_k[k], t_k[k]));
       ebar[pbase + i] = SUM_ONLY ? b : div_by_k(P, b);
     }
   }

@@ -105,10 +105,11 @@ class ShardedRun:
 
 
 def sharded_sae(num_workers, tensor_sizes, x0, group=None, barrier=None, allreduce_average=False, **kw) -> ShardedRun:
-    """ShardedRun over the CUDA library: every rank passes the same num_workers, tensor_sizes, x0 and options."""
+    """ShardedRun over the CUDA library: every rank passes the same num_workers, tensor_sizes, x0 and options
+    (compressor: scaled sign, the default, or Top-K)."""
     from . import binding as sb
 
     def make(begin, count):
-        return sb.Sae(num_workers, tensor_sizes, x0, compressor=sb.SIGN, shard=(begin, count), **kw)
+        return sb.Sae(num_workers, tensor_sizes, x0, shard=(begin, count), **kw)
 
     return ShardedRun(num_workers, make, group=group, barrier=barrier, allreduce_average=allreduce_average)

@@ -67,8 +67,9 @@ def test_random_sharded_configuration(case):
     d = int(np.sum(sizes))
     scales = synth.tensor_scales(c["seed"], len(sizes), -4.0, -1.0)
     x0 = synth.x0_numpy(c["seed"], d)
-    kw = dict(compressor=so.SIGN, server_compress=c["dc"], mode=c["mode"], avg_period=c["p"], momentum=c["mu"],
-              weight_decay=c["lam"])
+    comp = so.TOPK if case % 3 == 2 else so.SIGN
+    kw = dict(compressor=comp, server_compress=c["dc"], mode=c["mode"], avg_period=c["p"], momentum=c["mu"],
+              weight_decay=c["lam"], topk_num=1, topk_den=c["den"])
     orc = so.Oracle(K, sizes, x0, threads=4, **kw)
     ranges = [worker_range(K, world, r) for r in range(world)]
     shards = [sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), shard=rg, **kw) for rg in ranges]

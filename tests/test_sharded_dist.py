@@ -24,9 +24,9 @@ class Fake:
     def __init__(self, begin, count):
         self.begin, self.count, self.attached = begin, count, []
     def shard_export(self):
-        return struct.pack("<ii", self.begin, self.count) + bytes(504)
+        return struct.pack("<ii", self.begin, self.count) + bytes(1016)
     def shard_attach(self, blob):
-        assert len(blob) == 512
+        assert len(blob) == 1024
         self.attached.append(struct.unpack("<ii", blob[:8]))
     def step_begin(self, g, lr): log.append(("begin", lr))
     def step_end(self): log.append(("end",))

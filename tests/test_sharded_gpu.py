@@ -84,7 +84,7 @@ def test_sharded_handle_checks_its_arguments():
     d = int(np.sum(SIZES))
     x0 = torch.zeros(d, device="cuda")
     with pytest.raises(sb.SaeError):
-        sb.Sae(4, SIZES, x0, compressor=so.TOPK, shard=(0, 2))          # scaled sign only
+        sb.Sae(4, SIZES, x0, compressor=so.IDENTITY, shard=(0, 2))      # the identity compressor is not sharded
     with pytest.raises(sb.SaeError):
         sb.Sae(4, SIZES, x0, shard=(3, 2))                               # rows beyond K
     a = sb.Sae(4, SIZES, x0, shard=(0, 2))
@@ -255,5 +255,88 @@ def test_error_averaging_by_allreduce(world):
                 # a mean of K terms of mixed sign: a few roundings of the largest term, absolute
                 exp_e = orc.get(orc.E, b)
                 np.testing.assert_allclose(got_e, exp_e, rtol=2e-6, atol=2.0 ** -22 * float(np.abs(exp_e).max()))
+    for s in shards:
+        s.close()
+
+
+
+def compare_topk_shard(shard, begin, orc, dc, tag):
+    cpu = lambda t: t.cpu().numpy()
+    from parity_util import mask_words
+    shard.sync()
+    assert_same(f"{tag} x", cpu(shard.get_params()), orc.get(orc.X))
+    assert_same(f"{tag} e_srv", cpu(shard.get_state(sb.STATE_SERVER_ERROR)), orc.get(orc.E_SRV))
+    for kl in range(shard.K):
+        k = begin + kl
+        if shard.keeps_momentum:
+            assert_same(f"{tag} m[{k}]", cpu(shard.get_state(sb.STATE_MOMENTUM, kl)), orc.get(orc.M, k))
+        assert_same(f"{tag} e[{k}]", cpu(shard.get_state(sb.STATE_WORKER_ERROR, kl)), orc.get(orc.E, k))
+        assert_same(f"{tag} tau[{k}]", cpu(shard.get_state(sb.STATE_WORKER_TAU, kl)).view(np.uint32).astype(np.uint64),
+                    orc.tau(k))
+    if dc:
+        assert_same(f"{tag} tau_srv", cpu(shard.get_state(sb.STATE_SERVER_TAU)).view(np.uint32).astype(np.uint64),
+                    orc.tau(-1))
+        assert_same(f"{tag} mask_srv", cpu(shard.get_state(sb.STATE_SERVER_MASK)).view(np.uint32),
+                    mask_words(orc.get(orc.C_DELTA_SRV) != 0, orc.sizes))
+
+
+@pytest.mark.parametrize("K,world", [(4, 2), (3, 2), (5, 3), (2, 1)])
+@pytest.mark.parametrize("p", [0, 1, 3])
+@pytest.mark.parametrize("dc,mode,lam,den", [(1, so.SAEF, 0.0, 100), (0, so.EF, 1e-4, 10)])
+def test_topk_shards_in_one_process_match_the_oracle(K, world, p, dc, mode, lam, den):
+    """Top-K messages as lists of selected entries, added in k order by every shard."""
+    import torch
+    d = int(np.sum(SIZES))
+    seed = 13
+    scales = synth.tensor_scales(seed, len(SIZES), -4.0, -1.0)
+    x0 = synth.x0_numpy(seed, d)
+    kw = dict(compressor=so.TOPK, server_compress=dc, mode=mode, avg_period=p, momentum=0.9, weight_decay=lam,
+              topk_num=1, topk_den=den)
+    orc = so.Oracle(K, SIZES, x0, threads=4, **kw)
+    ranges = [worker_range(K, world, r) for r in range(world)]
+    shards = [sb.Sae(K, SIZES, torch.from_numpy(x0).cuda(), shard=rg, **kw) for rg in ranges]
+    blobs = [s.shard_export() for s in shards]
+    for s in shards:
+        for b in blobs:
+            s.shard_attach(b)
+    for t in range(7):
+        g = synth.grads_numpy(seed, t, K, SIZES, scales, 66, 100.0)
+        orc.step(g, 0.1)
+        gd = torch.from_numpy(g).cuda().view(K, d)
+        for s, (b, c) in zip(shards, ranges):
+            s.step_begin(gd[b:b + c].contiguous(), 0.1)
+        for s in shards:
+            s.step_end()
+        for s, (b, c) in zip(shards, ranges):
+            compare_topk_shard(s, b, orc, dc, tag=f"topk K={K} world={world} p={p} shard@{b} t={t + 1}")
+    for s in shards:
+        s.close()
+
+
+def test_topk_shards_with_overflowing_lists():
+    """Gradients of one constant magnitude: every entry ties the k-th magnitude, so all n are selected and the
+    lists overflow their regions; the readers then take that worker's stored row with its threshold."""
+    import torch
+    sizes = [20000, 64, 9000]
+    K, d = 3, sum(sizes)
+    x0 = np.zeros(d, dtype=np.float32)
+    kw = dict(compressor=so.TOPK, avg_period=2, momentum=0.0, topk_num=1, topk_den=100)
+    orc = so.Oracle(K, sizes, x0, threads=4, **kw)
+    ranges = [(0, 2), (2, 1)]
+    shards = [sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), shard=rg, **kw) for rg in ranges]
+    for s in shards:
+        for blob in [q.shard_export() for q in shards]:
+            s.shard_attach(blob)
+    rng = np.random.default_rng(3)
+    for t in range(4):
+        g = (rng.integers(0, 2, size=(K, d)).astype(np.float32) * 2 - 1) * np.float32(0.25)
+        orc.step(g.ravel(), 0.5)
+        gd = torch.from_numpy(g).cuda()
+        for s, (b, c) in zip(shards, ranges):
+            s.step_begin(gd[b:b + c].contiguous(), 0.5)
+        for s in shards:
+            s.step_end()
+        for s, (b, c) in zip(shards, ranges):
+            compare_topk_shard(s, b, orc, 1, tag=f"overflow t={t + 1} shard@{b}")
     for s in shards:
         s.close()
