@@ -917,7 +917,9 @@ int sae_shard_export(sae_handle* h, void* blob_host, size_t bytes) {
   b.T = h->P.T; b.nwords = h->P.nwords; b.dpad = h->P.dpad;
   b.compressor = h->cfg.compressor; b.cand_stride = h->cand_stride;
   b.raw[0] = h->words; b.raw[1] = h->scale[0]; b.raw[2] = h->scale[1]; b.raw[3] = h->D;
-  b.raw[4] = h->msg_entries; b.raw[5] = h->msg_count; b.raw[6] = h->tau[0]; b.raw[7] = h->tau[1];
+  if (h->cfg.compressor == SAE_COMPRESSOR_TOPK) {
+    b.raw[4] = h->msg_entries; b.raw[5] = h->msg_count; b.raw[6] = h->tau[0]; b.raw[7] = h->tau[1];
+  }
   for (int q = 0; q < kShardBufs; ++q)
     if (b.raw[q]) SAE_CUDA(h, cudaIpcGetMemHandle(&b.ipc[q], b.raw[q]));
   memset(blob_host, 0, SAE_SHARD_BLOB_BYTES);
