@@ -6,6 +6,8 @@ import sys
 
 import pytest
 
+from conftest import free_port
+
 from paper_2008_05823_b200.sharded import worker_range
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -72,7 +74,7 @@ def test_rank_logic_world_size_2(tmp_path):
     script.write_text(WORKER.format(root=ROOT))
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="2")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
-           "127.0.0.1", "--master-port", "29751", str(script)]
+           "127.0.0.1", "--master-port", free_port(), str(script)]
     res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
     assert res.returncode == 0, res.stderr[-3000:]
     assert res.stdout.count("OK") == 2

@@ -13,6 +13,8 @@ import sys
 import numpy as np
 import pytest
 
+from conftest import free_port
+
 from oracle import sae_oracle as so
 from paper_2008_05823_b200 import binding as sb
 from paper_2008_05823_b200 import synth
@@ -109,7 +111,7 @@ def test_sharded_handle_checks_its_arguments():
 def test_two_processes_on_one_gpu_through_ipc():
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="2")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2", "--master-addr",
-           "127.0.0.1", "--master-port", "29741", os.path.join(ROOT, "tests", "shard_ipc_worker.py")]
+           "127.0.0.1", "--master-port", free_port(), os.path.join(ROOT, "tests", "shard_ipc_worker.py")]
     res = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     assert res.returncode == 0, (res.stdout[-2000:], res.stderr[-3000:])
     assert res.stdout.count("SHARD_OK") == 2, res.stdout[-2000:]
@@ -170,7 +172,7 @@ sys.path.insert(0, {root!r}); sys.path.insert(0, os.path.join({root!r}, "tests")
 from oracle import sae_oracle as so
 from paper_2008_05823_b200 import synth
 from paper_2008_05823_b200.sharded import sharded_sae
-os.environ.setdefault("MASTER_ADDR", "127.0.0.1"); os.environ.setdefault("MASTER_PORT", "29761")
+os.environ.setdefault("MASTER_ADDR", "127.0.0.1"); os.environ.setdefault("MASTER_PORT", {port!r})
 torch.cuda.set_device(0)
 dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
 sizes = [33, 4096, 5000]
@@ -197,7 +199,7 @@ def test_stream_ordered_barrier_with_the_nccl_backend(tmp_path):
     """World size 1 (this box has one GPU): the NCCL code path of the rank logic -- all-gather of the row
     descriptions, the one-element all-reduce as the stream-ordered barrier, orderly shutdown."""
     script = tmp_path / "nccl_worker.py"
-    script.write_text(NCCL_WORKER.format(root=ROOT))
+    script.write_text(NCCL_WORKER.format(root=ROOT, port=free_port()))
     res = subprocess.run([sys.executable, str(script)], cwd=ROOT, capture_output=True, text=True, timeout=600,
                          env=dict(os.environ, OMP_NUM_THREADS="2"))
     assert res.returncode == 0, (res.stdout[-1000:], res.stderr[-3000:])
