@@ -27,8 +27,8 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after, srv_pending; const float* grads; float lr, eta_prev; };
-struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after; uint64_t stamp; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot; const float* grads; float lr, eta_prev; };
+struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after; uint64_t stamp; };
 
 }  // namespace
 
@@ -49,7 +49,12 @@ struct sae_handle {
   float *scale[2], *scale_srv;
   u32 *tau[2], *tau_srv;
   L1Record *recs, *recs_srv;
-  L1Record* recs_srv_alt;  // second server-record buffer (inline_fin: the two alternate with the step parity)
+  // inline_fin: the worker records alternate between two buffers with the step parity and the server records
+  // rotate through this step's, the previous step's (still needed while its server lines are pending) and
+  // the one the server pass clears for the next step -- four buffers rather than three, so that the rotation
+  // has a period that divides the usual gradient-ring lengths and few distinct step graphs exist
+  L1Record *recs_alt, *recs_srv_alt, *recs_srv_alt2, *recs_srv_alt3;
+  int rot;
   int srv_pending;         // the last step's server lines (e = Delta - C(Delta), x -= C(Delta)) are still owed:
                            // e_srv holds Delta, the server records hold its L1 sum; the next server pass
                            // (or flush_server, before anything reads x or e) carries them out
@@ -178,7 +183,7 @@ cudaError_t dalloc(T** p, size_t count) {
 void free_all(sae_handle* h) {
   void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->ebar_alt, h->m, h->D, h->etmp,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
-                  h->tau_srv, h->recs, h->recs_srv, h->recs_srv_alt, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
+                  h->tau_srv, h->recs, h->recs_alt, h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
   for (void* p : ptrs) if (p) cudaFree(p);
@@ -241,6 +246,10 @@ int flush_server(sae_handle* h) {
   ApplyArgs aa;
   memset(&aa, 0, sizeof(aa));
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
+  if (h->inline_fin) {      // the last step accumulated into the buffer before the current rotation index
+    L1Record* rs[4] = {h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3};
+    aa.recs_srv = rs[(h->rot + 3) % 4];
+  }
   aa.tau_srv = h->tau_srv; aa.mask_srv = h->mask_srv;
   const bool dcs = h->cfg.server_compress != 0;
   if (h->cfg.compressor == SAE_COMPRESSOR_TOPK) {
@@ -373,18 +382,21 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   ServerArgs sa;
   memset(&sa, 0, sizeof(sa));
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
-  // inline_fin: step t accumulates the server's L1 into one buffer while the apply kernel clears the other
-  L1Record* const recs_srv_now = (h->inline_fin && cur) ? h->recs_srv_alt : h->recs_srv;
-  L1Record* const recs_srv_next = (h->inline_fin && !cur) ? h->recs_srv_alt : h->recs_srv;
+  // inline_fin: rotating record buffers (see the handle)
+  L1Record* rs3[4] = {h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3};
+  L1Record* const recs_now = (h->inline_fin && cur) ? h->recs_alt : h->recs;
+  L1Record* const recs_other = (h->inline_fin && !cur) ? h->recs_alt : h->recs;
+  L1Record* const recs_srv_now = h->inline_fin ? rs3[h->rot] : h->recs_srv;
+  wa.recs = recs_now;
   sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = recs_srv_now; sa.status = h->status;
-  sa.word_rows = nullptr; sa.scale_rows = nullptr; sa.recs = h->recs; sa.scale_out = h->scale[cur];
+  sa.word_rows = nullptr; sa.scale_rows = nullptr; sa.recs = recs_now; sa.scale_out = h->scale[cur];
+  sa.recs_clear = recs_other; sa.recs_srv_clear = rs3[(h->rot + 1) % 4]; sa.recs_srv_prev = rs3[(h->rot + 3) % 4];
   sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0; sa.ebar = ebar_now(h);
   sa.m = h->m; sa.ebar_in = ebar_now(h); sa.eta = lr;
   ApplyArgs aa;
   memset(&aa, 0, sizeof(aa));
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = ebar_now(h); aa.m = h->m; aa.D = h->D;
   aa.scale_cur = h->scale[cur]; aa.scale_srv = h->scale_srv; aa.recs_srv = recs_srv_now; aa.tau_cur = h->tau[cur];
-  aa.recs_clear = h->inline_fin ? h->recs : nullptr; aa.recs_srv_clear = recs_srv_next;
   aa.tau_srv = h->tau_srv;
   aa.mask_srv = h->mask_srv; aa.eta = lr;
 
@@ -399,7 +411,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (pending_in) {
       FusedArgs fa;
       fa.g = grads; fa.m = h->m; fa.ebar = ebar_now(h); fa.x = h->x; fa.scale_prev = h->scale[h->last];
-      fa.words = h->words; fa.recs = h->recs; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
+      fa.words = h->words; fa.recs = recs_now; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
       launch_fused(h, sp, fa);
     } else if (h->esrc == ESRC_UNIFORM) {
       if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
@@ -409,7 +421,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     }
     // The server lines of this step can be left to the next step's server pass when nothing in between
     // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
-    const bool lazy_ok = SAE_LAZY_SERVER && !h->inline_fin && !sp.wd;
+    const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
     if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
     const bool pending = h->srv_pending != 0;
     if (!h->inline_fin)
@@ -420,8 +432,12 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
     const int nblk = (P.ntiles + tpb - 1) / tpb;
     if (h->inline_fin) {
-      if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true>), nblk, P, sa, tpb);
+      if (pending) {
+        if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true, true>), nblk, P, sa, tpb);
+        else LAUNCH(h, S_SERVER, (k_server_sign<false, false, true, true>), nblk, P, sa, tpb);
+      } else if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true>), nblk, P, sa, tpb);
       else LAUNCH(h, S_SERVER, (k_server_sign<false, false, true>), nblk, P, sa, tpb);
+      h->rot = (h->rot + 1) % 4;
     } else if (pending) {
       if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, true>), nblk, P, sa, tpb);
       else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, true>), nblk, P, sa, tpb);
@@ -502,16 +518,17 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   if (!usable) return do_step_direct(h, grads, lr);
 
   StepGraphKey key;
-  key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending;
+  key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending; key.rot = h->rot;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.srv_pending == key.srv_pending && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
-      h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->eta_prev = lr; h->t += 1;
+      h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->rot = e.rot_after;
+      h->eta_prev = lr; h->t += 1;
       e.stamp = ++h->graph_clock;
       h->graph_misses = 0;
       return SAE_OK;
@@ -532,7 +549,8 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   }
   StepGraph e;
   e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
-  e.esrc_after = h->esrc; e.last_after = h->last; e.pending_after = h->srv_pending; e.stamp = ++h->graph_clock;
+  e.esrc_after = h->esrc; e.last_after = h->last; e.pending_after = h->srv_pending; e.rot_after = h->rot;
+  e.stamp = ++h->graph_clock;
   ce = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
   if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); return SAE_ERR_CUDA; }
@@ -707,7 +725,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->recs, sign ? KT : 0); ALLOC0(h->recs_srv, sign ? T : 0);
   // latency-bound sizes (the whole K x d state fits L2 several times over): one launch fewer per step
   h->inline_fin = (sign && !shard && (long long)K * dpad <= (1ll << 24)) ? 1 : 0;
-  if (h->inline_fin) ALLOC0(h->recs_srv_alt, T);
+  if (h->inline_fin) {
+    ALLOC0(h->recs_srv_alt, T); ALLOC0(h->recs_srv_alt2, T); ALLOC0(h->recs_srv_alt3, T); ALLOC0(h->recs_alt, KT);
+  }
   ALLOC0(h->hist, topk ? KT * HIST_BINS : 0);
   ALLOC0(h->sel, topk ? KT : 0);
   std::vector<long long> cand_off(T, 0);
@@ -1190,6 +1210,10 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
     SAE_CUDA(h, cudaMemsetAsync(h->recs, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
     SAE_CUDA(h, cudaMemsetAsync(h->recs_srv, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
     SAE_CUDA(h, cudaMemsetAsync(h->recs_srv_alt, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
+    SAE_CUDA(h, cudaMemsetAsync(h->recs_srv_alt2, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
+    SAE_CUDA(h, cudaMemsetAsync(h->recs_srv_alt3, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));
+    SAE_CUDA(h, cudaMemsetAsync(h->recs_alt, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
+    h->rot = 0;
   }
   return SAE_OK;
 }

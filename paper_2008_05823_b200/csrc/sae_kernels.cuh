@@ -79,6 +79,9 @@ struct ServerArgs {
   // small problems: the scales are formed here from the workers' exact L1 records (no separate launch)
   const L1Record* recs;            // [K][T]
   float* scale_out;                // [K][T] this step's scales, written by the block that holds a tensor's first tile
+  L1Record* recs_clear;            // [K][T] the other worker-record buffer: cleared here for the next worker pass
+  L1Record* recs_srv_clear;        // [T] the server-record buffer the next step accumulates into: cleared here
+  const L1Record* recs_srv_prev;   // [T] the previous step's server records (LAZY: its server scale comes from them)
   // deferred server update of the previous step (LAZY): e_srv still holds that step's Delta and x is not yet
   // re-updated; both are brought up to date here, element by element, before this step's Delta is formed
   float* x;                        // [dpad]
@@ -119,7 +122,9 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
 }
 
 // FIN (small, latency-bound problems): the worker scales are not read but formed here from the exact L1
-// records, which saves the launch of k_finalize_scales; the records are then cleared by k_apply.
+// records, which saves the launch of k_finalize_scales.  The record buffers rotate (two for the workers,
+// three for the server) so that this pass can also clear the ones the next step accumulates into: nobody
+// reads those any more, and nothing else would clear them.
 // LAZY: the previous step left its server lines pending (e = Delta - C(Delta), x = x - C(Delta): the work of
 // k_apply); they are carried out here on the fly -- the same two subtractions per parameter -- so that the
 // server error and the parameters make one trip through memory per step instead of two.  This pass has
@@ -148,12 +153,28 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
           const L1Record r = A.recs[(long long)k * P.T + ti.j];
           const float s = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
           s_k[k] = s;
-          if (ti.t0 == 0) A.scale_out[(long long)k * P.T + ti.j] = s;
+          if (ti.t0 == 0) {
+            A.scale_out[(long long)k * P.T + ti.j] = s;
+            L1Record* c = A.recs_clear + (long long)k * P.T + ti.j;
+            c->limb[0] = 0; c->limb[1] = 0; c->limb[2] = 0;
+          }
         } else {
           s_k[k] = TABLE ? A.scale_rows[k][ti.j] : A.scale_cur[(long long)k * P.T + ti.j];
         }
       }
-      if (LAZY && DC && tid == 0) sh_s_old = A.scale_srv_prev[ti.j];
+      if (FIN && tid == 0 && ti.t0 == 0) {
+        L1Record* c = A.recs_srv_clear + ti.j;
+        c->limb[0] = 0; c->limb[1] = 0; c->limb[2] = 0;
+      }
+      if (LAZY && DC && tid == 0) {
+        if (FIN) {
+          const L1Record r = A.recs_srv_prev[ti.j];
+          sh_s_old = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
+          if (ti.t0 == 0) A.scale_srv[ti.j] = sh_s_old;
+        } else {
+          sh_s_old = A.scale_srv_prev[ti.j];
+        }
+      }
       __syncthreads();
       cur_j = ti.j;
     }
@@ -489,9 +510,7 @@ struct ApplyArgs {
   const u32* tau_cur;      // [K][T]
   const u32* tau_srv;      // [T]
   u32* mask_srv;           // [nwords] Top-K: server selection of this step
-  // small problems (no k_finalize_scales launch): records to clear once the server pass has read them
-  L1Record* recs_clear;      // [K][T] the workers' records, or null
-  L1Record* recs_srv_clear;  // [T] the server records the NEXT step accumulates into (the other of two buffers)
+
   float eta;
 };
 
@@ -530,13 +549,6 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
       if (COMP == 2) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
     }
     __syncthreads();
-  }
-  if (A.recs_clear && ti.t0 == 0) {
-    for (int k = tid; k < P.K; k += THREADS) {
-      L1Record* r = A.recs_clear + (long long)k * P.T + ti.j;
-      r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0;
-    }
-    if (tid == 0) { L1Record* r = A.recs_srv_clear + ti.j; r->limb[0] = 0; r->limb[1] = 0; r->limb[2] = 0; }
   }
   __shared__ float sh_s_srv;
   if (SRV == 1) {
