@@ -278,4 +278,45 @@ __device__ __forceinline__ u32 pack_row4(bool p0, bool p1, bool p2, bool p3) {
   return w;
 }
 
+// ---- mbarrier / bulk-copy (TMA) primitives ----------------------------------------------------------
+// Every wait on an mbarrier is bounded: after WAIT_LIMIT polls the waiter gives up and the caller raises
+// STATUS_TIMEOUT in the handle's status word.
+constexpr u32 WAIT_LIMIT = 1u << 24;
+constexpr u32 STATUS_TIMEOUT = 2u;
+
+__device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(u64* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(u64* bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the completion of the phase with the given parity; false = gave up.
+__device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity) {
+  const u32 addr = smem_u32(bar);
+  for (u32 it = 0; it < WAIT_LIMIT; ++it) {
+    u32 done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+// 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on `bar`.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 }  // namespace sae

@@ -105,6 +105,9 @@ struct ServerArgs {
 // pass; plain loads, also from a peer GPU's memory).
 constexpr int SRV_E = 16;   // consecutive parameters per thread; THREADS * SRV_E == TILE
 constexpr int SRV_B = 8;    // workers per batch of word loads
+#ifndef SAE_K3_STAGE
+#define SAE_K3_STAGE 1
+#endif
 static_assert(THREADS * SRV_E == TILE, "one pass of the block covers one tile");
 
 __device__ __forceinline__ u64 pack2(u32 lo, u32 hi) {
@@ -129,12 +132,24 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
 // k_apply); they are carried out here on the fly -- the same two subtractions per parameter -- so that the
 // server error and the parameters make one trip through memory per step instead of two.  This pass has
 // the memory bandwidth to spare (it is bound by instruction issue).
+// Staging (all but FIN): a full tile's server error (LAZY: and parameters) is fetched by one bulk
+// asynchronous copy (TMA) into shared memory when the block reaches the tile and is first read after the
+// worker loop, so that its memory latency passes under the loop without holding registers for it.
 template <bool DC, bool TABLE = false, bool FIN = false, bool LAZY = false>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
   __shared__ float sh_s_old;
   __shared__ const u32* s_row[TABLE ? MAX_WORKERS : 1];
+  constexpr bool STAGE = SAE_K3_STAGE && !FIN;
+  __shared__ alignas(128) float s_e[STAGE ? TILE : 4];
+  __shared__ alignas(128) float s_x[(STAGE && LAZY) ? TILE : 4];
+  __shared__ alignas(8) u64 s_bar;
+  u32 phase = 0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (STAGE && tid == 0) {
+    mbar_init(&s_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");   // (made visible by the first barrier below)
+  }
   if (TABLE) {
     for (int k = tid; k < P.K; k += THREADS) s_row[k] = A.word_rows[k];     // visible after the barrier below
   }
@@ -186,6 +201,14 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
     u32* wsp = A.words_srv + (pbase >> 5);
 
     if (ti.cnt == TILE) {
+      if constexpr (STAGE) {
+        __syncthreads();                          // nobody still reads the previous tile's staged rows
+        if (tid == 0) {
+          mbar_arrive_expect_tx(&s_bar, (LAZY ? 2u : 1u) * TILE * (u32)sizeof(float));
+          bulk_load(s_e, ep, TILE * (u32)sizeof(float), &s_bar);
+          if (LAZY) bulk_load(s_x, xp, TILE * (u32)sizeof(float), &s_bar);
+        }
+      }
       const int i = tid * SRV_E;
       const int wi = i >> 5, sh = (32 - SRV_E) - (i & 31);   // this thread's bits go to the top of the word
       u64 a2[SRV_E / 2];
@@ -194,8 +217,8 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
       // Single-way: the server error is fetched ahead of the worker loop, so that its latency hides under
       // the loop.  (Double-way has enough independent work after the loop; fetching early there only
       // costs registers.)
-      float4 ev[DC ? 1 : SRV_E / 4];
-      if constexpr (!DC) {
+      float4 ev[(DC || STAGE) ? 1 : SRV_E / 4];
+      if constexpr (!DC && !STAGE) {
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) ev[q] = ld4(ep + i + 4 * q);
       }
@@ -230,6 +253,13 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
           }
         }
       }
+      if constexpr (STAGE) {
+        if (!mbar_wait(&s_bar, phase)) {           // gave up: flag it and leave (the whole block does)
+          if (tid == 0) atomicOr(A.status, STATUS_TIMEOUT);
+          return;
+        }
+        phase ^= 1u;
+      }
       u32 bits = 0;
 #pragma unroll
       for (int q = 0; q < SRV_E / 4; ++q) {
@@ -237,10 +267,12 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         unpack2(a2[2 * q], a0, a1);
         unpack2(a2[2 * q + 1], a3, a4);
         float4 e;
-        if constexpr (DC) e = ld4(ep + i + 4 * q); else e = ev[q];
+        if constexpr (STAGE) e = ld4(s_e + i + 4 * q);
+        else if constexpr (DC) e = ld4(ep + i + 4 * q);
+        else e = ev[q];
         if constexpr (LAZY) {
           // e holds the previous step's Delta: C(Delta) is its scaled sign (double-way) or Delta itself
-          float4 xv = ld4(xp + i + 4 * q);
+          float4 xv = STAGE ? ld4(s_x + i + 4 * q) : ld4(xp + i + 4 * q);
           float4 cs;
           cs.x = DC ? sign_code(e.x, s_old) : e.x; cs.y = DC ? sign_code(e.y, s_old) : e.y;
           cs.z = DC ? sign_code(e.z, s_old) : e.z; cs.w = DC ? sign_code(e.w, s_old) : e.w;

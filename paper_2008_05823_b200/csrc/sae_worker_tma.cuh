@@ -40,8 +40,6 @@ constexpr int WT_SLICE = TILE / WT_CONSUMER_WARPS;          // elements of a til
 constexpr int WT_SLICE_ITERS = WT_SLICE / 128;              // float4 iterations per lane (2)
 constexpr int WT_SLICE_ROWS = WT_SLICE / 32;                // scalar rows per warp (8)
 static_assert(WT_SLICE % 128 == 0, "a consumer warp owns whole 128-element rows");
-constexpr u32 WAIT_LIMIT = 1u << 24;
-constexpr u32 STATUS_TIMEOUT = 2u;
 
 struct WtItem {          // description of one work item, written by the producer
   long long gofs;        // index of the tile's first gradient element in g
@@ -60,41 +58,6 @@ struct WtSmem {
   WtItem item[WT_STAGES];
   u32 cstage[WT_CONSUMER_WARPS][CAND_STAGE];   // Top-K: per-warp staging of candidate keys
 };
-
-__device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(u64* bar, u32 count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(u64* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(u64* bar, u32 bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Bounded wait for the completion of the phase with the given parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity) {
-  const u32 addr = smem_u32(bar);
-  for (u32 it = 0; it < WAIT_LIMIT; ++it) {
-    u32 done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(addr), "r"(parity)
-        : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-// 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on `bar`.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
 
 // Tile-table lookup of work item w (cnt = 0 marks "no such item").
 template <int ESRC, bool TOPK>
