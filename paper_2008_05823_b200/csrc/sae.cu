@@ -261,10 +261,9 @@ int flush_server(sae_handle* h) {
   return check_launch(h);
 }
 
-constexpr size_t kWorkerSmem = sizeof(WtSmem) + 128;
-
 template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK, bool MU0 = false>
 void launch_worker_wd(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
+  constexpr size_t kWorkerSmem = sizeof(WtSmemT<wt_stages(WRITE_D)>) + 128;
   static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
   if (configured_device != h->device) {
     cudaFuncSetAttribute(k_worker_tma<ESRC, SIGN, WRITE_D, WD, TOPK, MU0>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -23,9 +23,6 @@
 
 namespace sae {
 
-#ifndef SAE_WT_STAGES
-#define SAE_WT_STAGES 3
-#endif
 #ifndef SAE_WT_BLOCKS_PER_SM
 #define SAE_WT_BLOCKS_PER_SM 1
 #endif
@@ -35,7 +32,9 @@ namespace sae {
 #endif
 constexpr int WT_CONSUMER_WARPS = SAE_WT_CONSUMER_WARPS;
 constexpr int WT_THREADS = WT_CONSUMER_WARPS * 32 + 32;     // + one producer warp
-constexpr int WT_STAGES = SAE_WT_STAGES;
+// Ring depth: three stages of 48 KB when the pass also writes the model differences (20 bytes per element:
+// a fourth stage measured 1-2 % slower there), four when it moves 12 bytes per element (+2 %).
+__host__ __device__ constexpr int wt_stages(bool write_d) { return write_d ? 3 : 4; }
 constexpr int WT_SLICE = TILE / WT_CONSUMER_WARPS;          // elements of a tile owned by one consumer warp (256)
 constexpr int WT_SLICE_ITERS = WT_SLICE / 128;              // float4 iterations per lane (2)
 constexpr int WT_SLICE_ROWS = WT_SLICE / 32;                // scalar rows per warp (8)
@@ -51,11 +50,12 @@ struct WtItem {          // description of one work item, written by the produce
   u32 lo;               // Top-K: lower edge of the candidate window (NO_GUESS: collect nothing)
 };
 
-struct WtSmem {
-  alignas(128) float buf[WT_STAGES][3][TILE];   // [stage][g | m | e-source][element]
-  alignas(8) u64 full[WT_STAGES];
-  alignas(8) u64 empty[WT_STAGES];
-  WtItem item[WT_STAGES];
+template <int STAGES>
+struct WtSmemT {
+  alignas(128) float buf[STAGES][3][TILE];   // [stage][g | m | e-source][element]
+  alignas(8) u64 full[STAGES];
+  alignas(8) u64 empty[STAGES];
+  WtItem item[STAGES];
   u32 cstage[WT_CONSUMER_WARPS][CAND_STAGE];   // Top-K: per-warp staging of candidate keys
 };
 
@@ -86,6 +86,8 @@ template <int ESRC, bool SIGN, bool WRITE_D, bool WD, bool TOPK, bool MU0 = fals
 __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma(Plan P, StepParams sp, WorkerArgs A,
                                                                                   long long nitems) {
   extern __shared__ unsigned char smem_raw[];
+  constexpr int WT_STAGES = wt_stages(WRITE_D);
+  using WtSmem = WtSmemT<WT_STAGES>;
   WtSmem& S = *reinterpret_cast<WtSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
