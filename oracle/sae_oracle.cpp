@@ -21,6 +21,12 @@
 //   * weight decay: coupled L2, lambda * (point where the gradient is evaluated) added to the gradient;
 //   * Top-K: k = max(1, floor(n*num/den)); every entry whose magnitude ties the k-th largest is kept,
 //     exact zeros are never selected.
+//   * local steps (Section 2 names the extension -- "the local model difference will be communicated every
+//     several iterations" -- without spelling it out): with period H, iteration t communicates iff
+//     (t+1) mod H = 0; on the other iterations a worker only does its own lines, and its model difference
+//     keeps accumulating in the place of its error: e^(k) <- Delta^(k) = e^(k) + eta m^(k), nothing is sent,
+//     x and the server error stay.  The gradient point x - e^(k) of the step-ahead branch is then the
+//     worker's local model one step ahead.  Step-ahead branch without error averaging only.
 //
 // Threads: `threads` > 1 only distributes independent units (whole (worker, tensor) pairs for the
 // compressor, single elements for the elementwise loops); each unit is still computed sequentially,
@@ -133,6 +139,7 @@ void compress(int compressor, const R* v, int64_t n, uint32_t num, uint32_t den,
 template <class R>
 struct Oracle {
   int K, T, compressor, server_compress, mode, avg_period, threads;
+  int local_steps = 1;                      // H: communicate when (t+1) mod H == 0
   R mu, lambda;
   uint32_t num, den;
   std::vector<int64_t> n, off;
@@ -168,6 +175,12 @@ struct Oracle {
         m[q] = fma_r(mu, m[q], ge);                                    // m_{t+1} = mu m_t + grad
         D[q] = fma_r(eta, m[q], e[q]);                                 // Delta = e_t + eta m_{t+1}
       }
+    }
+    if (local_steps > 1 && (t + 1) % local_steps != 0) {
+      // not a communication iteration: the model difference stays with the worker and keeps growing
+      e = D;
+      t = t + 1;
+      return;
     }
     // c^(k) = C(Delta^(k)) per tensor;  e^(k)_{t+1} = Delta^(k) - C(Delta^(k)).
     #pragma omp parallel for collapse(2) num_threads(threads) schedule(dynamic, 1)
@@ -277,6 +290,13 @@ extern "C" {
   void sao_step_##SUF(void* h, const R* g, double eta) { ((Oracle<R>*)h)->step(g, (R)eta); }         \
   int sao_get_##SUF(void* h, int which, int k, R* out) { return get_real<R>((Oracle<R>*)h, which, k, out); } \
   int64_t sao_iteration_##SUF(void* h) { return ((Oracle<R>*)h)->t; }                                \
+  /* local-step period H >= 1; only before the first step, step-ahead branch, no error averaging */   \
+  int sao_set_local_steps_##SUF(void* h, int H) {                                                    \
+    Oracle<R>* o = (Oracle<R>*)h;                                                                    \
+    if (H < 1 || o->t != 0 || (H > 1 && (o->mode != MODE_SAEF || o->avg_period != 0))) return -1;    \
+    o->local_steps = H;                                                                              \
+    return 0;                                                                                        \
+  }                                                                                                  \
   int sao_range_flag_##SUF(void* h) { return ((Oracle<R>*)h)->range ? 1 : 0; }                       \
   /* Top-K thresholds (keys) of the last step: k >= 0 worker k, k < 0 server; T entries. */          \
   void sao_get_tau_##SUF(void* h, int k, uint64_t* out) {                                            \

@@ -34,6 +34,7 @@ def lib():
             getattr(L, f"sao_iteration_{suf}").argtypes = [C.c_void_p]
             getattr(L, f"sao_iteration_{suf}").restype = C.c_int64
             getattr(L, f"sao_range_flag_{suf}").argtypes = [C.c_void_p]
+            getattr(L, f"sao_set_local_steps_{suf}").argtypes = [C.c_void_p, C.c_int]
             getattr(L, f"sao_get_tau_{suf}").argtypes = [C.c_void_p, C.c_int, C.c_void_p]
             getattr(L, f"sao_get_tau_{suf}").restype = None
             getattr(L, f"sao_compress_{suf}").argtypes = [
@@ -60,7 +61,7 @@ class Oracle:
 
     def __init__(self, num_workers, tensor_sizes, x0, compressor=SIGN, server_compress=1, mode=SAEF,
                  avg_period=0, momentum=0.9, weight_decay=0.0, topk_num=1, topk_den=100, threads=1,
-                 dtype=np.float32):
+                 dtype=np.float32, local_steps=1):
         self.dtype = np.dtype(dtype)
         self.suf = "f32" if self.dtype == np.float32 else "f64"
         self.K = int(num_workers)
@@ -75,6 +76,9 @@ class Oracle:
             float(weight_decay), topk_num, topk_den, threads, _ptr(x0))
         if not self.h:
             raise ValueError("oracle rejected the configuration")
+        self.local_steps = int(local_steps)
+        if getattr(lib(), f"sao_set_local_steps_{self.suf}")(self.h, self.local_steps) != 0:
+            raise ValueError("local steps need the step-ahead branch without error averaging")
 
     def __del__(self):
         try:

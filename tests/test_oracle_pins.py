@@ -500,3 +500,108 @@ def test_fixed_point_l1_random(n, scale_exp, seed):
         assert not rg and S == _exact_fixed_sum(v)
     else:
         assert rg
+
+
+# ------------------------------------------------------------------------------------------------
+# local steps (Section 2: the model difference communicated every H iterations)
+# ------------------------------------------------------------------------------------------------
+def quad_problem(d, seed):
+    """f_k(y) = 0.5 y'A_k y - b_k'y with A_k symmetric positive definite: gradient A_k y - b_k."""
+    rng = np.random.default_rng(seed)
+    Q = rng.standard_normal((d, d)) * 0.1
+    return Q @ Q.T + 0.5 * np.eye(d), rng.standard_normal(d)
+
+
+@pytest.mark.parametrize("comp", [SIGN, TOPK, IDENTITY])
+def test_local_steps_period_one_is_algorithm_1(comp):
+    """H = 1 communicates every iteration: bit for bit the run without local steps."""
+    K, sizes = 3, [9, 64, 130]
+    x0, gs = rand_sizes_grads(K, sizes, 5, np.float32)
+    a = Oracle(K, sizes, x0, compressor=comp, momentum=0.9, weight_decay=1e-3, topk_den=10)
+    b = Oracle(K, sizes, x0, compressor=comp, momentum=0.9, weight_decay=1e-3, topk_den=10, local_steps=1)
+    for g in gs:
+        a.step(g, 0.1); b.step(g, 0.1)
+    for w in (a.X, a.E_SRV):
+        np.testing.assert_array_equal(a.get(w), b.get(w))
+    np.testing.assert_array_equal(a.get_all(a.E), b.get_all(b.E))
+
+
+@pytest.mark.parametrize("H", [2, 3, 5])
+def test_local_steps_single_worker_identity_is_momentum_sgd(H):
+    """K = 1, C = identity: the gradient point y = x - e^(1) follows plain momentum SGD with weight decay
+    (m <- mu m + grad f(y) + lambda y, y <- y - eta m) whatever the period; x itself moves only when communicating."""
+    d, steps, mu, lr, lam = 12, 11, 0.9, 0.07, 1e-2
+    A, b = quad_problem(d, 3)
+    x0 = np.random.default_rng(5).standard_normal(d)
+    o = Oracle(1, [5, 7], x0, compressor=IDENTITY, momentum=mu, weight_decay=lam, dtype=np.float64, local_steps=H)
+    y, m = x0.copy(), np.zeros(d)
+    for t in range(steps):
+        pt = o.step_ahead(0)
+        np.testing.assert_allclose(pt, y, rtol=0, atol=1e-12)
+        x_before = o.get(o.X)
+        o.step((A @ pt - b)[None, :], lr)
+        m = mu * m + (A @ y - b + lam * y)           # coupled L2 at the point where the gradient is taken
+        y = y - lr * m
+        if (t + 1) % H:
+            np.testing.assert_array_equal(o.get(o.X), x_before)          # nothing was communicated
+        else:
+            np.testing.assert_allclose(o.get(o.X), y, rtol=0, atol=1e-12)   # identity: no error is left
+            assert np.all(o.get(o.E, 0) == 0)
+
+
+@pytest.mark.parametrize("H", [2, 4])
+def test_local_steps_identity_is_periodic_model_averaging(H):
+    """C = identity, K workers with different objectives: every worker runs H momentum steps on its own
+    copy of the model, then the copies are averaged (local SGD with periodic averaging, written out
+    independently in numpy)."""
+    K, d, rounds, mu, lr = 3, 10, 3, 0.8, 0.05
+    probs = [quad_problem(d, 10 + k) for k in range(K)]
+    x0 = np.random.default_rng(6).standard_normal(d)
+    o = Oracle(K, [4, 6], x0, compressor=IDENTITY, momentum=mu, dtype=np.float64, local_steps=H)
+    xs = [x0.copy() for _ in range(K)]
+    ms = [np.zeros(d) for _ in range(K)]
+    for r in range(rounds):
+        for h in range(H):
+            g = np.stack([probs[k][0] @ o.step_ahead(k) - probs[k][1] for k in range(K)])
+            o.step(g, lr)
+            for k in range(K):
+                ms[k] = mu * ms[k] + (probs[k][0] @ xs[k] - probs[k][1])
+                xs[k] = xs[k] - lr * ms[k]
+        avg = np.mean(xs, axis=0)
+        xs = [avg.copy() for _ in range(K)]
+        np.testing.assert_allclose(o.get(o.X), avg, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("comp", [SIGN, TOPK])
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("H", [2, 3])
+def test_local_steps_auxiliary_identity(comp, dc, H):
+    """Eq. 3 holds at every iteration, communicating or not: x~ = x - (e + mean_k e^(k)) moves by
+    -(eta/K) sum_k m^(k); a local iteration leaves x, the server error and the messages alone."""
+    K, sizes, steps = 3, [1, 7, 32, 65, 200], 10
+    x0, gs = rand_sizes_grads(K, sizes, steps, np.float64)
+    o = Oracle(K, sizes, x0, compressor=comp, server_compress=dc, momentum=0.9, weight_decay=1e-3, topk_den=10,
+               dtype=np.float64, local_steps=H)
+    xt = aux(o)
+    for t, g in enumerate(gs):
+        lr = 0.1 if t % 2 else 0.05
+        x_before, es_before, e_before = o.get(o.X), o.get(o.E_SRV), o.get_all(o.E)
+        o.step(g, lr)
+        m = o.get_all(o.M)
+        xt_new = aux(o)
+        np.testing.assert_allclose(xt_new, xt - lr * m.mean(axis=0), rtol=0, atol=1e-13)
+        xt = xt_new
+        if (t + 1) % H:
+            np.testing.assert_array_equal(o.get(o.X), x_before)
+            np.testing.assert_array_equal(o.get(o.E_SRV), es_before)
+            np.testing.assert_allclose(o.get_all(o.E), e_before + lr * m, rtol=0, atol=1e-15)
+        else:
+            np.testing.assert_array_equal(o.get(o.X), x_before - o.get(o.C_DELTA_SRV))
+
+
+def test_local_steps_rejects_ef_and_averaging():
+    x0 = np.zeros(12, np.float32)
+    with pytest.raises(ValueError):
+        Oracle(2, [5, 7], x0, mode=EF, local_steps=2)
+    with pytest.raises(ValueError):
+        Oracle(2, [5, 7], x0, avg_period=4, local_steps=2)
