@@ -335,6 +335,9 @@ def main():
     ap.add_argument("--topk-percent", type=float, default=None, help="Top-K sparsity in percent (Table 1: 1, 5, 10)")
     ap.add_argument("--block-size", type=int, default=0,
                     help="block-wise compression: cut every tensor into segments of this many elements")
+    ap.add_argument("--local-steps", type=int, default=1,
+                    help="communicate the model differences every H iterations (needs --avg-period 0); a step is "
+                         "still one iteration, so the figure averages H - 1 local iterations and one communicating one")
     ap.add_argument("--sharded", action="store_true",
                     help="sharded operation: the workers are split over the ranks (strong scaling of one job); "
                          "with one rank it times the same two-phase, table-driven path on one GPU")
@@ -415,7 +418,7 @@ def main():
     def make():
         return sb.Sae(K, w.tensor_sizes, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
                       avg_period=p, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
-                      topk_den=w.topk_den)
+                      topk_den=w.topk_den, local_steps=args.local_steps)
 
     # ---- device-resident throughput ------------------------------------------------------------------
     sae = make()
@@ -546,6 +549,7 @@ def main():
                            "mode": "saef" if w.mode == configs.SAEF else "ef",
                            "server_compress": "double-way" if w.server_compress else "single-way",
                            "topk": f"{w.topk_num}/{w.topk_den}" if w.compressor == configs.TOPK else None,
+                           "local_steps": args.local_steps,
                            "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
                            "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient set "
                                  f"(ring of {ring})"},

@@ -106,6 +106,23 @@ int sae_step(sae_handle *h, const float *grads, float lr);
  */
 int sae_step_host(sae_handle *h, const float *grads_host, float lr);
 
+/*
+ * Local steps (Section 2: Algorithm 1 "can be easily extended to local SGD, where the local model
+ * difference will be communicated every several (>1) iterations"; the paper does not spell the extension
+ * out, this is the reading built here).  With period H, iteration t communicates iff (t+1) mod H = 0 and is
+ * then exactly sae_step above.  On the other iterations only the worker lines run:
+ *   xh = x - e^(k);  m^(k) = mu m^(k) + (g^(k) + lambda xh);  e^(k) = e^(k) + lr m^(k)
+ * i.e. the model difference stays with the worker and keeps accumulating in the place of its error;
+ * nothing is compressed or sent, x and the server error do not change.  sae_get_step_ahead(k) = x - e^(k)
+ * is then worker k's local model one step ahead, the point of its next gradient, and
+ * SAE_STATE_WORKER_ERROR returns that running difference.  A local iteration is one pass over g, m^(k)
+ * and the stored difference (20 bytes per worker-element) and no server pass.
+ * period >= 1 (1 = Algorithm 1 as printed).  Only before the first step, in SAE_MODE_SAEF, with
+ * avg_period = 0 and not on a shard; otherwise SAE_ERR_INVALID_ARG.  Checkpoints carry the period and
+ * load only into a handle set to the same one.
+ */
+int sae_set_local_steps(sae_handle *h, int32_t period);
+
 /* Algorithm 1, "Output": x_t into out (device, d floats, caller layout). */
 int sae_get_params(sae_handle *h, float *out);
 /* Same into HOST memory (through a library-owned device buffer allocated by the first call);

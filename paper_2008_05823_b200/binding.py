@@ -26,7 +26,7 @@ EXPORTS = ["sae_init", "sae_step", "sae_step_host", "sae_get_params", "sae_get_p
            "sae_last_cuda_error", "sae_sign_compress_noalloc", "sae_noalloc_max_elements", "sae_state_bytes",
            "sae_save_state", "sae_load_state", "sae_get_mismatch", "sae_init_shard", "sae_shard_export",
            "sae_shard_attach", "sae_shard_detach", "sae_step_begin", "sae_step_end", "sae_shard_set_avg_mode", "sae_avg_due",
-           "sae_num_padded", "sae_avg_local_sum", "sae_avg_set"]
+           "sae_num_padded", "sae_avg_local_sum", "sae_avg_set", "sae_set_local_steps"]
 
 SHARD_BLOB_BYTES = 1024
 
@@ -91,6 +91,7 @@ def lib():
         L.sae_step_begin.argtypes = [vp, vp, f32]
         L.sae_step_end.argtypes = [vp]
         L.sae_shard_set_avg_mode.argtypes = [vp, i32]
+        L.sae_set_local_steps.argtypes = [vp, i32]
         L.sae_avg_due.argtypes = [vp]
         L.sae_num_padded.argtypes = [vp]
         L.sae_num_padded.restype = i64
@@ -116,7 +117,8 @@ class Sae:
     gradients are [num_local][d], and worker indices of the getters are local."""
 
     def __init__(self, num_workers, tensor_sizes, x0, compressor=SIGN, server_compress=1, mode=SAEF, avg_period=0,
-                 momentum=0.9, weight_decay=0.0, topk_num=1, topk_den=100, device=None, stream=None, shard=None):
+                 momentum=0.9, weight_decay=0.0, topk_num=1, topk_den=100, device=None, stream=None, shard=None,
+                 local_steps=1):
         import torch
         self.torch = torch
         if not (x0.is_cuda and x0.dtype == torch.float32 and x0.is_contiguous()):
@@ -143,8 +145,14 @@ class Sae:
                    "sae_init_shard")
             self.K = int(shard[1])          # rows held here: gradients are [K][d], getters take 0..K-1
         self.h = h
+        if local_steps != 1:
+            self.set_local_steps(local_steps)
         self.d = int(lib().sae_num_params(h))
         self.nwords = int(lib().sae_num_words(h))
+
+    def set_local_steps(self, period):
+        """sae_set_local_steps: the model differences are communicated every `period` iterations."""
+        _check(lib().sae_set_local_steps(self.h, int(period)), "sae_set_local_steps", self.h)
 
     def close(self):
         if getattr(self, "h", None):

@@ -27,7 +27,7 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot; const float* grads; float lr, eta_prev; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm; const float* grads; float lr, eta_prev; };
 struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after; uint64_t stamp; };
 
 }  // namespace
@@ -91,6 +91,7 @@ struct sae_handle {
   Plan P_all;                       // the plan with K = K_total (server pass, averaging)
   int attached;                     // workers whose message rows are known
   int mid_step;                     // sae_step_begin done, sae_step_end due
+  int local_steps;                  // H: iteration t communicates iff (t+1) mod H == 0 (1: every iteration)
   int avg_external;                 // the averaging sum is all-reduced by the caller instead of pulled in k order
   int avg_owed;                     // ... and is owed before the next sae_step_begin
   float lr_pending;
@@ -364,6 +365,9 @@ void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa) {
   }
 }
 
+// Does iteration t = h->t send the model differences?  (Every iteration unless local steps are set.)
+bool communicates(const sae_handle* h) { return h->local_steps <= 1 || (h->t + 1) % h->local_steps == 0; }
+
 int do_step_direct(sae_handle* h, const float* grads, float lr) {
   const sae_config& c = h->cfg;
   const Plan& P = h->P;
@@ -399,6 +403,21 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   aa.tau_srv = h->tau_srv;
   aa.mask_srv = h->mask_srv; aa.eta = lr;
 
+  if (!communicates(h)) {
+    // Local iteration (Section 2: the model difference is communicated every H iterations): the worker lines
+    // only.  The model difference keeps accumulating in D^(k), which from now on stands for e^(k) as it is.
+    switch (h->esrc) {
+      case ESRC_UNIFORM: launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa); break;
+      case ESRC_LAZY_SIGN: launch_worker<ESRC_LAZY_SIGN, false, true>(h, sp, wa); break;
+      case ESRC_LAZY_TOPK: launch_worker<ESRC_LAZY_TOPK, false, true>(h, sp, wa); break;
+      case ESRC_LOCAL_D: launch_worker<ESRC_LOCAL_D, false, true>(h, sp, wa); break;
+      default: return SAE_ERR_INVALID_ARG;
+    }
+    h->esrc = ESRC_LOCAL_D;
+    h->eta_prev = lr;
+    h->t += 1;
+    return check_launch(h);
+  }
   if (c.compressor == SAE_COMPRESSOR_SIGN) {
     // The model differences need not be stored when the previous error was uniform and the next
     // pre-step averages: the averaging pass recomputes them from m and ebar with the same fused op.
@@ -415,6 +434,8 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     } else if (h->esrc == ESRC_UNIFORM) {
       if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
       else launch_worker<ESRC_UNIFORM, true, false>(h, sp, wa);
+    } else if (h->esrc == ESRC_LOCAL_D) {
+      launch_worker<ESRC_LOCAL_D, true, true>(h, sp, wa);
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
@@ -465,6 +486,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (nod) { src.m = h->m; src.ebar = ebar_now(h); src.eta = lr; src.recompute = 1; }
     if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
     else if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
+    else if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true, true>(h, sp, wa);
     else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
     topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
     // the averaged error (if the pre-step averages) comes out of the same pass over D as the server's sum
@@ -489,7 +511,8 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
   } else {
     // identity: every error stays exactly zero, so e^(k) is the (all-zero) uniform vector forever
-    launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
+    if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true>(h, sp, wa);
+    else launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
     LAUNCH(h, S_SERVER, (k_server_dense<0, false>), P.ntiles, P, sa);
     launch_apply<0, 0>(h, AVG_NONE, aa);
     h->esrc = ESRC_UNIFORM;
@@ -518,12 +541,13 @@ int do_step(sae_handle* h, const float* grads, float lr) {
 
   StepGraphKey key;
   key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending; key.rot = h->rot;
+  key.comm = communicates(h) ? 1 : 0;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
       h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->rot = e.rot_after;
@@ -597,7 +621,7 @@ struct CkptHeader {
   int32_t esrc, last;
   float eta_prev;
   int32_t worker_begin, num_workers_total;     // which workers of how many this handle owns (sharded operation)
-  int32_t pad;
+  int32_t local_steps;                         // 0 in checkpoints written before local steps existed (= 1)
 };
 constexpr uint64_t kCkptMagic = 0x5341455F434B5032ull;   // "SAE_CKP2"
 
@@ -669,7 +693,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   h->cfg.tensor_sizes = h->sizes.data();
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
-  h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f;
+  h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f; h->local_steps = 1;
   h->graphs_enabled = 1; h->graph_misses = 0; h->graph_clock = 0;
   h->fused_ok = (!shard && cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
                  (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
@@ -1020,6 +1044,13 @@ int sae_shard_detach(sae_handle* h) {
   return SAE_OK;
 }
 
+int sae_set_local_steps(sae_handle* h, int32_t period) {
+  if (!h || period < 1 || h->t != 0 || h->shard) return SAE_ERR_INVALID_ARG;
+  if (period > 1 && (h->cfg.mode != SAE_MODE_SAEF || h->cfg.avg_period != 0)) return SAE_ERR_INVALID_ARG;
+  h->local_steps = period;
+  return SAE_OK;
+}
+
 int sae_shard_set_avg_mode(sae_handle* h, int32_t external_sum) {
   if (!h || !h->shard || h->mid_step || h->avg_owed) return SAE_ERR_INVALID_ARG;
   h->avg_external = external_sum ? 1 : 0;
@@ -1174,6 +1205,7 @@ int sae_save_state(sae_handle* h, void* out, size_t bytes) {
   hd.topk_num = h->cfg.topk_num; hd.topk_den = h->cfg.topk_den; hd.momentum = h->cfg.momentum;
   hd.weight_decay = h->cfg.weight_decay; hd.d = h->P.d; hd.t = h->t; hd.esrc = h->esrc; hd.last = h->last;
   hd.eta_prev = h->eta_prev; hd.worker_begin = h->k0; hd.num_workers_total = h->K_total;
+  hd.local_steps = h->local_steps;
   SAE_CUDA(h, cudaMemcpyAsync(out, &hd, sizeof(hd), cudaMemcpyHostToDevice, h->stream));
   SAE_CUDA(h, cudaStreamSynchronize(h->stream));        // hd lives on this stack frame
   char* q = (char*)out + 256;
@@ -1195,7 +1227,8 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
   if (hd.magic != kCkptMagic || hd.K != h->P.K || hd.T != h->P.T || hd.d != h->P.d || hd.compressor != c.compressor ||
       hd.server_compress != c.server_compress || hd.mode != c.mode || hd.avg_period != c.avg_period ||
       hd.topk_num != c.topk_num || hd.topk_den != c.topk_den || hd.momentum != c.momentum ||
-      hd.weight_decay != c.weight_decay || hd.worker_begin != h->k0 || hd.num_workers_total != h->K_total)
+      hd.weight_decay != c.weight_decay || hd.worker_begin != h->k0 || hd.num_workers_total != h->K_total ||
+      std::max(hd.local_steps, 1) != h->local_steps)
     return SAE_ERR_INVALID_ARG;                         // a checkpoint of a different configuration
   if (hd.esrc == ESRC_PENDING_AVG && !h->fused_ok) return SAE_ERR_INVALID_ARG;
   const char* q = (const char*)in + 256;

@@ -19,10 +19,12 @@ constexpr int ESRC_UNIFORM = 0;    // e^(k) = ebar for all k (after an averaging
 constexpr int ESRC_LAZY_SIGN = 1;  // e^(k) = D^(k) - C(D^(k)) with last step's scales, D^(k) = last Delta^(k)
 constexpr int ESRC_LAZY_TOPK = 2;  // same with last step's Top-K thresholds
 constexpr int ESRC_PENDING_AVG = 3;  // p = 1, scaled sign: e^(k) = mean_k(fma(eta_prev, m^(k), ebar) - C(.)), not yet formed
+constexpr int ESRC_LOCAL_D = 4;    // local steps: D^(k) is the running local model difference (the error plus the
+                                   // local updates not yet communicated) and takes the place of e^(k) as it is
 
 template <int ESRC>
 __device__ __forceinline__ float prev_error(float v, float sprev, u32 tprev) {
-  if (ESRC == ESRC_UNIFORM) return v;
+  if (ESRC == ESRC_UNIFORM || ESRC == ESRC_LOCAL_D) return v;
   if (ESRC == ESRC_LAZY_SIGN) return __fsub_rn(v, sign_code(v, sprev));
   return __fsub_rn(v, topk_selected(v, tprev) ? v : 0.0f);
 }
@@ -685,6 +687,7 @@ struct ExportArgs {
 __device__ __forceinline__ float current_error(const ExportArgs& A, const Plan& P, int j, long long p) {
   if (A.esrc == ESRC_UNIFORM) return A.ebar[p];
   const float v = A.D[(long long)A.k * P.dpad + p];
+  if (A.esrc == ESRC_LOCAL_D) return v;
   if (A.esrc == ESRC_LAZY_SIGN) return prev_error<ESRC_LAZY_SIGN>(v, A.scale_last[(long long)A.k * P.T + j], 0u);
   return prev_error<ESRC_LAZY_TOPK>(v, 0.0f, A.tau_last[(long long)A.k * P.T + j]);
 }
