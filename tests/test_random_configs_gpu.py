@@ -1,5 +1,5 @@
 """Seeded random configurations (worker count, tensor list, compressor, schedule, branch, momentum, weight
-decay, single/double-way, learning rates), unsharded and sharded, against the oracle: every combination the
+decay, single/double-way, learning rates), unsharded, sharded and with local steps, against the oracle: every combination the
 hand-written cases do not name explicitly still has to give the oracle's bits."""
 import numpy as np
 import pytest
@@ -95,3 +95,31 @@ def test_random_sharded_configuration(case):
                 assert_same(f"{tag} e[{b + kl}]", cpu(s.get_state(sb.STATE_WORKER_ERROR, kl)), orc.get(orc.E, b + kl))
     for s in shards:
         s.close()
+
+
+@pytest.mark.parametrize("case", range(40))
+def test_random_local_steps_configuration(case):
+    """The same draw with the model differences communicated every H iterations (step-ahead branch, p = inf)."""
+    import torch
+    c = draw(200 + case)
+    H = int(np.random.default_rng(case).integers(2, 6))
+    K, sizes = c["K"], c["sizes"]
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(c["seed"], len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(c["seed"], d)
+    kw = dict(compressor=c["comp"], server_compress=c["dc"], momentum=c["mu"], weight_decay=c["lam"], topk_num=1,
+              topk_den=c["den"], local_steps=H)
+    orc = so.Oracle(K, sizes, x0, threads=4, **kw)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
+    for t in range(2 * H + 1):
+        g = synth.grads_numpy(c["seed"], t, K, sizes, scales, 66, 100.0)
+        lr = c["lrs"][t % 3]
+        orc.step(g, lr)
+        gpu.step(torch.from_numpy(g).cuda(), lr)
+        comm = (t + 1) % H == 0
+        if case % 2 == 0 or comm or t == 2 * H:
+            compare_state(gpu, orc, c["comp"], check_messages=comm, tag=f"local case {case} H={H} {c} t={t + 1}")
+            if comm:
+                compare_server_messages(gpu, orc, c["comp"], c["dc"], tag=f"local case {case} t={t + 1}")
+    assert not orc.range_flag
+    gpu.close()
