@@ -345,10 +345,21 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 // LSRV != 0 (Top-K): the previous step left its server lines pending -- e = Delta - C(Delta), x = x - C(Delta)
 // and the server's selection words; they are carried out here on the fly with last step's server threshold
 // (LSRV 2) or with C = identity (LSRV 1, single-way), the same operations the apply kernel would have done.
+#ifndef SAE_DENSE_B
+#define SAE_DENSE_B 8
+#endif
+#ifndef SAE_DENSE_MINB
+#define SAE_DENSE_MINB 5
+#endif
+#ifndef SAE_DENSE_B_AVG
+#define SAE_DENSE_B_AVG 4
+#endif
+
 template <int COMP, bool AVG, bool RECOMP = false, int LSRV = 0>
-__global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
+__global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
+  constexpr int DENSE_B = AVG ? SAE_DENSE_B_AVG : SAE_DENSE_B;   // workers per batch of row loads
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
   const bool emit = (COMP == 2) && A.emit_srv;
@@ -367,7 +378,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   const u32 t_old = (LSRV == 2) ? A.tau_srv_prev[ti.j] : 0u;
   const int lane = tid & 31, warp = tid >> 5;
   if (ti.cnt == TILE) {
-#pragma unroll 2
+#pragma unroll 1
     for (int it = 0; it < VEC_ITERS; ++it) {
       const int i = it * (THREADS * 4) + tid * 4;
       float4 e = ld4(ep + i);
@@ -388,9 +399,19 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       if (RECOMP) eold = ld4(eo + i);
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
-#pragma unroll 8
-      for (int k = 0; k < P.K; ++k) {
-        float4 v = RECOMP ? ld4(dp + (long long)k * P.dpad + i) : ld4_stream(dp + (long long)k * P.dpad + i);
+      // the rows of DENSE_B workers are fetched as one batch of independent loads before any of them is used
+      for (int k0 = 0; k0 < P.K; k0 += DENSE_B) {
+        float4 vb[DENSE_B];
+#pragma unroll
+        for (int u = 0; u < DENSE_B; ++u) {
+          const float* src = dp + (long long)(k0 + u) * P.dpad + i;
+          vb[u] = (k0 + u < P.K) ? (RECOMP ? ld4(src) : ld4_stream(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < DENSE_B; ++u) {
+        if (k0 + u < P.K) {
+        const int k = k0 + u;
+        float4 v = vb[u];
         if (RECOMP) {
           v.x = __fmaf_rn(A.eta, v.x, eold.x); v.y = __fmaf_rn(A.eta, v.y, eold.y);
           v.z = __fmaf_rn(A.eta, v.z, eold.z); v.w = __fmaf_rn(A.eta, v.w, eold.w);
@@ -404,6 +425,8 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
         if (AVG) {
           b0 = __fadd_rn(b0, __fsub_rn(v.x, c0)); b1 = __fadd_rn(b1, __fsub_rn(v.y, c1));
           b2 = __fadd_rn(b2, __fsub_rn(v.z, c2)); b3 = __fadd_rn(b3, __fsub_rn(v.w, c3));
+        }
+        }
         }
       }
       if (AVG) st4(A.ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
