@@ -168,6 +168,18 @@ struct LaunchScope {
     kern<<<(unsigned)(grid), THREADS, 0, (h)->stream>>>(__VA_ARGS__);      \
   } while (0)
 
+// The dense server pass reads through a shared-memory ring above the 48 KB that need no opt-in.
+#define LAUNCH_DENSE(h, kern, grid, ...)                                                                   \
+  do {                                                                                                     \
+    static thread_local int configured_device_ = -1;                                                       \
+    if (configured_device_ != (h)->device) {                                                               \
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDenseSmem);            \
+      configured_device_ = (h)->device;                                                                    \
+    }                                                                                                      \
+    LaunchScope ls_(h, S_SERVER);                                                                          \
+    kern<<<(unsigned)(grid), THREADS, kDenseSmem, (h)->stream>>>(__VA_ARGS__);                             \
+  } while (0)
+
 int check_launch(sae_handle* h) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { h->last_cuda_error = (int)e; return SAE_ERR_CUDA; }
@@ -493,9 +505,9 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (nod) sa.ebar = ebar_other(h);          // becomes the current one when `last` flips below
 #define SAE_DENSE(AVGF, RECF)                                                                              \
     do {                                                                                                   \
-      if (lsrv == 0) LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 0>), P.ntiles, P, sa);             \
-      else if (lsrv == 1) LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 1>), P.ntiles, P, sa);        \
-      else LAUNCH(h, S_SERVER, (k_server_dense<2, AVGF, RECF, 2>), P.ntiles, P, sa);                       \
+      if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, AVGF, RECF, 0>), P.ntiles, P, sa);                 \
+      else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, AVGF, RECF, 1>), P.ntiles, P, sa);            \
+      else LAUNCH_DENSE(h, (k_server_dense<2, AVGF, RECF, 2>), P.ntiles, P, sa);                           \
     } while (0)
     if (nod) SAE_DENSE(true, true);
     else if (avg_after) SAE_DENSE(true, false);
@@ -513,7 +525,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // identity: every error stays exactly zero, so e^(k) is the (all-zero) uniform vector forever
     if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true>(h, sp, wa);
     else launch_worker<ESRC_UNIFORM, false, true>(h, sp, wa);
-    LAUNCH(h, S_SERVER, (k_server_dense<0, false>), P.ntiles, P, sa);
+    LAUNCH_DENSE(h, (k_server_dense<0, false>), P.ntiles, P, sa);
     launch_apply<0, 0>(h, AVG_NONE, aa);
     h->esrc = ESRC_UNIFORM;
   }

@@ -345,21 +345,31 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 // LSRV != 0 (Top-K): the previous step left its server lines pending -- e = Delta - C(Delta), x = x - C(Delta)
 // and the server's selection words; they are carried out here on the fly with last step's server threshold
 // (LSRV 2) or with C = identity (LSRV 1, single-way), the same operations the apply kernel would have done.
-#ifndef SAE_DENSE_B
-#define SAE_DENSE_B 8
+// Full tiles are read through a ring of DENSE_RING thread-private 16-byte slots in shared memory filled by
+// asynchronous copies (cp.async): the reads of a thread -- per group of four parameters the server error,
+// (deferred lines) the parameters, (recompute) the old averaged error, then the K rows in k order -- form one
+// sequence, and the copy of element q + DENSE_RING - 1 of that sequence is issued when element q is consumed,
+// so about DENSE_RING - 1 loads per thread are in flight at any time whatever K is and without holding
+// registers for them.  A thread reads back only what it copied itself: no block-level synchronisation.
+#ifndef SAE_DENSE_RING
+#define SAE_DENSE_RING 8
 #endif
-#ifndef SAE_DENSE_MINB
-#define SAE_DENSE_MINB 5
-#endif
-#ifndef SAE_DENSE_B_AVG
-#define SAE_DENSE_B_AVG 4
-#endif
+constexpr int DENSE_RING = SAE_DENSE_RING;
+constexpr size_t kDenseSmem = (size_t)DENSE_RING * THREADS * sizeof(float4);
+
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((u32)__cvta_generic_to_shared(dst_smem)), "l"(src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 template <int COMP, bool AVG, bool RECOMP = false, int LSRV = 0>
-__global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P, ServerArgs A) {
+__global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
-  constexpr int DENSE_B = AVG ? SAE_DENSE_B_AVG : SAE_DENSE_B;   // workers per batch of row loads
+  extern __shared__ float4 ring[];                       // [DENSE_RING][THREADS]
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
   const bool emit = (COMP == 2) && A.emit_srv;
@@ -378,12 +388,41 @@ __global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P
   const u32 t_old = (LSRV == 2) ? A.tau_srv_prev[ti.j] : 0u;
   const int lane = tid & 31, warp = tid >> 5;
   if (ti.cnt == TILE) {
+    constexpr int NPRE = 1 + (LSRV != 0 ? 1 : 0) + (RECOMP ? 1 : 0);   // reads ahead of the rows, per iteration
+    const int per_it = NPRE + P.K;
+    // the prefetch stream: element `pq` of iteration `pit` goes into slot `pslot`
+    int pit = 0, pq = 0, pslot = 0;
+    auto issue_next = [&]() {
+      if (pit < VEC_ITERS) {
+        const int i = pit * (THREADS * 4) + tid * 4;
+        const float* src;
+        if (pq == 0) src = ep + i;
+        else if (LSRV != 0 && pq == 1) src = xp + i;
+        else if (RECOMP && pq == NPRE - 1) src = eo + i;
+        else src = dp + (long long)(pq - NPRE) * P.dpad + i;
+        cp_async16(&ring[pslot * THREADS + tid], src);
+        if (++pq == per_it) { pq = 0; ++pit; }
+        if (++pslot == DENSE_RING) pslot = 0;
+      }
+      cp_async_commit();                                  // (an empty group past the end keeps the count uniform)
+    };
+    // the consumer: waits until the oldest outstanding copy has landed, reads it, and issues the next copy
+    int cslot = 0;
+    auto take = [&]() -> float4 {
+      cp_async_wait<DENSE_RING - 2>();
+      const float4 v = ring[cslot * THREADS + tid];
+      if (++cslot == DENSE_RING) cslot = 0;
+      issue_next();
+      return v;
+    };
+#pragma unroll 1
+    for (int q = 0; q < DENSE_RING - 1; ++q) issue_next();
 #pragma unroll 1
     for (int it = 0; it < VEC_ITERS; ++it) {
       const int i = it * (THREADS * 4) + tid * 4;
-      float4 e = ld4(ep + i);
+      float4 e = take();
       if (LSRV != 0) {
-        float4 xv = ld4(xp + i);
+        float4 xv = take();
         const bool q0 = LSRV == 1 || topk_selected(e.x, t_old), q1 = LSRV == 1 || topk_selected(e.y, t_old);
         const bool q2 = LSRV == 1 || topk_selected(e.z, t_old), q3 = LSRV == 1 || topk_selected(e.w, t_old);
         const float c0 = q0 ? e.x : 0.0f, c1 = q1 ? e.y : 0.0f, c2 = q2 ? e.z : 0.0f, c3 = q3 ? e.w : 0.0f;
@@ -396,22 +435,12 @@ __global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P
         }
       }
       float4 eold = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (RECOMP) eold = ld4(eo + i);
+      if (RECOMP) eold = take();
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
-      // the rows of DENSE_B workers are fetched as one batch of independent loads before any of them is used
-      for (int k0 = 0; k0 < P.K; k0 += DENSE_B) {
-        float4 vb[DENSE_B];
-#pragma unroll
-        for (int u = 0; u < DENSE_B; ++u) {
-          const float* src = dp + (long long)(k0 + u) * P.dpad + i;
-          vb[u] = (k0 + u < P.K) ? (RECOMP ? ld4(src) : ld4_stream(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int u = 0; u < DENSE_B; ++u) {
-        if (k0 + u < P.K) {
-        const int k = k0 + u;
-        float4 v = vb[u];
+#pragma unroll 4
+      for (int k = 0; k < P.K; ++k) {
+        float4 v = take();
         if (RECOMP) {
           v.x = __fmaf_rn(A.eta, v.x, eold.x); v.y = __fmaf_rn(A.eta, v.y, eold.y);
           v.z = __fmaf_rn(A.eta, v.z, eold.z); v.w = __fmaf_rn(A.eta, v.w, eold.w);
@@ -426,8 +455,6 @@ __global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P
           b0 = __fadd_rn(b0, __fsub_rn(v.x, c0)); b1 = __fadd_rn(b1, __fsub_rn(v.y, c1));
           b2 = __fadd_rn(b2, __fsub_rn(v.z, c2)); b3 = __fadd_rn(b3, __fsub_rn(v.w, c3));
         }
-        }
-        }
       }
       if (AVG) st4(A.ebar + pbase + i, make_float4(div_by_k(P, b0), div_by_k(P, b1), div_by_k(P, b2), div_by_k(P, b3)));
       float4 ds;
@@ -441,6 +468,7 @@ __global__ void __launch_bounds__(THREADS, SAE_DENSE_MINB) k_server_dense(Plan P
         stage_row4(stg, lo, mag_key(ds.x), mag_key(ds.y), mag_key(ds.z), mag_key(ds.w));
       }
     }
+    cp_async_wait<0>();
   } else {
     for (int r = 0; r < ROWS; ++r) {
       const int i = r * THREADS + tid;
