@@ -31,7 +31,11 @@ FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case of the same kernel, which grows in
 # proportion to the elements processed).  None until a capture exists for the variant.
 # sign_p1: 13.64 B at K = 4 = 12 B per worker-element + (8 B of ebar + sign words) per parameter.
-WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0), "topk": None}   # (per worker-element, per parameter), profiles/worker_pass_sign_cfg2shapes_4workers.md
+# topk_p1: 1324.2 MB for 4 x 25.56 M worker-elements = 12 B per worker-element + 3.81 B per parameter (ebar);
+# topk_general: 2027.4 MB = 19.83 B per worker-element (candidate lists included).
+WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0),      # (per worker-element, per parameter)
+                          "topk_p1": (12.0, 3.81), "topk_general": (19.83, 0.0),      # profiles/worker_pass_sign_cfg2shapes_4workers.md,
+                          "mu0": None}                                                # profiles/topk_passes_cfg3shapes_4workers.md
 
 
 def measured_peak():
@@ -193,7 +197,7 @@ def algorithmic_bytes(w, avg_period):
         # scaled sign: g R, m RW | ebar RW (the pending average is formed in this pass);
         # Top-K: g R, m RW | ebar R (Delta is not stored: the server pass recomputes it from m)
         worker = 12 * Wd + 4 * d if topk else 12 * Wd + 8 * d
-        variant = "topk" if topk else "sign_p1"
+        variant = "topk_p1" if topk else "sign_p1"
     elif w.momentum == 0.0:
         step = 12 * Wd + 16 * d              # g R, e RW | x RW, e_srv RW  (mu = 0: no momentum rows)
         worker = 12 * Wd                     # g R, Delta(e) RW
@@ -201,7 +205,7 @@ def algorithmic_bytes(w, avg_period):
     else:
         step = 20 * Wd + 16 * d              # g R, m RW, e RW | x RW, e_srv RW
         worker = 20 * Wd                     # g R, m RW, Delta(e) RW
-        variant = "topk" if topk else "sign_general"
+        variant = "topk_general" if topk else "sign_general"
     return step, worker, variant
 
 
