@@ -353,8 +353,15 @@ void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, c
   const long long nitems = (long long)h->P.ntiles * FwGeom<K>::SUB;
   long long grid = h->persistent_blocks / SAE_WT_BLOCKS_PER_SM;      // one block per SM
   if (nitems < grid) grid = nitems;
+  // Runs of one plan tile per block when the tensors are short (block-wise compression: a few tiles each) and
+  // there is enough work to keep every block busy that way; long tensors stream best with the ranges dealt
+  // out one by one (runs cost 4-5 % there).
+  const bool short_tensors = h->P.ntiles < 4LL * h->P.T;
+  int chunk_log2 = 0;
+  if (short_tensors && nitems >= 8 * grid * FwGeom<K>::SUB)
+    while ((1 << chunk_log2) < FwGeom<K>::SUB) ++chunk_log2;
   LaunchScope ls(h, S_WORKER);
-  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, h->tm_m, tm_g);
+  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, chunk_log2, h->tm_m, tm_g);
 }
 
 template <int K>

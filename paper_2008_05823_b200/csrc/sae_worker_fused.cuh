@@ -130,8 +130,26 @@ __device__ __forceinline__ FwItem fw_lookup(const Plan& P, int g_tma_ok, long lo
   return it;
 }
 
+// The q-th element range of block b: the blocks take runs of `chunk` consecutive ranges in turn.  With runs
+// of one plan tile (chunk = SUB) the consecutive ranges of a block mostly belong to the same tensor even when
+// the tensors are single tiles (block-wise compression), so the L1 partials are committed once per run
+// instead of once per range; chunk = 1 (long tensors, small problems) deals the ranges out one by one.
+// (chunk = 2^chunk_log2)
+__device__ __forceinline__ long long fw_range_of(int q, int chunk_log2) {
+  return (((long long)(q >> chunk_log2) * gridDim.x + blockIdx.x) << chunk_log2) + (q & ((1 << chunk_log2) - 1));
+}
+// how many ranges this block takes in all
+__device__ __forceinline__ int fw_ranges_of_block(long long nitems, int chunk_log2) {
+  const long long cycle = (long long)gridDim.x << chunk_log2;
+  const long long full = nitems / cycle;
+  const long long rest = nitems - full * cycle - ((long long)blockIdx.x << chunk_log2);
+  const long long tail = rest < 0 ? 0 : (rest > (1LL << chunk_log2) ? (1LL << chunk_log2) : rest);
+  return (int)((full << chunk_log2) + tail);
+}
+
 template <int K, bool WD>
 __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepParams sp, FusedArgs A, long long nitems,
+                                                                 int chunk_log2,
                                                                  const __grid_constant__ CUtensorMap tm_m,
                                                                  const __grid_constant__ CUtensorMap tm_g) {
   typedef FwGeom<K> G;
@@ -141,6 +159,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   constexpr int FW_BOX = G::BOX;
   Smem& S = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nmine = fw_ranges_of_block(nitems, chunk_log2);
   if (tid == 0) {
     for (int s = 0; s < FW_STAGES; ++s) {
       mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], FW_WARPS); mbar_init(&S.avgd[s], FW_AVG_WARPS);
@@ -152,12 +171,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   if (warp == FW_WARPS) {
     // ---------------- producer ----------------
     // nitems counts element ranges; each is issued as HALVES consecutive items (one per group of KH workers)
-    const long long GR = gridDim.x;
-    long long wb = blockIdx.x;
-    FwItem nxt = fw_lookup<K>(P, A.g_tma_ok, wb + lane * GR, nitems);
-    for (int p0 = 0; wb < nitems; p0 += 32, wb += 32 * GR) {
+    FwItem nxt = fw_lookup<K>(P, A.g_tma_ok, fw_range_of(lane, chunk_log2), nitems);
+    for (int p0 = 0; p0 < nmine; p0 += 32) {
       const FwItem cur = nxt;
-      nxt = fw_lookup<K>(P, A.g_tma_ok, wb + (32 + lane) * GR, nitems);
+      nxt = fw_lookup<K>(P, A.g_tma_ok, fw_range_of(p0 + 32 + lane, chunk_log2), nitems);
       for (int l = 0; l < 32; ++l) {
         // the range of lane l, broadcast so that the lanes can share the issue of its copies
         const int cnt = __shfl_sync(0xffffffffu, cur.cnt, l);
@@ -217,9 +234,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     for (int c = 0; c < CH; ++c)
 #pragma unroll
       for (int v = 0; v < V; ++v) { eb[c][v] = 0.0f; a[c][v] = 0.0f; }
-    for (int i = 0;; ++i) {
-      const long long w = blockIdx.x + (long long)(i / G::HALVES) * gridDim.x;
-      if (w >= nitems) break;
+    for (int i = 0; i < nmine * G::HALVES; ++i) {
       const int hh = i % G::HALVES;
       const int s = i % FW_STAGES;
       if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
@@ -279,9 +294,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   int acc_j = -1;
   const int row0 = warp * G::RPW;                       // first row of this warp inside an item
   const int kl0 = row0 / G::ROWS_PER_WORKER;            // its (first) worker inside the item's group
-  for (int i = 0;; ++i) {
-    const long long w = blockIdx.x + (long long)(i / G::HALVES) * gridDim.x;
-    if (w >= nitems) break;
+  for (int i = 0; i < nmine * G::HALVES; ++i) {
     const int hh = i % G::HALVES;
     const int s = i % FW_STAGES;
     if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
