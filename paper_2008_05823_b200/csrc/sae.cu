@@ -27,8 +27,8 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm; const float* grads; float lr, eta_prev; };
-struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after; uint64_t stamp; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm, tail; const float* grads; float lr, eta_prev; };
+struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after, tail_after; uint64_t stamp; };
 
 }  // namespace
 
@@ -92,6 +92,11 @@ struct sae_handle {
   int attached;                     // workers whose message rows are known
   int mid_step;                     // sae_step_begin done, sae_step_end due
   int local_steps;                  // H: iteration t communicates iff (t+1) mod H == 0 (1: every iteration)
+  // Top-K, p = 1, K = 8 or 16, no weight decay: the tail of a step (worker-axis aggregation, averaged error,
+  // server lines) is left to the worker pass of the next step, which reads the same momentum rows anyway
+  int fused_topk_ok;
+  int tail_pending;                 // the last step stopped after its threshold select
+  float* ssum;                      // [dpad] ordered worker-axis sum of the selected entries (folded form)
   int avg_external;                 // the averaging sum is all-reduced by the caller instead of pulled in k order
   int avg_owed;                     // ... and is owed before the next sae_step_begin
   float lr_pending;
@@ -198,7 +203,7 @@ void free_all(sae_handle* h) {
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
                   h->tau_srv, h->recs, h->recs_alt, h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
-                  h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n};
+                  h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n, h->ssum};
   for (void* p : ptrs) if (p) cudaFree(p);
   void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows,
                   (void*)h->d_entry_rows, (void*)h->d_count_rows, (void*)h->d_tau_rows[0], (void*)h->d_tau_rows[1],
@@ -254,7 +259,33 @@ CandArgs cand_args(sae_handle* h, bool server) {
 #ifndef SAE_LAZY_SERVER
 #define SAE_LAZY_SERVER 1        // 0: every step runs its own apply kernel
 #endif
+// Top-K, folded form: carries out the tail the last step left to the next worker pass -- the dense server
+// pass over the momentum rows (worker-axis aggregation, averaged error, any older pending server lines) and
+// the server's threshold select -- the way a step that does not fold would have done it itself.  The step has
+// already flipped `last`: its thresholds are tau[last], the uniform error it started from is ebar_other, the
+// new one goes to ebar_now.  The server lines of that step are then pending like after any other step.
+int flush_tail(sae_handle* h) {
+  if (!h->tail_pending) return SAE_OK;
+  const Plan& P = h->P;
+  const bool dc = h->cfg.server_compress != 0;
+  ServerArgs sa;
+  memset(&sa, 0, sizeof(sa));
+  sa.e_srv = h->e_srv; sa.tau_cur = h->tau[h->last]; sa.status = h->status;
+  sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0;
+  sa.m = h->m; sa.ebar_in = ebar_other(h); sa.ebar = ebar_now(h); sa.eta = h->eta_prev;
+  sa.x = h->x; sa.mask_srv = h->mask_srv;
+  const int lsrv = h->srv_pending ? (dc ? 2 : 1) : 0;
+  if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 0>), P.ntiles, P, sa);
+  else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 1>), P.ntiles, P, sa);
+  else LAUNCH_DENSE(h, (k_server_dense<2, true, true, 2>), P.ntiles, P, sa);
+  if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
+  h->srv_pending = 1;
+  h->tail_pending = 0;
+  return check_launch(h);
+}
+
 int flush_server(sae_handle* h) {
+  { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
   if (!h->srv_pending) return SAE_OK;
   ApplyArgs aa;
   memset(&aa, 0, sizeof(aa));
@@ -341,13 +372,13 @@ bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int K, bool WD>
+template <int K, bool WD, bool TOPK = false>
 void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, const CUtensorMap& tm_g) {
-  constexpr size_t kFusedSmem = sizeof(FwSmemT<K>) + 128;
+  constexpr size_t kFusedSmem = sizeof(FwSmemT<K, TOPK>) + 128;
   static_assert(kFusedSmem <= 227 * 1024, "the ring must fit the shared memory of one block");
   static thread_local int configured_device = -1;
   if (configured_device != h->device) {
-    cudaFuncSetAttribute(k_worker_fused<K, WD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
+    cudaFuncSetAttribute(k_worker_fused<K, WD, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
     configured_device = h->device;
   }
   const long long nitems = (long long)h->P.ntiles * FwGeom<K>::SUB;
@@ -361,7 +392,7 @@ void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, c
   if (short_tensors && nitems >= 8 * grid * FwGeom<K>::SUB)
     while ((1 << chunk_log2) < FwGeom<K>::SUB) ++chunk_log2;
   LaunchScope ls(h, S_WORKER);
-  k_worker_fused<K, WD><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, chunk_log2, h->tm_m, tm_g);
+  k_worker_fused<K, WD, TOPK><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, chunk_log2, h->tm_m, tm_g);
 }
 
 template <int K>
@@ -369,11 +400,17 @@ void launch_fused_k(sae_handle* h, const StepParams& sp, const FusedArgs& fa, co
   if (sp.wd) launch_fused_kw<K, true>(h, sp, fa, tm_g); else launch_fused_kw<K, false>(h, sp, fa, tm_g);
 }
 
-void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa) {
+void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa, bool topk = false) {
   // the gradients live in the caller's buffer: encode their tensor map for this step (host-only work)
   CUtensorMap tm_g;
   memset(&tm_g, 0, sizeof(tm_g));
   fa.g_tma_ok = make_row_map(&tm_g, fa.g, h->P.d, h->P.K, h->P.d) ? 1 : 0;
+  if (topk) {                          // (K = 8 or 16, no weight decay: checked by the caller)
+    if (h->P.K == 8) launch_fused_kw<8, false, true>(h, sp, fa, tm_g);
+    else launch_fused_kw<16, false, true>(h, sp, fa, tm_g);
+    return;
+  }
+  fa.ebar_out = fa.ebar;
   switch (h->P.K) {
     case 1: launch_fused_k<1>(h, sp, fa, tm_g); break;
     case 2: launch_fused_k<2>(h, sp, fa, tm_g); break;
@@ -503,11 +540,37 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     sa.x = h->x; sa.mask_srv = h->mask_srv;
     DeltaSrc src = stored_rows(h->D);
     if (nod) { src.m = h->m; src.ebar = ebar_now(h); src.eta = lr; src.recompute = 1; }
+    // Folded form: this step stops after its threshold select; the rest (aggregation, averaged error, server
+    // lines) is done by the next step's worker pass and a parameter-sized server pass behind it.
+    const bool fold = nod && h->fused_topk_ok && lazy_ok;
+    if (h->tail_pending) {
+      if (!fold) return SAE_ERR_INVALID_ARG;
+      FusedArgs fa;
+      memset(&fa, 0, sizeof(fa));
+      fa.g = grads; fa.m = h->m; fa.ebar = ebar_other(h); fa.ebar_out = ebar_now(h); fa.x = h->x;
+      fa.tau_prev = h->tau[h->last]; fa.ssum = h->ssum; fa.cand = wa.cand; fa.status = h->status;
+      fa.eta_prev = h->eta_prev;
+      launch_fused(h, sp, fa, true);
+      topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+      sa.ssum = h->ssum;
+      if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 0, true>), P.ntiles, P, sa);
+      else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 1, true>), P.ntiles, P, sa);
+      else LAUNCH_DENSE(h, (k_server_dense<2, false, false, 2, true>), P.ntiles, P, sa);
+      if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
+      h->srv_pending = 1;                    // the previous step's server lines now wait for the next server pass
+      h->last = cur; h->eta_prev = lr; h->t += 1;
+      return check_launch(h);
+    }
     if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
     else if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
     else if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true, true>(h, sp, wa);
     else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
     topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+    if (fold) {                              // first folded step: nothing to catch up with, the tail stays open
+      h->tail_pending = 1;
+      h->last = cur; h->eta_prev = lr; h->t += 1;
+      return check_launch(h);
+    }
     // the averaged error (if the pre-step averages) comes out of the same pass over D as the server's sum
     if (nod) sa.ebar = ebar_other(h);          // becomes the current one when `last` flips below
 #define SAE_DENSE(AVGF, RECF)                                                                              \
@@ -560,16 +623,17 @@ int do_step(sae_handle* h, const float* grads, float lr) {
 
   StepGraphKey key;
   key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending; key.rot = h->rot;
-  key.comm = communicates(h) ? 1 : 0;
+  key.comm = communicates(h) ? 1 : 0; key.tail = h->tail_pending;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.tail == key.tail && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
       h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->rot = e.rot_after;
+      h->tail_pending = e.tail_after;
       h->eta_prev = lr; h->t += 1;
       e.stamp = ++h->graph_clock;
       h->graph_misses = 0;
@@ -592,6 +656,7 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   StepGraph e;
   e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
   e.esrc_after = h->esrc; e.last_after = h->last; e.pending_after = h->srv_pending; e.rot_after = h->rot;
+  e.tail_after = h->tail_pending;
   e.stamp = ++h->graph_clock;
   ce = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
@@ -625,6 +690,7 @@ ExportArgs export_args(sae_handle* h, int what, int k, bool need_error) {
 
 int export_vec(sae_handle* h, int what, int k, float* out) {
   if (what != EXP_M) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }     // x and e must be up to date
+  else { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
   const ExportArgs ea = export_args(h, what, k, what == EXP_WERR || what == EXP_STEP_AHEAD);
   LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
   return check_launch(h);
@@ -759,6 +825,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   if (h->fused_ok) ALLOC0(h->etmp, dpad);
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
   if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
+  h->fused_topk_ok = (h->topk_nod && (K == 8 || K == 16) && dpad < (1ll << 31) && d < (1ll << 31)) ? 1 : 0;
+  h->tail_pending = 0;
+  if (h->fused_topk_ok) ALLOC0(h->ssum, dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);
   ALLOC0(h->mask_srv, topk ? nwords : 0);
@@ -815,6 +884,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
     TRY(cudaStreamSynchronize(h->stream));     // host tables above go out of scope
   }
 #undef TRY
+  if (rc == SAE_OK && h->fused_topk_ok && !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_topk_ok = 0;
   if (rc == SAE_OK && h->fused_ok) {
     // the folded-averaging pass needs a tensor map over the momentum rows and 32-bit TMA coordinates
     if (dpad >= (1ll << 31) || d >= (1ll << 31) || !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_ok = 0;
@@ -1172,6 +1242,7 @@ int sae_get_state(sae_handle* h, int32_t which, int32_t worker, void* out, size_
   if (per_worker && (worker < 0 || worker >= P.K)) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
+  { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
   if (which == SAE_STATE_SERVER_SCALES || which == SAE_STATE_SERVER_MASK) {
     int rcf = flush_server(h);
     if (rcf != SAE_OK) return rcf;
@@ -1257,6 +1328,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
   }
   h->t = hd.t; h->esrc = hd.esrc; h->last = hd.last; h->eta_prev = hd.eta_prev;
   h->srv_pending = 0;        // a checkpoint is taken with the server lines carried out
+  h->tail_pending = 0;
   if (h->inline_fin) {       // the L1 records are transient, but nothing else clears them before the next step
     SAE_CUDA(h, cudaMemsetAsync(h->recs, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
     SAE_CUDA(h, cudaMemsetAsync(h->recs_srv, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));

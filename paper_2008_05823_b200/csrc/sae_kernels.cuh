@@ -75,6 +75,7 @@ struct ServerArgs {
   const float* m;          // [K][dpad] } recompute variant: Delta^(k) = fma(eta, m^(k), ebar_in), not stored
   const float* ebar_in;    // [dpad]    } (ebar_in and ebar are different buffers)
   float eta;
+  const float* ssum;       // [dpad] (SUM variant) ordered worker-axis sum of the selected entries, not yet divided by K
   // sharded operation: worker k's message lives with its owner (possibly another GPU's memory, read in place)
   const u32* const* word_rows;     // [K] -> worker k's [nwords] sign words
   const float* const* scale_rows;  // [K] -> worker k's [T] scales of this step
@@ -365,7 +366,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int COMP, bool AVG, bool RECOMP = false, int LSRV = 0>
+// SUM (Top-K, p = 1, folded form): the ordered worker-axis sum of the selected entries was already formed by
+// the worker pass of the following step (k_worker_fused<.., TOPK>) and is only read here; no rows are touched.
+template <int COMP, bool AVG, bool RECOMP = false, int LSRV = 0, bool SUM = false>
 __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) {
   __shared__ u32 t_k[MAX_WORKERS];
   __shared__ u32 cstage[(COMP == 2) ? (THREADS / 32) * CAND_STAGE : 1];
@@ -383,13 +386,15 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   float* ep = A.e_srv + pbase;
   const float* __restrict__ dp = (RECOMP ? A.m : A.D) + pbase;
   const float* __restrict__ eo = A.ebar_in + pbase;      // read only when RECOMP
+  const float* __restrict__ sump = A.ssum + pbase;       // read only when SUM
   float* xp = A.x + pbase;                               // (LSRV only)
   u32* mwp = A.mask_srv + (pbase >> 5);                  // (LSRV 2 only)
   const u32 t_old = (LSRV == 2) ? A.tau_srv_prev[ti.j] : 0u;
   const int lane = tid & 31, warp = tid >> 5;
   if (ti.cnt == TILE) {
-    constexpr int NPRE = 1 + (LSRV != 0 ? 1 : 0) + (RECOMP ? 1 : 0);   // reads ahead of the rows, per iteration
-    const int per_it = NPRE + P.K;
+    constexpr int NPRE = 1 + (LSRV != 0 ? 1 : 0) + ((RECOMP || SUM) ? 1 : 0);   // reads ahead of the rows, per iteration
+    const int nrows = SUM ? 0 : P.K;
+    const int per_it = NPRE + nrows;
     // the prefetch stream: element `pq` of iteration `pit` goes into slot `pslot`
     int pit = 0, pq = 0, pslot = 0;
     auto issue_next = [&]() {
@@ -399,6 +404,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
         if (pq == 0) src = ep + i;
         else if (LSRV != 0 && pq == 1) src = xp + i;
         else if (RECOMP && pq == NPRE - 1) src = eo + i;
+        else if (SUM && pq == NPRE - 1) src = sump + i;
         else src = dp + (long long)(pq - NPRE) * P.dpad + i;
         cp_async16(&ring[pslot * THREADS + tid], src);
         if (++pq == per_it) { pq = 0; ++pit; }
@@ -438,8 +444,9 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       if (RECOMP) eold = take();
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
       float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
+      if (SUM) { const float4 sv = take(); a0 = sv.x; a1 = sv.y; a2 = sv.z; a3 = sv.w; }
 #pragma unroll 4
-      for (int k = 0; k < P.K; ++k) {
+      for (int k = 0; k < nrows; ++k) {
         float4 v = take();
         if (RECOMP) {
           v.x = __fmaf_rn(A.eta, v.x, eold.x); v.y = __fmaf_rn(A.eta, v.y, eold.y);
@@ -475,9 +482,9 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       float ds = 0.0f;
       bool qs = false;
       if (i < ti.cnt) {
-        float a = 0.f, b = 0.f;
+        float a = SUM ? sump[i] : 0.f, b = 0.f;
         const float ebo = RECOMP ? eo[i] : 0.0f;
-        for (int k = 0; k < P.K; ++k) {
+        for (int k = 0; k < (SUM ? 0 : P.K); ++k) {
           float v = dp[(long long)k * P.dpad + i];
           if (RECOMP) v = __fmaf_rn(A.eta, v, ebo);
           const float c = (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f;

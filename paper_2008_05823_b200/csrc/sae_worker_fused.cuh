@@ -85,7 +85,7 @@ struct FwItem {
   int h;             // which group of KH workers
 };
 
-template <int K>
+template <int K, bool TOPK = false>
 struct FwSmemT {
   typedef FwGeom<K> G;
   alignas(128) float m[G::STAGES][G::MBUF];
@@ -95,13 +95,18 @@ struct FwSmemT {
   alignas(8) u64 empty[G::STAGES];
   alignas(8) u64 avgd[G::STAGES];   // "ebar' of this stage is ready": one arrival per averager warp
   FwItem item[G::STAGES];
-  float sc[G::STAGES][32];      // last step's scales of the item's tensor, one per worker
+  float sc[G::STAGES][32];      // last step's scales (Top-K: threshold bit patterns) of the item's tensor, one per worker
+  u32 cstage[TOPK ? FW_WARPS : 1][TOPK ? CAND_STAGE : 1];   // Top-K: per-warp staging of candidate keys
 };
 
 struct FusedArgs {
   const float* g;
   float* m;
-  float* ebar;             // in: ebar of the previous step, out: the averaged error of this pre-step
+  float* ebar;             // in: ebar of the previous step
+  float* ebar_out;         // out: the averaged error of this pre-step (scaled sign: the same buffer)
+  const u32* tau_prev;     // Top-K: [K][T] thresholds of the previous step
+  float* ssum;             // Top-K: [dpad] out: sum_k C(Delta^(k)) of the previous step, k in order, not divided by K
+  CandArgs cand;           // Top-K: candidate lists for this step's differences
   const float* x;
   const float* scale_prev; // [K][T] scales of the previous step
   u32* words;
@@ -147,14 +152,20 @@ __device__ __forceinline__ int fw_ranges_of_block(long long nitems, int chunk_lo
   return (int)((full << chunk_log2) + tail);
 }
 
-template <int K, bool WD>
+// TOPK (Top-K, p = 1, K = 8 or 16): the same structure with the compressor changed.  The averagers apply the
+// previous step's thresholds instead of its scales and also form that step's ordered worker-axis sum of the
+// selected entries (the aggregation of the server line: it needs the same rows in the same order), which a
+// parameter-sized server pass then only reads; the workers collect this step's candidate keys instead of L1
+// partials and sign bits.  The differences are never stored.
+template <int K, bool WD, bool TOPK = false>
 __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepParams sp, FusedArgs A, long long nitems,
                                                                  int chunk_log2,
                                                                  const __grid_constant__ CUtensorMap tm_m,
                                                                  const __grid_constant__ CUtensorMap tm_g) {
   typedef FwGeom<K> G;
   extern __shared__ unsigned char smem_raw[];
-  typedef FwSmemT<K> Smem;
+  typedef FwSmemT<K, TOPK> Smem;
+  static_assert(!TOPK || (G::WPW == 1 && G::HALVES == 1), "Top-K form: a worker warp serves one worker");
   constexpr int FW_STAGES = G::STAGES;
   constexpr int FW_BOX = G::BOX;
   Smem& S = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
@@ -186,7 +197,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 #pragma unroll
         for (int hh = 0; hh < G::HALVES; ++hh) {
           float scale_k = 0.0f;
-          if (cnt > 0 && lane < G::KH) scale_k = __ldg(A.scale_prev + (long long)(hh * G::KH + lane) * P.T + j);
+          if (cnt > 0 && lane < G::KH) {
+            if (TOPK) scale_k = __uint_as_float(__ldg(A.tau_prev + (long long)(hh * G::KH + lane) * P.T + j));
+            else scale_k = __ldg(A.scale_prev + (long long)(hh * G::KH + lane) * P.T + j);
+          }
           const int i = (p0 + l) * G::HALVES + hh;
           const int s = i % FW_STAGES;
           int ok = 1;
@@ -229,11 +243,11 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     constexpr int V = EPT < 4 ? EPT : 4;             // handled in chunks of V consecutive elements
     constexpr int CH = EPT / V;
     const int ta = tid - (FW_WARPS + 1) * 32;
-    float eb[CH][V], a[CH][V];
+    float eb[CH][V], a[CH][V], s2[CH][V];          // (s2: Top-K only)
 #pragma unroll
     for (int c = 0; c < CH; ++c)
 #pragma unroll
-      for (int v = 0; v < V; ++v) { eb[c][v] = 0.0f; a[c][v] = 0.0f; }
+      for (int v = 0; v < V; ++v) { eb[c][v] = 0.0f; a[c][v] = 0.0f; s2[c][v] = 0.0f; }
     for (int i = 0; i < nmine * G::HALVES; ++i) {
       const int hh = i % G::HALVES;
       const int s = i % FW_STAGES;
@@ -252,7 +266,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           if (e0 < it.cnt) {
             if (hh == 0) {
 #pragma unroll
-              for (int v = 0; v < V; ++v) { eb[c][v] = se0[e0 + v]; a[c][v] = 0.0f; }
+              for (int v = 0; v < V; ++v) { eb[c][v] = se0[e0 + v]; a[c][v] = 0.0f; s2[c][v] = 0.0f; }
             }
 #pragma unroll
             for (int k = 0; k < G::KH; ++k) {
@@ -260,7 +274,13 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 #pragma unroll
               for (int v = 0; v < V; ++v) {
                 const float dk = __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[c][v]);
-                a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, sign_code(dk, sk)));
+                if (TOPK) {
+                  const float ck = topk_selected(dk, __float_as_uint(sk)) ? dk : 0.0f;
+                  a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, ck));
+                  s2[c][v] = __fadd_rn(s2[c][v], ck);
+                } else {
+                  a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, sign_code(dk, sk)));
+                }
               }
             }
             if (hh == G::HALVES - 1) {
@@ -270,7 +290,8 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
                   const float en = div_by_k(P, a[c][v]);
 #pragma unroll
                   for (int hq = 0; hq < G::HALVES; ++hq) S.e[(i - hh + hq) % FW_STAGES][e0 + v] = en;
-                  A.ebar[it.pbase + e0 + v] = en;
+                  A.ebar_out[it.pbase + e0 + v] = en;
+                  if (TOPK) A.ssum[it.pbase + e0 + v] = s2[c][v];
                 }
               }
             }
@@ -294,6 +315,8 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   int acc_j = -1;
   const int row0 = warp * G::RPW;                       // first row of this warp inside an item
   const int kl0 = row0 / G::ROWS_PER_WORKER;            // its (first) worker inside the item's group
+  WarpStage stg; stg.buf = S.cstage[TOPK ? warp : 0]; stg.n = 0;   // Top-K: this warp's candidate keys of (kl0, stg_j)
+  int stg_j = 0;
   for (int i = 0; i < nmine * G::HALVES; ++i) {
     const int hh = i % G::HALVES;
     const int s = i % FW_STAGES;
@@ -303,7 +326,9 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     }
     const FwItem it = S.item[s];
     if (it.cnt > 0) {
-      if (it.j != acc_j) {
+      if (TOPK) {
+        if (it.j != stg_j) { stage_flush(stg, A.cand, kl0, stg_j); stg_j = it.j; }
+      } else if (it.j != acc_j) {
         if (acc_j >= 0) {
 #pragma unroll
           for (int a = 0; a < G::NACC; ++a) {
@@ -314,6 +339,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         }
         acc_j = it.j;
       }
+      const u32 lo = TOPK ? window_lo(__float_as_uint(S.sc[s][kl0])) : NO_GUESS;
       const float* sm = S.m[s];
       const float* sg = S.g[s];
       const float* se = S.e[s];
@@ -345,10 +371,17 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           dl.z = worker_update<WD>(Gq.z, M.z, E.z, X.z, sp, mn.z);
           dl.w = worker_update<WD>(Gq.w, M.w, E.w, X.w, sp, mn.w);
           st4(mp + e0, mn);
-          if (G::NACC == 1 || a == 0) lane_add4(acc[0], dl);
-          else lane_add4(acc[G::NACC - 1], dl);
-          const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
-          if ((lane & 7) == 0) wp[e0 >> 5] = wd;
+          if (TOPK) {
+            if (lo != NO_GUESS) {
+              if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand, kl0, stg_j);
+              stage_row4(stg, lo, mag_key(dl.x), mag_key(dl.y), mag_key(dl.z), mag_key(dl.w));
+            }
+          } else {
+            if (G::NACC == 1 || a == 0) lane_add4(acc[0], dl);
+            else lane_add4(acc[G::NACC - 1], dl);
+            const u32 wd = pack_row4(dl.x >= 0.0f, dl.y >= 0.0f, dl.z >= 0.0f, dl.w >= 0.0f);
+            if ((lane & 7) == 0) wp[e0 >> 5] = wd;
+          }
         } else if (rr * 128 < it.cnt) {
           // ragged last row of a tensor, or gradients that could not be fetched by TMA
           const float* gp = A.g + (long long)k * P.d + it.goff;
@@ -363,11 +396,20 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
               float mn;
               dl = worker_update<WD>(gv, sm[rbase + c * 32 + lane], se[e], xv, sp, mn);
               mp[e] = mn;
-              if (G::NACC == 1 || a == 0) lane_add(acc[0], dl);
-              else lane_add(acc[G::NACC - 1], dl);
+              if (!TOPK) {
+                if (G::NACC == 1 || a == 0) lane_add(acc[0], dl);
+                else lane_add(acc[G::NACC - 1], dl);
+              }
             }
-            const u32 wd = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
-            if (lane == 0 && (rr * 128 + c * 32) < it.cnt) wp[(rr * 128 + c * 32) >> 5] = wd;
+            if (TOPK) {
+              if (lo != NO_GUESS) {
+                if (stg.n > CAND_STAGE - 32) stage_flush(stg, A.cand, kl0, stg_j);
+                stage_row1(stg, lo, valid, mag_key(dl));
+              }
+            } else {
+              const u32 wd = __ballot_sync(0xffffffffu, valid && dl >= 0.0f);
+              if (lane == 0 && (rr * 128 + c * 32) < it.cnt) wp[(rr * 128 + c * 32) >> 5] = wd;
+            }
           }
         }
       }
@@ -375,7 +417,9 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     __syncwarp();
     if (lane == 0) mbar_arrive(&S.empty[s]);
   }
-  if (acc_j >= 0) {
+  if (TOPK) {
+    stage_flush(stg, A.cand, kl0, stg_j);
+  } else if (acc_j >= 0) {
 #pragma unroll
     for (int a = 0; a < G::NACC; ++a) {
       const int kk = (a / G::WPW) * G::KH + kl0 + (a % G::WPW);

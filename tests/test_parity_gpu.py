@@ -453,3 +453,43 @@ def test_pending_server_lines_survive_a_checkpoint_and_a_side_stream():
         a.close()
         b.close()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("K", [8, 16])
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("every", [1, 2, 5])
+def test_topk_folded_tail(K, dc, every):
+    """Top-K, p = 1, K = 8 or 16, no weight decay: a step stops after its threshold select and the next step's
+    worker pass does the rest; a getter in between carries the open tail out the unfolded way.  Looking at
+    the state every step, every second step and every fifth step mixes both forms in every order."""
+    run_pair(K, RAGGED + [40000], so.TOPK, 11, p=1, dc=dc, seed=11, lrs=[0.1, 0.05, 0.2], every=every, num=1, den=20,
+             outliers=(66, 100.0))
+
+
+@pytest.mark.parametrize("K", [8, 16])
+def test_topk_folded_tail_graph_replay_and_checkpoint(K):
+    import torch
+    sizes = RAGGED + [40000]
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(12, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(12, d)
+    kw = dict(compressor=so.TOPK, avg_period=1, momentum=0.9, topk_num=1, topk_den=20)
+    orc = so.Oracle(K, sizes, x0, threads=4, **kw)
+    with torch.cuda.stream(torch.cuda.Stream()):          # graph replay: the open tail is part of the graph key
+        a = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
+        gs = [torch.from_numpy(synth.grads_numpy(12, t, K, sizes, scales, 66, 100.0)).cuda() for t in range(4)]
+        for t in range(9):
+            orc.step(gs[t % 4].cpu().numpy(), 0.1)
+            a.step(gs[t % 4], 0.1)
+        blob = a.save_state()                             # taken with a tail open: the save closes it
+        b = sb.Sae(K, sizes, torch.zeros(d, device="cuda"), **kw)
+        b.load_state(blob)
+        for t in range(9, 16):
+            orc.step(gs[t % 4].cpu().numpy(), 0.1)
+            a.step(gs[t % 4], 0.1)
+            b.step(gs[t % 4], 0.1)
+        compare_state(a, orc, so.TOPK, tag="continued")
+        compare_state(b, orc, so.TOPK, tag="restored")
+        compare_server_messages(a, orc, so.TOPK, 1, tag="continued")
+        compare_server_messages(b, orc, so.TOPK, 1, tag="restored")
+        a.close(); b.close()
