@@ -45,6 +45,8 @@ struct sae_handle {
   float *x, *e_srv, *ebar, *m, *D;
   float* etmp;           // [dpad] the pending average, materialised for getters only
   CUtensorMap tm_m;      // momentum rows [K][dpad] as a tensor map (folded-averaging worker pass)
+  CUtensorMap tm_D;      // stored model differences [K][dpad] (folded Top-K tail with stored differences)
+  int fused_gen_ok;      // Top-K, p != 1, K = 8 or 16: the tail of a non-averaging step is folded into the next worker pass
   u32 *words, *words_srv, *mask_srv;
   float *scale[2], *scale_srv;
   u32 *tau[2], *tau_srv;
@@ -272,12 +274,18 @@ int flush_tail(sae_handle* h) {
   memset(&sa, 0, sizeof(sa));
   sa.e_srv = h->e_srv; sa.tau_cur = h->tau[h->last]; sa.status = h->status;
   sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0;
-  sa.m = h->m; sa.ebar_in = ebar_other(h); sa.ebar = ebar_now(h); sa.eta = h->eta_prev;
+  sa.m = h->m; sa.ebar_in = ebar_other(h); sa.ebar = ebar_now(h); sa.eta = h->eta_prev; sa.D = h->D;
   sa.x = h->x; sa.mask_srv = h->mask_srv;
   const int lsrv = h->srv_pending ? (dc ? 2 : 1) : 0;
-  if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 0>), P.ntiles, P, sa);
-  else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 1>), P.ntiles, P, sa);
-  else LAUNCH_DENSE(h, (k_server_dense<2, true, true, 2>), P.ntiles, P, sa);
+  if (h->topk_nod) {
+    if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 0>), P.ntiles, P, sa);
+    else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, true, true, 1>), P.ntiles, P, sa);
+    else LAUNCH_DENSE(h, (k_server_dense<2, true, true, 2>), P.ntiles, P, sa);
+  } else {                                     // stored differences, a step whose pre-step does not average
+    if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 0>), P.ntiles, P, sa);
+    else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 1>), P.ntiles, P, sa);
+    else LAUNCH_DENSE(h, (k_server_dense<2, false, false, 2>), P.ntiles, P, sa);
+  }
   if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
   h->srv_pending = 1;
   h->tail_pending = 0;
@@ -372,16 +380,17 @@ bool make_row_map(CUtensorMap* map, const float* base, long long inner, int rows
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int K, bool WD, bool TOPK = false>
+template <int K, bool WD, int MODE = 0>
 void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, const CUtensorMap& tm_g) {
-  constexpr size_t kFusedSmem = sizeof(FwSmemT<K, TOPK>) + 128;
+  constexpr size_t kFusedSmem = sizeof(FwSmemT<K, MODE>) + 128;
   static_assert(kFusedSmem <= 227 * 1024, "the ring must fit the shared memory of one block");
   static thread_local int configured_device = -1;
   if (configured_device != h->device) {
-    cudaFuncSetAttribute(k_worker_fused<K, WD, TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
+    cudaFuncSetAttribute(k_worker_fused<K, WD, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmem);
     configured_device = h->device;
   }
-  const long long nitems = (long long)h->P.ntiles * FwGeom<K>::SUB;
+  typedef FwGeom<K, MODE> G;
+  const long long nitems = (long long)h->P.ntiles * G::SUB;
   long long grid = h->persistent_blocks / SAE_WT_BLOCKS_PER_SM;      // one block per SM
   if (nitems < grid) grid = nitems;
   // Runs of one plan tile per block when the tensors are short (block-wise compression: a few tiles each) and
@@ -389,10 +398,11 @@ void launch_fused_kw(sae_handle* h, const StepParams& sp, const FusedArgs& fa, c
   // out one by one (runs cost 4-5 % there).
   const bool short_tensors = h->P.ntiles < 4LL * h->P.T;
   int chunk_log2 = 0;
-  if (short_tensors && nitems >= 8 * grid * FwGeom<K>::SUB)
-    while ((1 << chunk_log2) < FwGeom<K>::SUB) ++chunk_log2;
+  if (short_tensors && nitems >= 8 * grid * G::SUB)
+    while ((1 << chunk_log2) < G::SUB) ++chunk_log2;
   LaunchScope ls(h, S_WORKER);
-  k_worker_fused<K, WD, TOPK><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, chunk_log2, h->tm_m, tm_g);
+  k_worker_fused<K, WD, MODE><<<(unsigned)grid, FW_THREADS, kFusedSmem, h->stream>>>(h->P, sp, fa, nitems, chunk_log2, h->tm_m, tm_g,
+                                                                                      MODE == 2 ? h->tm_D : h->tm_m);
 }
 
 template <int K>
@@ -400,14 +410,19 @@ void launch_fused_k(sae_handle* h, const StepParams& sp, const FusedArgs& fa, co
   if (sp.wd) launch_fused_kw<K, true>(h, sp, fa, tm_g); else launch_fused_kw<K, false>(h, sp, fa, tm_g);
 }
 
-void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa, bool topk = false) {
+void launch_fused(sae_handle* h, const StepParams& sp, FusedArgs fa, int mode = 0) {
   // the gradients live in the caller's buffer: encode their tensor map for this step (host-only work)
   CUtensorMap tm_g;
   memset(&tm_g, 0, sizeof(tm_g));
   fa.g_tma_ok = make_row_map(&tm_g, fa.g, h->P.d, h->P.K, h->P.d) ? 1 : 0;
-  if (topk) {                          // (K = 8 or 16, no weight decay: checked by the caller)
-    if (h->P.K == 8) launch_fused_kw<8, false, true>(h, sp, fa, tm_g);
-    else launch_fused_kw<16, false, true>(h, sp, fa, tm_g);
+  if (mode == 1) {                     // (K = 8 or 16, no weight decay: checked by the caller)
+    if (h->P.K == 8) launch_fused_kw<8, false, 1>(h, sp, fa, tm_g);
+    else launch_fused_kw<16, false, 1>(h, sp, fa, tm_g);
+    return;
+  }
+  if (mode == 2) {
+    if (h->P.K == 8) launch_fused_kw<8, false, 2>(h, sp, fa, tm_g);
+    else launch_fused_kw<16, false, 2>(h, sp, fa, tm_g);
     return;
   }
   fa.ebar_out = fa.ebar;
@@ -536,21 +551,25 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // the server lines wait for the next dense server pass unless the worker pass needs x (weight decay)
     const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
     if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
-    const int lsrv = h->srv_pending ? (dc ? 2 : 1) : 0;
+    int lsrv = h->srv_pending ? (dc ? 2 : 1) : 0;
     sa.x = h->x; sa.mask_srv = h->mask_srv;
     DeltaSrc src = stored_rows(h->D);
     if (nod) { src.m = h->m; src.ebar = ebar_now(h); src.eta = lr; src.recompute = 1; }
     // Folded form: this step stops after its threshold select; the rest (aggregation, averaged error, server
     // lines) is done by the next step's worker pass and a parameter-sized server pass behind it.
-    const bool fold = nod && h->fused_topk_ok && lazy_ok;
+    // With stored differences (p != 1) the same holds for the steps whose pre-step does not average: the next
+    // worker pass reads the stored rows anyway (it forms e^(k) = D - C(D) from them).
+    const bool fold = lazy_ok && h->local_steps <= 1 &&
+                      (nod ? h->fused_topk_ok != 0 : (h->fused_gen_ok && !avg_after));
+    bool worker_done = false;
     if (h->tail_pending) {
-      if (!fold) return SAE_ERR_INVALID_ARG;
+      if (!lazy_ok || (!nod && h->esrc != ESRC_LAZY_TOPK)) return SAE_ERR_INVALID_ARG;
       FusedArgs fa;
       memset(&fa, 0, sizeof(fa));
-      fa.g = grads; fa.m = h->m; fa.ebar = ebar_other(h); fa.ebar_out = ebar_now(h); fa.x = h->x;
+      fa.g = grads; fa.m = h->m; fa.ebar = ebar_other(h); fa.ebar_out = ebar_now(h); fa.x = h->x; fa.D = h->D;
       fa.tau_prev = h->tau[h->last]; fa.ssum = h->ssum; fa.cand = wa.cand; fa.status = h->status;
       fa.eta_prev = h->eta_prev;
-      launch_fused(h, sp, fa, true);
+      launch_fused(h, sp, fa, nod ? 1 : 2);
       topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
       sa.ssum = h->ssum;
       if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 0, true>), P.ntiles, P, sa);
@@ -558,16 +577,20 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
       else LAUNCH_DENSE(h, (k_server_dense<2, false, false, 2, true>), P.ntiles, P, sa);
       if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
       h->srv_pending = 1;                    // the previous step's server lines now wait for the next server pass
-      h->last = cur; h->eta_prev = lr; h->t += 1;
-      return check_launch(h);
+      h->tail_pending = 0;
+      lsrv = dc ? 2 : 1;
+      worker_done = true;
     }
-    if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
-    else if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
-    else if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true, true>(h, sp, wa);
-    else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
-    topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
-    if (fold) {                              // first folded step: nothing to catch up with, the tail stays open
+    if (!worker_done) {
+      if (nod) launch_worker<ESRC_UNIFORM, false, false, true>(h, sp, wa);
+      else if (h->esrc == ESRC_UNIFORM) launch_worker<ESRC_UNIFORM, false, true, true>(h, sp, wa);
+      else if (h->esrc == ESRC_LOCAL_D) launch_worker<ESRC_LOCAL_D, false, true, true>(h, sp, wa);
+      else launch_worker<ESRC_LAZY_TOPK, false, true, true>(h, sp, wa);
+      topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+    }
+    if (fold) {                              // this step's own tail stays open for the next worker pass
       h->tail_pending = 1;
+      h->esrc = avg_after ? ESRC_UNIFORM : ESRC_LAZY_TOPK;
       h->last = cur; h->eta_prev = lr; h->t += 1;
       return check_launch(h);
     }
@@ -827,7 +850,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
   h->fused_topk_ok = (h->topk_nod && (K == 8 || K == 16) && dpad < (1ll << 31) && d < (1ll << 31)) ? 1 : 0;
   h->tail_pending = 0;
-  if (h->fused_topk_ok) ALLOC0(h->ssum, dpad);
+  h->fused_gen_ok = (!shard && topk && cfg->avg_period != 1 && (K == 8 || K == 16) && dpad < (1ll << 31) &&
+                     d < (1ll << 31)) ? 1 : 0;
+  if (h->fused_topk_ok || h->fused_gen_ok) ALLOC0(h->ssum, dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);
   ALLOC0(h->mask_srv, topk ? nwords : 0);
@@ -885,6 +910,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   }
 #undef TRY
   if (rc == SAE_OK && h->fused_topk_ok && !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_topk_ok = 0;
+  if (rc == SAE_OK && h->fused_gen_ok &&
+      !(h->m && h->D && make_row_map(&h->tm_m, h->m, dpad, K, dpad) && make_row_map(&h->tm_D, h->D, dpad, K, dpad)))
+    h->fused_gen_ok = 0;
   if (rc == SAE_OK && h->fused_ok) {
     // the folded-averaging pass needs a tensor map over the momentum rows and 32-bit TMA coordinates
     if (dpad >= (1ll << 31) || d >= (1ll << 31) || !make_row_map(&h->tm_m, h->m, dpad, K, dpad)) h->fused_ok = 0;

@@ -49,14 +49,18 @@ constexpr int fw_stages(int K) { return fw_split(K) ? 6 : 3; }
 constexpr int fw_tilef(int K) { return (fw_mbuf(K) / fw_kh(K)) < FW_MAXTILE ? (fw_mbuf(K) / fw_kh(K)) : FW_MAXTILE; }
 constexpr int fw_box(int K) { return fw_tilef(K) < FW_MAXBOX ? fw_tilef(K) : FW_MAXBOX; }
 
-template <int K>
+// MODE 0: scaled sign (folded averaging); 1: Top-K with p = 1 (folded tail, differences not stored);
+// 2: Top-K with stored differences (folded tail; a stage carries three arrays -- momentum, gradient and
+// stored difference rows -- so the stages are 3 x 16 KB and there are four of them).
+template <int K, int MODE = 0>
 struct FwGeom {
   static constexpr int HALVES = fw_halves(K);                 // items per element range
   static constexpr int KH = fw_kh(K);                         // workers per item
-  static constexpr int MBUF = fw_mbuf(K);
-  static constexpr int STAGES = fw_stages(K);
-  static constexpr int TILEF = fw_tilef(K);                   // elements per item
-  static constexpr int BOX = fw_box(K);                       // inner extent of the TMA boxes
+  static constexpr int MBUF = MODE == 2 ? 4096 : fw_mbuf(K);
+  static constexpr int STAGES = MODE == 2 ? 4 : fw_stages(K);
+  static constexpr int TILEF = (MBUF / KH) < FW_MAXTILE ? (MBUF / KH) : FW_MAXTILE;   // elements per item
+  static constexpr int BOX = TILEF < FW_MAXBOX ? TILEF : FW_MAXBOX;                  // inner extent of the TMA boxes
+  static_assert(BOX == fw_box(K), "one tensor map per array serves every mode");
   static constexpr int SUB = TILE / TILEF;                    // element ranges per 4096-element plan tile
   static constexpr int ROWS_PER_WORKER = TILEF / 128;
   static constexpr int RPW = KH * ROWS_PER_WORKER / FW_WARPS; // 128-element rows per warp and item
@@ -85,11 +89,13 @@ struct FwItem {
   int h;             // which group of KH workers
 };
 
-template <int K, bool TOPK = false>
+template <int K, int MODE = 0>
 struct FwSmemT {
-  typedef FwGeom<K> G;
+  typedef FwGeom<K, MODE> G;
+  static constexpr bool TOPK = MODE != 0;
   alignas(128) float m[G::STAGES][G::MBUF];
   alignas(128) float g[G::STAGES][G::MBUF];
+  alignas(128) float dd[MODE == 2 ? G::STAGES : 1][MODE == 2 ? G::MBUF : 32];   // stored differences (MODE 2)
   alignas(128) float e[G::STAGES][G::TILEF];
   alignas(8) u64 full[G::STAGES];
   alignas(8) u64 empty[G::STAGES];
@@ -105,6 +111,7 @@ struct FusedArgs {
   float* ebar;             // in: ebar of the previous step
   float* ebar_out;         // out: the averaged error of this pre-step (scaled sign: the same buffer)
   const u32* tau_prev;     // Top-K: [K][T] thresholds of the previous step
+  float* D;                // Top-K with stored differences: [K][dpad] in: last step's, out: this step's
   float* ssum;             // Top-K: [dpad] out: sum_k C(Delta^(k)) of the previous step, k in order, not divided by K
   CandArgs cand;           // Top-K: candidate lists for this step's differences
   const float* x;
@@ -116,9 +123,9 @@ struct FusedArgs {
   int g_tma_ok;            // the gradient buffer admits a tensor map (16-byte aligned base and row pitch)
 };
 
-template <int K>
+template <int K, int MODE>
 __device__ __forceinline__ FwItem fw_lookup(const Plan& P, int g_tma_ok, long long w, long long nitems) {
-  typedef FwGeom<K> G;
+  typedef FwGeom<K, MODE> G;
   FwItem it;
   it.pbase = 0; it.goff = 0; it.j = 0; it.cnt = 0; it.gvec = 0; it.h = 0;
   if (w >= nitems) { it.cnt = -1; return it; }
@@ -157,14 +164,16 @@ __device__ __forceinline__ int fw_ranges_of_block(long long nitems, int chunk_lo
 // selected entries (the aggregation of the server line: it needs the same rows in the same order), which a
 // parameter-sized server pass then only reads; the workers collect this step's candidate keys instead of L1
 // partials and sign bits.  The differences are never stored.
-template <int K, bool WD, bool TOPK = false>
+template <int K, bool WD, int MODE = 0>
 __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepParams sp, FusedArgs A, long long nitems,
                                                                  int chunk_log2,
                                                                  const __grid_constant__ CUtensorMap tm_m,
-                                                                 const __grid_constant__ CUtensorMap tm_g) {
-  typedef FwGeom<K> G;
+                                                                 const __grid_constant__ CUtensorMap tm_g,
+                                                                 const __grid_constant__ CUtensorMap tm_d) {
+  typedef FwGeom<K, MODE> G;
+  constexpr bool TOPK = MODE != 0, GEN = MODE == 2;
   extern __shared__ unsigned char smem_raw[];
-  typedef FwSmemT<K, TOPK> Smem;
+  typedef FwSmemT<K, MODE> Smem;
   static_assert(!TOPK || (G::WPW == 1 && G::HALVES == 1), "Top-K form: a worker warp serves one worker");
   constexpr int FW_STAGES = G::STAGES;
   constexpr int FW_BOX = G::BOX;
@@ -182,10 +191,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   if (warp == FW_WARPS) {
     // ---------------- producer ----------------
     // nitems counts element ranges; each is issued as HALVES consecutive items (one per group of KH workers)
-    FwItem nxt = fw_lookup<K>(P, A.g_tma_ok, fw_range_of(lane, chunk_log2), nitems);
+    FwItem nxt = fw_lookup<K, MODE>(P, A.g_tma_ok, fw_range_of(lane, chunk_log2), nitems);
     for (int p0 = 0; p0 < nmine; p0 += 32) {
       const FwItem cur = nxt;
-      nxt = fw_lookup<K>(P, A.g_tma_ok, fw_range_of(p0 + 32 + lane, chunk_log2), nitems);
+      nxt = fw_lookup<K, MODE>(P, A.g_tma_ok, fw_range_of(p0 + 32 + lane, chunk_log2), nitems);
       for (int l = 0; l < 32; ++l) {
         // the range of lane l, broadcast so that the lanes can share the issue of its copies
         const int cnt = __shfl_sync(0xffffffffu, cur.cnt, l);
@@ -217,13 +226,14 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           if (cnt == 0) {
             if (lane == 0) mbar_arrive(&S.full[s]);
           } else if (lane == 0) {
-            const u32 ebytes = (hh == 0) ? (u32)((cnt + 31) & ~31) * 4u : 0u;    // rows are padded to 32 elements
+            const u32 ebytes = (hh == 0 && !GEN) ? (u32)((cnt + 31) & ~31) * 4u : 0u;    // rows are padded to 32 elements
             const int chunks = (cnt + FW_BOX - 1) / FW_BOX;
             constexpr u32 BOXB = (u32)(G::KH * FW_BOX * 4);
-            mbar_arrive_expect_tx(&S.full[s], ebytes + (u32)chunks * BOXB * (gtma ? 2u : 1u));
-            if (hh == 0) bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);  // the old ebar travels with the first group
+            mbar_arrive_expect_tx(&S.full[s], ebytes + (u32)chunks * BOXB * ((gtma ? 2u : 1u) + (GEN ? 1u : 0u)));
+            if (hh == 0 && !GEN) bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);  // the old ebar travels with the first group
             for (int c = 0; c < chunks; ++c) {
               tma_load_2d(&S.m[s][c * G::KH * FW_BOX], &tm_m, (int)pbase + c * FW_BOX, hh * G::KH, &S.full[s]);
+              if (GEN) tma_load_2d(&S.dd[s][c * G::KH * FW_BOX], &tm_d, (int)pbase + c * FW_BOX, hh * G::KH, &S.full[s]);
               if (gtma) tma_load_2d(&S.g[s][c * G::KH * FW_BOX], &tm_g, (int)goff + c * FW_BOX, hh * G::KH, &S.full[s]);
             }
           }
@@ -257,7 +267,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       }
       const FwItem it = S.item[s];
       if (it.cnt > 0) {
-        const float* sm = S.m[s];
+        const float* sm = GEN ? S.dd[s] : S.m[s];           // (MODE 2: the stored differences themselves)
         const float* se0 = S.e[(i - hh) % FW_STAGES];       // the first group's stage holds the old ebar
         const float* sc = S.sc[s];
 #pragma unroll
@@ -266,15 +276,17 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           if (e0 < it.cnt) {
             if (hh == 0) {
 #pragma unroll
-              for (int v = 0; v < V; ++v) { eb[c][v] = se0[e0 + v]; a[c][v] = 0.0f; s2[c][v] = 0.0f; }
+              for (int v = 0; v < V; ++v) { eb[c][v] = GEN ? 0.0f : se0[e0 + v]; a[c][v] = 0.0f; s2[c][v] = 0.0f; }
             }
 #pragma unroll
             for (int k = 0; k < G::KH; ++k) {
               const float sk = sc[k];
 #pragma unroll
               for (int v = 0; v < V; ++v) {
-                const float dk = __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[c][v]);
-                if (TOPK) {
+                const float dk = GEN ? sm[G::idx(k, e0) + v] : __fmaf_rn(A.eta_prev, sm[G::idx(k, e0) + v], eb[c][v]);
+                if (GEN) {
+                  s2[c][v] = __fadd_rn(s2[c][v], topk_selected(dk, __float_as_uint(sk)) ? dk : 0.0f);
+                } else if (TOPK) {
                   const float ck = topk_selected(dk, __float_as_uint(sk)) ? dk : 0.0f;
                   a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, ck));
                   s2[c][v] = __fadd_rn(s2[c][v], ck);
@@ -287,10 +299,12 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
 #pragma unroll
               for (int v = 0; v < V; ++v) {
                 if (e0 + v < it.cnt) {
-                  const float en = div_by_k(P, a[c][v]);
+                  if (!GEN) {
+                    const float en = div_by_k(P, a[c][v]);
 #pragma unroll
-                  for (int hq = 0; hq < G::HALVES; ++hq) S.e[(i - hh + hq) % FW_STAGES][e0 + v] = en;
-                  A.ebar_out[it.pbase + e0 + v] = en;
+                    for (int hq = 0; hq < G::HALVES; ++hq) S.e[(i - hh + hq) % FW_STAGES][e0 + v] = en;
+                    A.ebar_out[it.pbase + e0 + v] = en;
+                  }
                   if (TOPK) A.ssum[it.pbase + e0 + v] = s2[c][v];
                 }
               }
@@ -343,7 +357,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       const float* sm = S.m[s];
       const float* sg = S.g[s];
       const float* se = S.e[s];
-      // ebar' of this range comes from the averager warps
+      const float* sd = S.dd[GEN ? s : 0];
+      const u32 tk = TOPK ? __float_as_uint(S.sc[s][kl0]) : 0u;
+      // ebar' of this range comes from the averager warps (MODE 2: nothing is handed over, but the averagers
+      // must be done with the stage before the workers release it)
       if (!mbar_wait(&S.avgd[s], (i / FW_STAGES) & 1)) {
         if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
         return;
@@ -356,13 +373,21 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         const int k = hh * G::KH + kl;
         const int a = hh * G::WPW + ((G::WPW == 1) ? 0 : (kl - kl0));
         float* mp = A.m + (long long)k * P.dpad + it.pbase;
+        float* dp = A.D + (long long)k * P.dpad + it.pbase;                        // (MODE 2)
         u32* wp = A.words + (long long)k * P.nwords + (it.pbase >> 5);
         const int rbase = G::idx(kl, rr * 128);                // the row's position in the stage buffers
         if (it.gvec && rr * 128 + 128 <= it.cnt) {
           const int e0 = rr * 128 + lane * 4;
           const float4 Gq = *reinterpret_cast<const float4*>(sg + rbase + lane * 4);
           const float4 M = *reinterpret_cast<const float4*>(sm + rbase + lane * 4);
-          const float4 E = *reinterpret_cast<const float4*>(se + e0);
+          float4 E;
+          if (GEN) {                             // e^(k) = D - C(D) with last step's threshold, formed on the fly
+            const float4 Dv = *reinterpret_cast<const float4*>(sd + rbase + lane * 4);
+            E.x = prev_error<ESRC_LAZY_TOPK>(Dv.x, 0.0f, tk); E.y = prev_error<ESRC_LAZY_TOPK>(Dv.y, 0.0f, tk);
+            E.z = prev_error<ESRC_LAZY_TOPK>(Dv.z, 0.0f, tk); E.w = prev_error<ESRC_LAZY_TOPK>(Dv.w, 0.0f, tk);
+          } else {
+            E = *reinterpret_cast<const float4*>(se + e0);
+          }
           float4 X = make_float4(0.f, 0.f, 0.f, 0.f);
           if (WD) X = ld4(A.x + it.pbase + e0);
           float4 mn, dl;
@@ -371,6 +396,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           dl.z = worker_update<WD>(Gq.z, M.z, E.z, X.z, sp, mn.z);
           dl.w = worker_update<WD>(Gq.w, M.w, E.w, X.w, sp, mn.w);
           st4(mp + e0, mn);
+          if (GEN) st4(dp + e0, dl);
           if (TOPK) {
             if (lo != NO_GUESS) {
               if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand, kl0, stg_j);
@@ -394,8 +420,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
               const float xv = WD ? A.x[it.pbase + e] : 0.0f;
               const float gv = it.gvec ? sg[rbase + c * 32 + lane] : __ldcs(gp + e);
               float mn;
-              dl = worker_update<WD>(gv, sm[rbase + c * 32 + lane], se[e], xv, sp, mn);
+              const float ev = GEN ? prev_error<ESRC_LAZY_TOPK>(sd[rbase + c * 32 + lane], 0.0f, tk) : se[e];
+              dl = worker_update<WD>(gv, sm[rbase + c * 32 + lane], ev, xv, sp, mn);
               mp[e] = mn;
+              if (GEN) dp[e] = dl;
               if (!TOPK) {
                 if (G::NACC == 1 || a == 0) lane_add(acc[0], dl);
                 else lane_add(acc[G::NACC - 1], dl);

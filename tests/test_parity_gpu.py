@@ -458,22 +458,30 @@ def test_pending_server_lines_survive_a_checkpoint_and_a_side_stream():
 @pytest.mark.parametrize("K", [8, 16])
 @pytest.mark.parametrize("dc", [0, 1])
 @pytest.mark.parametrize("every", [1, 2, 5])
-def test_topk_folded_tail(K, dc, every):
-    """Top-K, p = 1, K = 8 or 16, no weight decay: a step stops after its threshold select and the next step's
-    worker pass does the rest; a getter in between carries the open tail out the unfolded way.  Looking at
-    the state every step, every second step and every fifth step mixes both forms in every order."""
-    run_pair(K, RAGGED + [40000], so.TOPK, 11, p=1, dc=dc, seed=11, lrs=[0.1, 0.05, 0.2], every=every, num=1, den=20,
+@pytest.mark.parametrize("p", [1, 0, 3])
+def test_topk_folded_tail(K, dc, every, p):
+    """Top-K, K = 8 or 16, no weight decay: a step (with p != 1: one whose pre-step does not average) stops
+    after its threshold select and the next step's worker pass does the rest; a getter in between carries
+    the open tail out the unfolded way.  Looking at the state every step, every second step and every fifth
+    step mixes both forms in every order."""
+    run_pair(K, RAGGED + [40000], so.TOPK, 11, p=p, dc=dc, seed=11, lrs=[0.1, 0.05, 0.2], every=every, num=1, den=20,
              outliers=(66, 100.0))
 
 
+@pytest.mark.parametrize("mode,mu", [(so.EF, 0.9), (so.SAEF, 0.5)])
+def test_topk_folded_tail_branches(mode, mu):
+    run_pair(8, RAGGED + [40000], so.TOPK, 9, p=0, mode=mode, mu=mu, seed=13, every=4, num=1, den=10, outliers=(66, 100.0))
+
+
 @pytest.mark.parametrize("K", [8, 16])
-def test_topk_folded_tail_graph_replay_and_checkpoint(K):
+@pytest.mark.parametrize("p", [1, 0, 4])
+def test_topk_folded_tail_graph_replay_and_checkpoint(K, p):
     import torch
     sizes = RAGGED + [40000]
     d = int(np.sum(sizes))
     scales = synth.tensor_scales(12, len(sizes), -4.0, -1.0)
     x0 = synth.x0_numpy(12, d)
-    kw = dict(compressor=so.TOPK, avg_period=1, momentum=0.9, topk_num=1, topk_den=20)
+    kw = dict(compressor=so.TOPK, avg_period=p, momentum=0.9, topk_num=1, topk_den=20)
     orc = so.Oracle(K, sizes, x0, threads=4, **kw)
     with torch.cuda.stream(torch.cuda.Stream()):          # graph replay: the open tail is part of the graph key
         a = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
