@@ -27,8 +27,8 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm, tail; const float* grads; float lr, eta_prev; };
-struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after, tail_after; uint64_t stamp; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm, tail, fresh; const float* grads; float lr, eta_prev; };
+struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after, tail_after, fresh_after; uint64_t stamp; };
 
 }  // namespace
 
@@ -97,7 +97,8 @@ struct sae_handle {
   // Top-K, p = 1, K = 8 or 16, no weight decay: the tail of a step (worker-axis aggregation, averaged error,
   // server lines) is left to the worker pass of the next step, which reads the same momentum rows anyway
   int fused_topk_ok;
-  int tail_pending;                 // the last step stopped after its threshold select
+  int tail_pending;                 // the last step stopped after its threshold select (scaled sign: after its scales)
+  int recs_srv_fresh;               // a server pass has added to the server's L1 records since they were last finalized
   float* ssum;                      // [dpad] ordered worker-axis sum of the selected entries (folded form)
   int avg_external;                 // the averaging sum is all-reduced by the caller instead of pulled in k order
   int avg_owed;                     // ... and is owed before the next sae_step_begin
@@ -272,6 +273,26 @@ int flush_tail(sae_handle* h) {
   const bool dc = h->cfg.server_compress != 0;
   ServerArgs sa;
   memset(&sa, 0, sizeof(sa));
+  if (h->cfg.compressor == SAE_COMPRESSOR_SIGN) {
+    // scaled sign, p = 1: the open tail is the server pass over the last step's message words (still in place)
+    const bool pending = h->srv_pending != 0;
+    LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.T + THREADS - 1) / THREADS, 0, P.T, h->d_n, h->recs, h->scale[h->last],
+           h->recs_srv, (pending && dc && h->recs_srv_fresh) ? h->scale_srv : nullptr);
+    sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[h->last]; sa.words_srv = h->words_srv;
+    sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status; sa.x = h->x;
+    sa.scale_srv_prev = h->scale_srv;
+    const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
+    const int nblk = (P.ntiles + tpb - 1) / tpb;
+    if (pending) {
+      if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, true>), nblk, P, sa, tpb);
+      else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, true>), nblk, P, sa, tpb);
+    } else if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
+    else LAUNCH(h, S_SERVER, k_server_sign<false>, nblk, P, sa, tpb);
+    h->recs_srv_fresh = 1;
+    h->srv_pending = 1;
+    h->tail_pending = 0;
+    return check_launch(h);
+  }
   sa.e_srv = h->e_srv; sa.tau_cur = h->tau[h->last]; sa.status = h->status;
   sa.cand_srv = cand_args(h, true); sa.tau_srv_prev = h->tau_srv; sa.emit_srv = dc ? 1 : 0;
   sa.m = h->m; sa.ebar_in = ebar_other(h); sa.ebar = ebar_now(h); sa.eta = h->eta_prev; sa.D = h->D;
@@ -497,10 +518,23 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     if (write_d && !h->D) return SAE_ERR_INVALID_ARG;
     // p = 1: the average is not formed here but at the head of the next worker pass
     const bool defer_avg = avg_after && !write_d && h->fused_ok;
+    // The server lines of this step can be left to the next step's server pass when nothing in between
+    // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
+    const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
+    // Folded form (p = 1 steady state, large problems): the whole server pass of this step stays open -- the
+    // next step's worker pass re-forms every message C(Delta^(k)) in its averager warps anyway and adds them up
+    // in k order on the way; a streaming server pass then only reads that sum.
+    // (Worth it from 32 workers on: the unpacking server pass costs K additions per parameter, the streaming
+    // one and the extra vector the worker pass writes do not depend on K -- config 4: 7.82 -> 7.62 ms per step,
+    // config 2 with 16 workers: 0.928 -> 0.938.)
+    const bool fold_sign = defer_avg && lazy_ok && !h->inline_fin && h->local_steps <= 1 && h->ssum != nullptr;
+    if (h->tail_pending && !(pending_in && fold_sign)) return SAE_ERR_INVALID_ARG;
     if (pending_in) {
       FusedArgs fa;
+      memset(&fa, 0, sizeof(fa));
       fa.g = grads; fa.m = h->m; fa.ebar = ebar_now(h); fa.x = h->x; fa.scale_prev = h->scale[h->last];
       fa.words = h->words; fa.recs = recs_now; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
+      fa.ssum = h->tail_pending ? h->ssum : nullptr;
       launch_fused(h, sp, fa);
     } else if (h->esrc == ESRC_UNIFORM) {
       if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
@@ -510,18 +544,35 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
-    // The server lines of this step can be left to the next step's server pass when nothing in between
-    // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
-    const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
     if (h->srv_pending && !lazy_ok) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
     const bool pending = h->srv_pending != 0;
-    if (!h->inline_fin)
+    if (!h->inline_fin) {
       LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.K * P.T + P.T + THREADS - 1) / THREADS, P.K, P.T, h->d_n, h->recs,
-             h->scale[cur], h->recs_srv, (pending && dc) ? h->scale_srv : nullptr);
+             h->scale[cur], h->recs_srv, (pending && dc && h->recs_srv_fresh) ? h->scale_srv : nullptr);
+      h->recs_srv_fresh = 0;
+    }
     sa.x = h->x; sa.scale_srv_prev = h->scale_srv;
     // consecutive tiles per block: enough blocks to fill the device several times over, at most 8 tiles each
     const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
     const int nblk = (P.ntiles + tpb - 1) / tpb;
+    if (h->tail_pending) {                        // the previous step's server pass, from the sum
+      sa.ssum = h->ssum;
+      if (pending) {
+        if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, true, true>), nblk, P, sa, tpb);
+        else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, true, true>), nblk, P, sa, tpb);
+      } else if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, false, true>), nblk, P, sa, tpb);
+      else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, false, true>), nblk, P, sa, tpb);
+      h->recs_srv_fresh = 1;
+      h->srv_pending = 1;                         // its server lines wait for the next server pass
+      h->tail_pending = 0;
+    }
+    if (fold_sign) {                              // this step's own server pass stays open
+      h->tail_pending = 1;
+      h->esrc = ESRC_PENDING_AVG;
+      h->last = cur; h->eta_prev = lr; h->t += 1;
+      return check_launch(h);
+    }
+    h->recs_srv_fresh = 1;                        // (the server pass below adds to the records)
     if (h->inline_fin) {
       if (pending) {
         if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, true, true>), nblk, P, sa, tpb);
@@ -646,17 +697,17 @@ int do_step(sae_handle* h, const float* grads, float lr) {
 
   StepGraphKey key;
   key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending; key.rot = h->rot;
-  key.comm = communicates(h) ? 1 : 0; key.tail = h->tail_pending;
+  key.comm = communicates(h) ? 1 : 0; key.tail = h->tail_pending; key.fresh = h->recs_srv_fresh;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.tail == key.tail && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.tail == key.tail && e.key.fresh == key.fresh && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
       h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->rot = e.rot_after;
-      h->tail_pending = e.tail_after;
+      h->tail_pending = e.tail_after; h->recs_srv_fresh = e.fresh_after;
       h->eta_prev = lr; h->t += 1;
       e.stamp = ++h->graph_clock;
       h->graph_misses = 0;
@@ -679,7 +730,7 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   StepGraph e;
   e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
   e.esrc_after = h->esrc; e.last_after = h->last; e.pending_after = h->srv_pending; e.rot_after = h->rot;
-  e.tail_after = h->tail_pending;
+  e.tail_after = h->tail_pending; e.fresh_after = h->recs_srv_fresh;
   e.stamp = ++h->graph_clock;
   ce = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
@@ -849,10 +900,12 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
   if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
   h->fused_topk_ok = (h->topk_nod && (K == 8 || K == 16) && dpad < (1ll << 31) && d < (1ll << 31)) ? 1 : 0;
-  h->tail_pending = 0;
+  h->tail_pending = 0; h->recs_srv_fresh = 0;
   h->fused_gen_ok = (!shard && topk && cfg->avg_period != 1 && (K == 8 || K == 16) && dpad < (1ll << 31) &&
                      d < (1ll << 31)) ? 1 : 0;
-  if (h->fused_topk_ok || h->fused_gen_ok) ALLOC0(h->ssum, dpad);
+  // (scaled sign: the folded server pass is for large problems, p = 1, K a power of two up to 32)
+  const bool sign_fold = h->fused_ok && K >= 32 && (long long)K * dpad > (1ll << 24);
+  if (h->fused_topk_ok || h->fused_gen_ok || sign_fold) ALLOC0(h->ssum, dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);
   ALLOC0(h->mask_srv, topk ? nwords : 0);
@@ -1356,7 +1409,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
   }
   h->t = hd.t; h->esrc = hd.esrc; h->last = hd.last; h->eta_prev = hd.eta_prev;
   h->srv_pending = 0;        // a checkpoint is taken with the server lines carried out
-  h->tail_pending = 0;
+  h->tail_pending = 0; h->recs_srv_fresh = 0;
   if (h->inline_fin) {       // the L1 records are transient, but nothing else clears them before the next step
     SAE_CUDA(h, cudaMemsetAsync(h->recs, 0, sizeof(L1Record) * (size_t)h->P.K * h->P.T, h->stream));
     SAE_CUDA(h, cudaMemsetAsync(h->recs_srv, 0, sizeof(L1Record) * (size_t)h->P.T, h->stream));

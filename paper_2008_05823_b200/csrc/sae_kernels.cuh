@@ -138,7 +138,10 @@ __device__ __forceinline__ u64 add_f32x2(u64 a, u64 b) {
 // Staging (all but FIN): a full tile's server error (LAZY: and parameters) is fetched by one bulk
 // asynchronous copy (TMA) into shared memory when the block reaches the tile and is first read after the
 // worker loop, so that its memory latency passes under the loop without holding registers for it.
-template <bool DC, bool TABLE = false, bool FIN = false, bool LAZY = false>
+// SUM (p = 1, folded form): the ordered sum of the workers' messages was already formed by the following step's
+// worker pass (its averager warps add the same +-s_k in the same order) and is only read here: no message
+// words, no worker loop -- a plain streaming pass.
+template <bool DC, bool TABLE = false, bool FIN = false, bool LAZY = false, bool SUM = false>
 __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, int tiles_per_block) {
   __shared__ float s_k[MAX_WORKERS];
   __shared__ float sh_s_old;
@@ -166,7 +169,7 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
     if (ti.j != cur_j) {
       if (DC && cur_j >= 0) { warp_commit(acc, A.recs_srv + cur_j, A.status); lane_acc_init(acc); }
       __syncthreads();                            // the previous tensor's scales are no longer read
-      for (int k = tid; k < P.K; k += THREADS) {
+      for (int k = tid; k < (SUM ? 0 : P.K); k += THREADS) {
         if (FIN) {
           const L1Record r = A.recs[(long long)k * P.T + ti.j];
           const float s = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
@@ -220,6 +223,11 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
       // Single-way: the server error is fetched ahead of the worker loop, so that its latency hides under
       // the loop.  (Double-way has enough independent work after the loop; fetching early there only
       // costs registers.)
+      float4 sv[SUM ? SRV_E / 4 : 1];              // (SUM) the tile of the sum: fetched while the staged rows arrive
+      if constexpr (SUM) {
+#pragma unroll
+        for (int q = 0; q < SRV_E / 4; ++q) sv[q] = ld4_stream(A.ssum + pbase + i + 4 * q);
+      }
       float4 ev[(DC || STAGE) ? 1 : SRV_E / 4];
       if constexpr (!DC && !STAGE) {
 #pragma unroll
@@ -232,8 +240,8 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
       u32 wn[SRV_B];
 #pragma unroll
       for (int u = 0; u < SRV_B; ++u)
-        wn[u] = (u < P.K) ? __ldg(TABLE ? s_row[u] + wofs : wk + (long long)u * P.nwords) : 0u;
-      for (int k0 = 0; k0 < P.K; k0 += SRV_B) {
+        wn[u] = (!SUM && u < P.K) ? __ldg(TABLE ? s_row[u] + wofs : wk + (long long)u * P.nwords) : 0u;
+      for (int k0 = 0; k0 < (SUM ? 0 : P.K); k0 += SRV_B) {
         u32 w[SRV_B];
 #pragma unroll
         for (int u = 0; u < SRV_B; ++u) w[u] = wn[u];
@@ -267,8 +275,12 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 #pragma unroll
       for (int q = 0; q < SRV_E / 4; ++q) {
         float a0, a1, a3, a4;
-        unpack2(a2[2 * q], a0, a1);
-        unpack2(a2[2 * q + 1], a3, a4);
+        if constexpr (SUM) {
+          a0 = sv[q].x; a1 = sv[q].y; a3 = sv[q].z; a4 = sv[q].w;
+        } else {
+          unpack2(a2[2 * q], a0, a1);
+          unpack2(a2[2 * q + 1], a3, a4);
+        }
         float4 e;
         if constexpr (STAGE) e = ld4(s_e + i + 4 * q);
         else if constexpr (DC) e = ld4(ep + i + 4 * q);
@@ -308,9 +320,9 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         const bool valid = i < ti.cnt;
         float ds = 0.0f;
         if (valid) {
-          float a = 0.f;
+          float a = SUM ? A.ssum[pbase + i] : 0.f;
           const int wi = i >> 5;
-          for (int k = 0; k < P.K; ++k) {
+          for (int k = 0; k < (SUM ? 0 : P.K); ++k) {
             const u32 w = __ldg(TABLE ? s_row[k] + (pbase >> 5) + wi : wp + (long long)k * P.nwords + wi) >> lane;
             const float s = s_k[k];
             a = __fadd_rn(a, (w & 1u) ? s : -s);

@@ -112,7 +112,8 @@ struct FusedArgs {
   float* ebar_out;         // out: the averaged error of this pre-step (scaled sign: the same buffer)
   const u32* tau_prev;     // Top-K: [K][T] thresholds of the previous step
   float* D;                // Top-K with stored differences: [K][dpad] in: last step's, out: this step's
-  float* ssum;             // Top-K: [dpad] out: sum_k C(Delta^(k)) of the previous step, k in order, not divided by K
+  float* ssum;             // [dpad] out: sum_k C(Delta^(k)) of the previous step, k in order, not divided by K
+                           // (Top-K: always; scaled sign: when not null)
   CandArgs cand;           // Top-K: candidate lists for this step's differences
   const float* x;
   const float* scale_prev; // [K][T] scales of the previous step
@@ -253,7 +254,10 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     constexpr int V = EPT < 4 ? EPT : 4;             // handled in chunks of V consecutive elements
     constexpr int CH = EPT / V;
     const int ta = tid - (FW_WARPS + 1) * 32;
-    float eb[CH][V], a[CH][V], s2[CH][V];          // (s2: Top-K only)
+    // scaled sign: the addends sign_code(...) are the previous step's messages C(Delta^(k)); their ordered sum is
+    // that step's worker-axis aggregation, written out when the caller left that step's server pass open
+    const bool emit_sum = TOPK || A.ssum != nullptr;
+    float eb[CH][V], a[CH][V], s2[CH][V];          // (s2: the ordered sum of the messages)
 #pragma unroll
     for (int c = 0; c < CH; ++c)
 #pragma unroll
@@ -291,7 +295,9 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
                   a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, ck));
                   s2[c][v] = __fadd_rn(s2[c][v], ck);
                 } else {
-                  a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, sign_code(dk, sk)));
+                  const float ck = sign_code(dk, sk);
+                  a[c][v] = __fadd_rn(a[c][v], __fsub_rn(dk, ck));
+                  if (emit_sum) s2[c][v] = __fadd_rn(s2[c][v], ck);
                 }
               }
             }
@@ -305,7 +311,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
                     for (int hq = 0; hq < G::HALVES; ++hq) S.e[(i - hh + hq) % FW_STAGES][e0 + v] = en;
                     A.ebar_out[it.pbase + e0 + v] = en;
                   }
-                  if (TOPK) A.ssum[it.pbase + e0 + v] = s2[c][v];
+                  if (emit_sum) A.ssum[it.pbase + e0 + v] = s2[c][v];
                 }
               }
             }

@@ -501,3 +501,40 @@ def test_topk_folded_tail_graph_replay_and_checkpoint(K, p):
         compare_server_messages(a, orc, so.TOPK, 1, tag="continued")
         compare_server_messages(b, orc, so.TOPK, 1, tag="restored")
         a.close(); b.close()
+
+
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("every", [1, 2, 3])
+def test_sign_folded_server_pass(dc, every):
+    """Scaled sign, p = 1, 32 workers, above the small-problem limit (K * d > 2^24), no weight decay: a step stops after its
+    scales; the next step's worker pass adds the messages up in k order on the way and a streaming server pass
+    reads that sum.  A getter in between runs the open server pass from the message words instead."""
+    run_pair(32, [500_000, 33, 70_000, 4096], so.SIGN, 7, p=1, dc=dc, seed=14, lrs=[0.1, 0.05, 0.2], every=every)
+
+
+def test_sign_folded_server_pass_checkpoint_and_graphs():
+    import torch
+    K, sizes = 32, [550_000, 33, 100_000]
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(15, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(15, d)
+    kw = dict(compressor=so.SIGN, avg_period=1, momentum=0.9)
+    orc = so.Oracle(K, sizes, x0, threads=4, **kw)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        a = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
+        gs = [torch.from_numpy(synth.grads_numpy(15, t, K, sizes, scales)).cuda() for t in range(3)]
+        for t in range(5):
+            orc.step(gs[t % 3].cpu().numpy(), 0.1)
+            a.step(gs[t % 3], 0.1)
+        blob = a.save_state()                             # taken with a server pass open: the save closes it
+        b = sb.Sae(K, sizes, torch.zeros(d, device="cuda"), **kw)
+        b.load_state(blob)
+        for t in range(5, 9):
+            orc.step(gs[t % 3].cpu().numpy(), 0.1)
+            a.step(gs[t % 3], 0.1)
+            b.step(gs[t % 3], 0.1)
+        compare_state(a, orc, so.SIGN, tag="continued")
+        compare_state(b, orc, so.SIGN, tag="restored")
+        compare_server_messages(a, orc, so.SIGN, 1, tag="continued")
+        compare_server_messages(b, orc, so.SIGN, 1, tag="restored")
+        a.close(); b.close()
