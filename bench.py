@@ -34,7 +34,10 @@ FALLBACK_HBM_GBS = 6650.0
 # topk_p1: 1324.2 MB for 4 x 25.56 M worker-elements = 12 B per worker-element + 3.81 B per parameter (ebar);
 # topk_general: 2027.4 MB = 19.83 B per worker-element (candidate lists included);
 # topk_p1_folded: 2765.3 MB for 8 x 25.56 M worker-elements = 12 B per worker-element + 12.18 B per parameter.
+# sign_p1_folded: the sign_p1 capture plus the 4-byte-per-parameter sum vector the folded form writes (derived, not
+# captured: a 32-worker case within the capture size rule does not reach the folded form's size threshold).
 WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0),      # (per worker-element, per parameter)
+                          "sign_p1_folded": (12.0, 10.56),
                           "topk_p1": (12.0, 3.81), "topk_general": (19.83, 0.0),      # profiles/worker_pass_sign_cfg2shapes_4workers.md,
                           "topk_p1_folded": (12.0, 12.18), "mu0": None}                                                # profiles/topk_passes_cfg3shapes_4workers.md
 
@@ -199,8 +202,11 @@ def algorithmic_bytes(w, avg_period):
         # Top-K: g R, m RW | ebar R (Delta is not stored: the server pass recomputes it from m)
         # Top-K with 8 or 16 workers and no weight decay, folded form: ebar R and W, and the worker-axis sum W
         folded = topk and w.num_workers in (8, 16) and w.weight_decay == 0.0
-        worker = (12 * Wd + (12 if folded else 4) * d) if topk else 12 * Wd + 8 * d
-        variant = ("topk_p1_folded" if folded else "topk_p1") if topk else "sign_p1"
+        # scaled sign with 32 workers, no weight decay, above the small-problem limit: the worker pass also writes
+        # the ordered sum of the previous step's messages (the folded server pass)
+        sign_folded = (not topk) and w.num_workers >= 32 and w.weight_decay == 0.0 and Wd > (1 << 24)
+        worker = (12 * Wd + (12 if folded else 4) * d) if topk else 12 * Wd + (12 if sign_folded else 8) * d
+        variant = ("topk_p1_folded" if folded else "topk_p1") if topk else ("sign_p1_folded" if sign_folded else "sign_p1")
     elif w.momentum == 0.0:
         step = 12 * Wd + 16 * d              # g R, e RW | x RW, e_srv RW  (mu = 0: no momentum rows)
         worker = 12 * Wd                     # g R, Delta(e) RW
