@@ -34,10 +34,10 @@ FALLBACK_HBM_GBS = 6650.0
 # topk_p1: 1324.2 MB for 4 x 25.56 M worker-elements = 12 B per worker-element + 3.81 B per parameter (ebar);
 # topk_general: 2027.4 MB = 19.83 B per worker-element (candidate lists included);
 # topk_p1_folded: 2765.3 MB for 8 x 25.56 M worker-elements = 12 B per worker-element + 12.18 B per parameter.
-# sign_p1_folded: the sign_p1 capture plus the 4-byte-per-parameter sum vector the folded form writes (derived, not
-# captured: a 32-worker case within the capture size rule does not reach the folded form's size threshold).
+# sign_p1_folded: 43.752 GB for 32 x 109.48 M worker-elements, captured on config 4 itself with one-pass metrics
+# (profiles/worker_and_server_pass_cfg4_dram_bytes.md) = 12 B per worker-element + 15.63 B per parameter.
 WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0),      # (per worker-element, per parameter)
-                          "sign_p1_folded": (12.0, 10.56),
+                          "sign_p1_folded": (12.0, 15.63),
                           "topk_p1": (12.0, 3.81), "topk_general": (19.83, 0.0),      # profiles/worker_pass_sign_cfg2shapes_4workers.md,
                           "topk_p1_folded": (12.0, 12.18), "mu0": None}                                                # profiles/topk_passes_cfg3shapes_4workers.md
 
