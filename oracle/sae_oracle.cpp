@@ -15,10 +15,11 @@
 //   * double -- the same steps in fp64 with a plain sequential L1 sum; used to check the paper's
 //               identities (Eq. 3 / Appendix A) to ~1e-12.
 //
-// Readings of the paper that nothing in it can confirm ("parity unpinned" for these three
+// Readings of the paper that nothing in it can confirm ("parity unpinned" for the sign(0) and Top-K
 // conventions, they are fixed here and in the CUDA path alike):
 //   * sign(0): the 1-bit code has no zero, so v >= 0 maps to +scale (hence +-0 -> +scale);
-//   * weight decay: coupled L2, lambda * (point where the gradient is evaluated) added to the gradient;
+//   * weight decay: coupled L2, lambda * (point where the gradient is evaluated) added to the gradient
+//     (a reading; the arithmetic itself is pinned to a library SGD optimiser with weight decay);
 //   * Top-K: k = max(1, floor(n*num/den)); every entry whose magnitude ties the k-th largest is kept,
 //     exact zeros are never selected.
 //   * local steps (Section 2 names the extension -- "the local model difference will be communicated every

@@ -200,6 +200,29 @@ def test_identity_compressor_is_momentum_sgd(K, mode):
     assert np.all(o.get_all(o.E) == 0) and np.all(o.get(o.E_SRV) == 0)
 
 
+@pytest.mark.parametrize("K", [1, 3])
+@pytest.mark.parametrize("mode", [EF, SAEF])
+@pytest.mark.parametrize("mu,lam", [(0.9, 1e-3), (0.0, 0.0), (0.5, 5e-2)])
+def test_identity_compressor_matches_library_sgd(K, mode, mu, lam):
+    """The same reduction against a library optimiser instead of a restatement: with the identity
+    compressor the trajectory is torch.optim.SGD (heavy ball, no dampening, no Nesterov, weight decay
+    added to the gradient) on the worker-averaged gradient, with a learning rate that changes per step."""
+    import torch
+    sizes = [7, 1, 40]
+    x0, gs = rand_sizes_grads(K, sizes, 9, np.float64, seed=3)
+    lrs = [0.1, 0.1, 0.05, 0.05, 0.2, 0.1, 0.01, 0.01, 0.1]
+    o = Oracle(K, sizes, x0, compressor=IDENTITY, mode=mode, momentum=mu, weight_decay=lam, dtype=np.float64)
+    p = torch.nn.Parameter(torch.tensor(x0, dtype=torch.float64))
+    opt = torch.optim.SGD([p], lr=0.1, momentum=mu, weight_decay=lam)
+    for g, lr in zip(gs, lrs):
+        o.step(g, lr)
+        for grp in opt.param_groups:
+            grp["lr"] = lr
+        p.grad = torch.tensor(g.astype(np.float64).mean(axis=0))
+        opt.step()
+    np.testing.assert_allclose(o.get(o.X), p.detach().numpy(), rtol=1e-11, atol=1e-13)
+
+
 def test_identity_closed_form_constant_gradient():
     """K = 1, constant gradient: x_T = x_0 - eta g sum_{t=1..T} (1 - mu^t)/(1 - mu)."""
     sizes = [4, 3]
