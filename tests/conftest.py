@@ -10,6 +10,11 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200 with -m gpu)")
+    # A fresh checkout has no built libraries (they are not in the history): build what is missing, once,
+    # so that the suite does not depend on a build step having run before it.  nvcc cross-compiles without a GPU.
+    from paper_2008_05823_b200 import build as cuda_build
+    if not all(os.path.exists(os.path.join(cuda_build.HERE, name)) for name in cuda_build.TARGETS):
+        cuda_build.build()
 
 
 def pytest_collection_modifyitems(config, items):
