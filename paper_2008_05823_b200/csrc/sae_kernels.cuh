@@ -111,6 +111,9 @@ constexpr int SRV_B = 8;    // workers per batch of word loads
 #ifndef SAE_K3_STAGE
 #define SAE_K3_STAGE 1
 #endif
+#ifndef SAE_K3_SUM_DIRECT
+#define SAE_K3_SUM_DIRECT 1
+#endif
 static_assert(THREADS * SRV_E == TILE, "one pass of the block covers one tile");
 
 __device__ __forceinline__ u64 pack2(u32 lo, u32 hi) {
@@ -146,7 +149,11 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
   __shared__ float s_k[MAX_WORKERS];
   __shared__ float sh_s_old;
   __shared__ const u32* s_row[TABLE ? MAX_WORKERS : 1];
-  constexpr bool STAGE = SAE_K3_STAGE && !FIN;
+  // (SUM: there is no worker loop for the staged copy to pass under -- staging would only put a wait between a
+  // tile's loads and its arithmetic -- so a thread fetches its 16 parameters of the sum, the server error and
+  // the parameters with twelve independent 16-byte loads up front.)
+  constexpr bool DIRECT = SUM && SAE_K3_SUM_DIRECT;
+  constexpr bool STAGE = SAE_K3_STAGE && !FIN && !DIRECT;
   __shared__ alignas(128) float s_e[STAGE ? TILE : 4];
   __shared__ alignas(128) float s_x[(STAGE && LAZY) ? TILE : 4];
   __shared__ alignas(8) u64 s_bar;
@@ -228,10 +235,15 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) sv[q] = ld4_stream(A.ssum + pbase + i + 4 * q);
       }
-      float4 ev[(DC || STAGE) ? 1 : SRV_E / 4];
-      if constexpr (!DC && !STAGE) {
+      float4 ev[((DC || STAGE) && !DIRECT) ? 1 : SRV_E / 4];
+      float4 xd[(DIRECT && LAZY) ? SRV_E / 4 : 1];
+      if constexpr (DIRECT || (!DC && !STAGE)) {
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) ev[q] = ld4(ep + i + 4 * q);
+      }
+      if constexpr (DIRECT && LAZY) {
+#pragma unroll
+        for (int q = 0; q < SRV_E / 4; ++q) xd[q] = ld4(xp + i + 4 * q);
       }
       // The words of SRV_B workers are fetched as one batch of independent loads, the next batch while
       // this one is consumed: without that the loop waits out one memory latency per worker.
@@ -283,11 +295,14 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         }
         float4 e;
         if constexpr (STAGE) e = ld4(s_e + i + 4 * q);
+        else if constexpr (DIRECT) e = ev[q];
         else if constexpr (DC) e = ld4(ep + i + 4 * q);
         else e = ev[q];
         if constexpr (LAZY) {
           // e holds the previous step's Delta: C(Delta) is its scaled sign (double-way) or Delta itself
-          float4 xv = STAGE ? ld4(s_x + i + 4 * q) : ld4(xp + i + 4 * q);
+          float4 xv;
+          if constexpr (DIRECT) xv = xd[q];
+          else xv = STAGE ? ld4(s_x + i + 4 * q) : ld4(xp + i + 4 * q);
           float4 cs;
           cs.x = DC ? sign_code(e.x, s_old) : e.x; cs.y = DC ? sign_code(e.y, s_old) : e.y;
           cs.z = DC ? sign_code(e.z, s_old) : e.z; cs.w = DC ? sign_code(e.w, s_old) : e.w;
