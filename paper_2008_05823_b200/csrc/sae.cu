@@ -14,6 +14,11 @@
 #include <new>
 #include <vector>
 
+// scaled sign, p = 1: from this many workers on, the server pass of a step is folded into the next worker pass
+#ifndef SAE_SIGN_FOLD_MIN_K
+#define SAE_SIGN_FOLD_MIN_K 32
+#endif
+
 using namespace sae;
 
 namespace {
@@ -526,7 +531,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // in k order on the way; a streaming server pass then only reads that sum.
     // (Worth it from 32 workers on: the unpacking server pass costs K additions per parameter, the streaming
     // one and the extra vector the worker pass writes do not depend on K -- config 4: 7.82 -> 7.62 ms per step,
-    // config 2 with 16 workers: 0.928 -> 0.938.)
+    // config 2 with 16 workers: 0.931 ms either way.)
     const bool fold_sign = defer_avg && lazy_ok && !h->inline_fin && h->local_steps <= 1 && h->ssum != nullptr;
     if (h->tail_pending && !(pending_in && fold_sign)) return SAE_ERR_INVALID_ARG;
     if (pending_in) {
@@ -904,7 +909,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   h->fused_gen_ok = (!shard && topk && cfg->avg_period != 1 && (K == 8 || K == 16) && dpad < (1ll << 31) &&
                      d < (1ll << 31)) ? 1 : 0;
   // (scaled sign: the folded server pass is for large problems, p = 1, K a power of two up to 32)
-  const bool sign_fold = h->fused_ok && K >= 32 && (long long)K * dpad > (1ll << 24);
+  const bool sign_fold = h->fused_ok && K >= SAE_SIGN_FOLD_MIN_K && (long long)K * dpad > (1ll << 24);
   if (h->fused_topk_ok || h->fused_gen_ok || sign_fold) ALLOC0(h->ssum, dpad);
   ALLOC0(h->words, sign ? (size_t)K * nwords : 0);
   ALLOC0(h->words_srv, sign ? nwords : 0);
