@@ -14,6 +14,10 @@
 #include <new>
 #include <vector>
 
+// folded Top-K forms: the workers' threshold select on a second stream beside the server pass and its select
+#ifndef SAE_TOPK_PARALLEL_SELECT
+#define SAE_TOPK_PARALLEL_SELECT 1
+#endif
 // scaled sign, p = 1: from this many workers on, the server pass of a step is folded into the next worker pass
 #ifndef SAE_SIGN_FOLD_MIN_K
 #define SAE_SIGN_FOLD_MIN_K 32
@@ -75,6 +79,14 @@ struct sae_handle {
   int2* work;            // work list of the radix select: data items and candidate chunks
   u32* work_count;
   u32* cand_n;           // [K][T] candidates captured for this step's select
+  // A second set of select scratch for the server's one row, a second stream and two events: in the folded
+  // Top-K forms the workers' threshold select (needs only the worker pass) runs beside the parameter-sized
+  // server pass and the server's own select (fork after the worker pass, join at the end of the step).
+  u32 *hist_srv, *work_count_srv, *cand_n_srv;
+  SelectState* sel_srv;
+  int2* work_srv;
+  cudaStream_t aux;
+  cudaEvent_t ev_fork, ev_join;
   long long cand_stride;
   u32* status;
   u32* status_host;      // pinned
@@ -213,6 +225,11 @@ void free_all(sae_handle* h) {
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
                   h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n, h->ssum};
   for (void* p : ptrs) if (p) cudaFree(p);
+  void* srv_sel[] = {h->hist_srv, h->work_count_srv, h->cand_n_srv, h->sel_srv, h->work_srv};
+  for (void* p : srv_sel) if (p) cudaFree(p);
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->aux) cudaStreamDestroy(h->aux);
   void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows,
                   (void*)h->d_entry_rows, (void*)h->d_count_rows, (void*)h->d_tau_rows[0], (void*)h->d_tau_rows[1],
                   (void*)h->msg_entries, (void*)h->msg_count, (void*)h->agg_acc};
@@ -230,16 +247,22 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
                      u32* tau_out, u32* fb, u32* fb_total) {
   const Plan& P = h->P;
   const int pairs = rows * P.T;
+  // the server's select has scratch of its own where a step may run it beside the workers' select
+  const bool own = (fb == h->fb_srv) && h->hist_srv != nullptr;
+  u32* hist = own ? h->hist_srv : h->hist;
+  SelectState* sel = own ? h->sel_srv : h->sel;
+  int2* work = own ? h->work_srv : h->work;
+  u32* work_count = own ? h->work_count_srv : h->work_count;
+  u32* cand_n = own ? h->cand_n_srv : h->cand_n;
   LAUNCH(h, S_TOPK_SELECT, k_topk_decide, (pairs + THREADS - 1) / THREADS, cand, rows, h->d_n, h->cfg.topk_num,
-         h->cfg.topk_den, tau_guess, h->cand_n, fb, fb_total, h->work, h->work_count);
+         h->cfg.topk_den, tau_guess, cand_n, fb, fb_total, work, work_count);
   const long long items = (long long)P.ntiles * rows;
-  LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, h->work, h->work_count);
+  LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, work, work_count);
   const long long hist_grid = 8LL * h->persistent_blocks;
   for (int level = 0; level < 3; ++level) {
-    LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, src, h->cand_n, h->sel, h->hist, h->work,
-           h->work_count);
-    LAUNCH(h, S_TOPK_SELECT, k_topk_select, pairs, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, h->hist, h->sel,
-           tau_out, h->work_count);
+    LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, src, cand_n, sel, hist, work, work_count);
+    LAUNCH(h, S_TOPK_SELECT, k_topk_select, pairs, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, hist, sel,
+           tau_out, work_count);
   }
 }
 
@@ -626,12 +649,27 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
       fa.tau_prev = h->tau[h->last]; fa.ssum = h->ssum; fa.cand = wa.cand; fa.status = h->status;
       fa.eta_prev = h->eta_prev;
       launch_fused(h, sp, fa, nod ? 1 : 2);
-      topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+      // The workers' select needs only the worker pass; the server pass and the server's select need only the
+      // sum it wrote.  Two chains of small dependent launches: run them side by side (not while kernels are
+      // being timed one by one).
+      const bool side = h->aux != nullptr && !h->profiling;
+      if (side) {
+        cudaStream_t main_stream = h->stream;
+        SAE_CUDA(h, cudaEventRecord(h->ev_fork, main_stream));
+        SAE_CUDA(h, cudaStreamWaitEvent(h->aux, h->ev_fork, 0));
+        h->stream = h->aux;
+        topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+        h->stream = main_stream;
+        SAE_CUDA(h, cudaEventRecord(h->ev_join, h->aux));
+      } else {
+        topk_thresholds(h, src, P.K, wa.cand, h->tau[h->last], h->tau[cur], h->fb, h->fb_total);
+      }
       sa.ssum = h->ssum;
       if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 0, true>), P.ntiles, P, sa);
       else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<2, false, false, 1, true>), P.ntiles, P, sa);
       else LAUNCH_DENSE(h, (k_server_dense<2, false, false, 2, true>), P.ntiles, P, sa);
       if (dc) topk_thresholds(h, stored_rows(h->e_srv), 1, sa.cand_srv, h->tau_srv, h->tau_srv, h->fb_srv, h->fb_total + 1);
+      if (side) SAE_CUDA(h, cudaStreamWaitEvent(h->stream, h->ev_join, 0));
       h->srv_pending = 1;                    // the previous step's server lines now wait for the next server pass
       h->tail_pending = 0;
       lsrv = dc ? 2 : 1;
@@ -945,6 +983,15 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->d_cand_off, T); ALLOC0(h->d_cand_cap, T);
   ALLOC0(h->work, topk ? (size_t)ntiles * K + (size_t)K * (h->cand_stride / CAND_CHUNK + T) : 0);
   ALLOC0(h->work_count, 1); ALLOC0(h->cand_n, topk ? KT : 0);
+#if SAE_TOPK_PARALLEL_SELECT
+  if (h->fused_topk_ok || h->fused_gen_ok) {
+    ALLOC0(h->hist_srv, (size_t)T * HIST_BINS); ALLOC0(h->sel_srv, T); ALLOC0(h->cand_n_srv, T); ALLOC0(h->work_count_srv, 1);
+    ALLOC0(h->work_srv, (size_t)ntiles + (size_t)(h->cand_stride / CAND_CHUNK + T));
+    TRY(cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking));
+    TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+    TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+  }
+#endif
   ALLOC0(h->status, 1);
   TRY(cudaMallocHost((void**)&h->status_host, sizeof(u32)));
   TRY(cudaMemcpyAsync(h->d_tile_tensor, tile_tensor.data(), sizeof(int) * ntiles, cudaMemcpyHostToDevice, h->stream));

@@ -405,7 +405,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   const bool emit = (COMP == 2) && A.emit_srv;
   const u32 lo = emit ? window_lo(A.tau_srv_prev[ti.j]) : NO_GUESS;
   WarpStage stg; stg.buf = cstage + ((COMP == 2) ? (tid >> 5) * CAND_STAGE : 0); stg.n = 0;
-  if (COMP == 2) {
+  if (COMP == 2 && !SUM) {                               // (SUM: no rows are read, so no worker thresholds either)
     for (int k = tid; k < P.K; k += THREADS) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
     __syncthreads();
   }
