@@ -96,6 +96,10 @@ int sae_init(const sae_config *cfg, const float *x0, sae_handle **out);
  * (state, grads pointer, lr) into a CUDA graph and later steps with the same key replay it with one
  * graph launch (the host cost of a step drops from one launch per kernel to one launch); if the
  * caller is itself capturing the stream, the kernels simply join that capture.
+ * Top-K with the folded tail (8 or 16 workers, no weight decay): part of a step -- the workers' threshold
+ * select -- runs on a second stream the handle owns (created by sae_init), forked from the handle's stream
+ * after the worker pass and joined to it again before the call returns, so all of a step's work stays
+ * ordered on the handle's stream as the caller sees it (inside a capture: two branches of the same graph).
  */
 int sae_step(sae_handle *h, const float *grads, float lr);
 
