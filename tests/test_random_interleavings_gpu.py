@@ -106,3 +106,30 @@ def test_random_calls_between_steps(case):
         compare_server_messages(gpu, orc, c["comp"], c["dc"], tag=f"case {case} end")
         assert not orc.range_flag
         gpu.close()
+
+
+def test_two_handles_alternate_on_one_stream():
+    """Two independent problems in the folded Top-K form stepped in turn on the same side stream: each handle
+    forks part of its step onto a stream of its own and joins it again, so neither may disturb the other."""
+    import torch
+    cases = [draw(NUM_DRAWN + 0), draw(NUM_DRAWN + 1)]            # K = 8 and K = 16, Top-K, p = 1
+    with torch.cuda.stream(torch.cuda.Stream()):
+        runs = []
+        for c in cases:
+            K, sizes = c["K"], c["sizes"]
+            d = int(np.sum(sizes))
+            scales = synth.tensor_scales(c["seed"], len(sizes), -4.0, -1.0)
+            x0 = synth.x0_numpy(c["seed"], d)
+            kw = dict(compressor=c["comp"], server_compress=1, avg_period=c["p"], momentum=0.9, topk_num=1, topk_den=100)
+            pool = [synth.grads_numpy(c["seed"], t, K, sizes, scales, 1000, 100.0) for t in range(2)]
+            runs.append(dict(orc=so.Oracle(K, sizes, x0, threads=8, **kw),
+                             gpu=sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw),
+                             pool=pool, dev=[torch.from_numpy(g).cuda() for g in pool]))
+        for t in range(6):
+            for r in runs:
+                r["orc"].step(r["pool"][t % 2], 0.1)
+                r["gpu"].step(r["dev"][t % 2], 0.1)
+        for i, r in enumerate(runs):
+            compare_state(r["gpu"], r["orc"], so.TOPK, tag=f"handle {i}")
+            compare_server_messages(r["gpu"], r["orc"], so.TOPK, 1, tag=f"handle {i}")
+            r["gpu"].close()
