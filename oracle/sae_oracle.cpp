@@ -22,8 +22,8 @@
 //     (a reading; the arithmetic itself is pinned to a library SGD optimiser with weight decay);
 //   * Top-K: k = max(1, floor(n*num/den)); every entry whose magnitude ties the k-th largest is kept,
 //     exact zeros are never selected.
-//   * local steps (Section 2 names the extension -- "the local model difference will be communicated every
-//     several iterations" -- without spelling it out): with period H, iteration t communicates iff
+//   * local steps (Section 2 names the extension to local SGD, where a worker sends its model difference only
+//     once in several iterations, without spelling it out): with period H, iteration t communicates iff
 //     (t+1) mod H = 0; on the other iterations a worker only does its own lines, and its model difference
 //     keeps accumulating in the place of its error: e^(k) <- Delta^(k) = e^(k) + eta m^(k), nothing is sent,
 //     x and the server error stay.  The gradient point x - e^(k) of the step-ahead branch is then the

@@ -8,6 +8,7 @@ import numpy as np
 import pytest
 
 from oracle import sae_oracle as so
+import scale_cases
 from oracle.sae_oracle import Oracle, IDENTITY, SIGN, TOPK, EF, SAEF
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
@@ -108,15 +109,52 @@ def test_sign_scale_within_rounding_of_exact_mean():
 
 
 def test_scale_from_fixed_truncates_to_53_bits():
-    # S = 2^100 + 2^47 + 1: bits below 2^48 are cleared before the division
-    S = (1 << 100) + (1 << 47) + 1
-    assert so.scale_from_fixed(S, 1) == np.float32(2.0 ** 36)
-    # a sum whose 54th bit would round up in a nearest conversion must not
-    S = (1 << 53) + 1
-    n = 3
-    exp = np.float32((float(1 << 53) / 3.0) * 2.0 ** -64)
-    assert so.scale_from_fixed(S, n) == exp
+    """Eq. 2's ||v||_1 / n from the exact sum: the bits below the top 53 are dropped, not rounded in.
+    S = 2^100 + 2^77 + 2^76 - 1, n = 1: float's last bit (2^77) is set, the next is clear and everything
+    below is set.  Truncation leaves the quotient below the midpoint of two floats (-> 2^36 + 2^13);
+    rounding the sum to 53 bits first would land on the midpoint and tie to even (-> 2^36 + 2^14)."""
+    S = (1 << 100) + (1 << 77) + (1 << 76) - 1
+    assert so.scale_from_fixed(S, 1) == np.float32(2.0 ** 36 + 2.0 ** 13)
+    assert scale_cases.scale_truncating(S, 1) == np.float32(2.0 ** 36 + 2.0 ** 13)
+    assert scale_cases.scale_rounding(S, 1) == np.float32(2.0 ** 36 + 2.0 ** 14)
+    # bits below 2^48 of a 101-bit sum never matter
+    assert so.scale_from_fixed((1 << 100) + (1 << 47) + 1, 1) == np.float32(2.0 ** 36)
     assert so.scale_from_fixed(0, 5) == 0.0
+
+
+def test_scale_from_fixed_against_exact_rationals():
+    """Random 60..120-bit sums and divisors against exact integer / fraction arithmetic written here."""
+    rng = np.random.default_rng(77)
+    for _ in range(4000):
+        bits = int(rng.integers(1, 121))
+        S = int(rng.integers(0, 1 << 62)) | (int(rng.integers(0, 1 << 62)) << 60)
+        S = (S & ((1 << bits) - 1)) | (1 << (bits - 1))
+        n = int(rng.integers(1, 1 << int(rng.integers(1, 31))))
+        assert so.scale_from_fixed(S, n) == scale_cases.scale_truncating(S, n), (S, n)
+
+
+@pytest.mark.parametrize("n", [1, 3, 8, 1000, 4097, 1 << 20])
+@pytest.mark.parametrize("top_bit", [60, 75, 95])
+def test_scale_from_fixed_where_truncating_and_rounding_differ(n, top_bit):
+    """Sums built so that the two readings give different floats: the oracle follows the truncating one."""
+    rng = np.random.default_rng(n + top_bit)
+    for _ in range(5):
+        S = scale_cases.discriminating_sum(n, top_bit, rng)
+        t, r = scale_cases.scale_truncating(S, n), scale_cases.scale_rounding(S, n)
+        assert t != r
+        assert so.scale_from_fixed(S, n) == t
+
+
+@pytest.mark.parametrize("n,top_bit", [(8, 60), (8, 90), (4096, 62), (5000, 70), (3 * 4096 + 7, 93)])
+def test_sign_compress_on_tensors_where_truncating_and_rounding_differ(n, top_bit):
+    """The same through the whole compressor: tensors whose exact L1 sum discriminates (values both below
+    and above 1, mixed signs, zeros in between)."""
+    v = scale_cases.discriminating_tensor(n, top_bit, seed=n)
+    S = scale_cases.fixed_sum(v)
+    assert so.l1_fixed(v) == (S, False)
+    _, s, _, rg = so.compress(SIGN, v)
+    assert not rg
+    assert s == scale_cases.scale_truncating(S, n) != scale_cases.scale_rounding(S, n)
 
 
 @pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1000, 4097])
