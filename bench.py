@@ -3,12 +3,16 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--avg-period p] [--impl reference]
 
 Prints ONE JSON line.  `value` = steps/s over all N GPUs with the gradients already resident in HBM
-(a ring of pre-generated gradient sets, each far larger than L2, cycled step by step); `e2e` = the
+(a ring of pre-generated gradient sets, each far larger than L2, cycled step by step) for a caller that
+does not read the state between steps; `with_step_ahead` = the same loop when the caller fetches the
+step-ahead point x - e^(k) (where Algorithm 1 evaluates the next gradient) after every step; `e2e` = the
 same step driven through the host-buffer entry points (pinned host gradients copied in, parameters
 copied out, inside the timed region); `roofline` = the dominant kernel (the worker pass) against the
-measured HBM copy bandwidth; `cpu_baseline` = the CPU oracle timed on a bounded sample of the same
-workload.  The path does not shard (the workers are a batch axis on one GPU), so N > 1 runs N
-independent replicas: no data-path collective, "scaling": "weak".
+measured HBM copy bandwidth; `all_configs` = every benchmark configuration under both averaging
+schedules (p = 1, and the paper's finite period), a short timed region each; `cpu_baseline` = the CPU
+oracle timed on whole steps of the same workload at full size where the host can hold it.  The path does
+not shard (the workers are a batch axis on one GPU), so N > 1 runs N independent replicas: no data-path
+collective, "scaling": "weak".
 
 `--impl reference` times the CPU oracle alone (there is no reference implementation of this paper).
 """
@@ -26,20 +30,24 @@ if ROOT not in sys.path:
 
 METRIC = "step-ahead EF steps/sec at W workers x d params"
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126 << 20
 
-# DRAM traffic of one worker-pass launch per worker-element, from the committed ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case of the same kernel, which grows in
-# proportion to the elements processed).  None until a capture exists for the variant.
-# sign_p1: 13.64 B at K = 4 = 12 B per worker-element + (8 B of ebar + sign words) per parameter.
-# topk_p1: 1324.2 MB for 4 x 25.56 M worker-elements = 12 B per worker-element + 3.81 B per parameter (ebar);
-# topk_general: 2027.4 MB = 19.83 B per worker-element (candidate lists included);
-# topk_p1_folded: 2765.3 MB for 8 x 25.56 M worker-elements = 12 B per worker-element + 12.18 B per parameter.
-# sign_p1_folded: 43.752 GB for 32 x 109.48 M worker-elements, captured on config 4 itself with one-pass metrics
-# (profiles/worker_and_server_pass_cfg4_dram_bytes.md) = 12 B per worker-element + 15.63 B per parameter.
-WORKER_PASS_DRAM_BYTES = {"sign_p1": (12.0, 6.56), "sign_general": (19.64, 0.0),      # (per worker-element, per parameter)
-                          "sign_p1_folded": (12.0, 15.63),
-                          "topk_p1": (12.0, 3.81), "topk_general": (19.83, 0.0),      # profiles/worker_pass_sign_cfg2shapes_4workers.md,
-                          "topk_p1_folded": (12.0, 12.18), "mu0": None}                                                # profiles/topk_passes_cfg3shapes_4workers.md
+# DRAM traffic of one worker-pass launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum), as
+# (bytes per worker-element, bytes per parameter, where the figure comes from).  The two-term form holds
+# because the traffic of these streaming passes grows in proportion to the elements processed; captures
+# on a smaller worker count of the same kernel are scaled by it.  The run itself cannot measure DRAM
+# counters: the source string says which capture a figure rests on, so a stale one is visible.
+WORKER_PASS_DRAM_BYTES = {
+    "sign_p1": (12.0, 6.56, "ncu capture of the folded-averaging worker pass, config-2 shapes at 4 workers"),
+    "sign_general": (19.64, 0.0, "ncu capture of the plain worker pass, config-2 shapes at 4 workers"),
+    "sign_p1_folded": (12.0, 15.63, "ncu capture of k_worker_fused<32> on config 4 itself (one-pass metrics), "
+                                    "43.752 GB per launch"),
+    "topk_p1": (12.0, 3.81, "ncu capture of the Top-K worker pass, config-3 shapes at 4 workers"),
+    "topk_general": (19.83, 0.0, "ncu capture of the Top-K worker pass with stored differences, config-3 shapes at 4 workers"),
+    "topk_p1_folded": (12.0, 12.18, "ncu capture of k_worker_fused<8, Top-K> on config 3"),
+    "mu0": None,
+}
 
 
 def measured_peak():
@@ -111,63 +119,196 @@ def sample_tensors(sizes, budget):
     return sorted(out)
 
 
-def cpu_baseline(w, avg_period, seed, steps, warmup, target_elems=40_000_000):
-    """The oracle, as it stands, on a sample of whole tensors of the workload (all K workers)."""
-    import numpy as np
+def _oracle_threads():
     from oracle import sae_oracle as so
+    return max(1, min(so.max_threads(), len(os.sched_getaffinity(0))))
+
+
+def _oracle_for(w, avg_period, sizes, x0, threads):
+    from oracle import sae_oracle as so
+    return so.Oracle(w.num_workers, sizes, x0, compressor=w.compressor, server_compress=w.server_compress,
+                     mode=w.mode, avg_period=avg_period, momentum=w.momentum, weight_decay=w.weight_decay,
+                     topk_num=w.topk_num, topk_den=w.topk_den, threads=threads)
+
+
+def _sampled_inputs(w, seed, js):
+    """x0 and two gradient sets restricted to the whole tensors `js` (host generator)."""
+    import numpy as np
     from paper_2008_05823_b200 import synth
-    K, sizes = w.num_workers, w.tensor_sizes
+    sizes = w.tensor_sizes
     offs = np.concatenate([[0], np.cumsum(sizes)])
-    js = sample_tensors(sizes, max(1, target_elems // K))
-    sub = [sizes[j] for j in js]
-    n_sub = int(sum(sub))
     scales = synth.workload_scales(w, seed)
-    threads = max(1, min(so.max_threads(), len(os.sched_getaffinity(0))))
     x0 = np.concatenate([synth.x0_numpy_range(seed, int(offs[j]), sizes[j]) for j in js])
-    orc = so.Oracle(K, sub, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
-                    avg_period=avg_period, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
-                    topk_den=w.topk_den, threads=threads)
     grads = [np.stack([np.concatenate([synth.grads_numpy_range(seed, t, k, int(offs[j]), sizes[j], scales[j],
                                                                w.outlier_per_65536, w.outlier_mult) for j in js])
-                       for k in range(K)]) for t in range(2)]
-    for t in range(warmup):
-        t0 = time.perf_counter()
-        orc.step(grads[t % 2], w.lr)
-        warm_dt = time.perf_counter() - t0
-    if steps <= 0:                      # aim at ~15 s of CPU work
-        steps = int(max(2, min(1000, 15.0 / max(warm_dt, 1e-3))))
+                       for k in range(w.num_workers)]) for t in range(2)]
+    return x0, grads
+
+
+def _full_inputs(w, seed, sets):
+    """x0 and `sets` whole gradient sets on the host.  With a CUDA device the seeded device generator makes
+    them (the same bits as the host generator, far faster) and they are copied over; otherwise numpy does."""
+    import numpy as np
+    from paper_2008_05823_b200 import synth
+    scales = synth.workload_scales(w, seed)
+    try:
+        import torch
+        cuda = torch.cuda.is_available()
+    except Exception:
+        cuda = False
+    if cuda:
+        dev = torch.device("cuda", torch.cuda.current_device())
+        gen = synth.DeviceGenerator(w.tensor_sizes, scales, device=dev)
+        x0d = torch.empty(w.d, device=dev)
+        gen.x0(x0d, seed)
+        x0 = x0d.cpu().numpy()
+        grads = []
+        for t in range(sets):
+            g = torch.empty(w.num_workers, w.d, device=dev)
+            gen.grads(g, w.num_workers, seed, t, w.outlier_per_65536, w.outlier_mult)
+            grads.append(g.cpu().numpy())
+            del g
+        torch.cuda.synchronize()
+        torch.cuda.empty_cache()
+        return x0, grads, "device generator, copied to the host"
+    x0 = synth.x0_numpy(seed, w.d)
+    grads = [synth.workload_grads_numpy(w, seed, t, scales) for t in range(sets)]
+    return x0, grads, "host generator"
+
+
+def _time_steps(orc, grads, lr, steps):
     t0 = time.perf_counter()
     for t in range(steps):
-        orc.step(grads[t % 2], w.lr)
-    dt = time.perf_counter() - t0
-    frac = n_sub / w.d
-    # the same oracle on one core (a few steps): the plain single-threaded figure
-    orc1 = so.Oracle(K, sub, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
-                     avg_period=avg_period, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
-                     topk_den=w.topk_den, threads=1)
-    orc1.step(grads[0], w.lr)
-    n1 = int(max(1, min(steps, 3.0 / max(warm_dt * threads / 4, 1e-3))))
-    t0 = time.perf_counter()
-    for t in range(n1):
-        orc1.step(grads[(t + 1) % 2], w.lr)
-    dt1 = time.perf_counter() - t0
-    single = {"value": n1 / dt1 * frac, "unit": "steps/s", "cores": 1, "steps": n1, "seconds": dt1}
-    return {"value": steps / dt * frac, "unit": "steps/s", "cores": threads, "kind": "oracle", "single_thread": single,
-            "sample": f"{len(js)} of {len(sizes)} whole tensors ({n_sub} of {w.d} params = {100 * frac:.2f}%), all "
-                      f"{K} workers, {steps} steps in {dt:.2f} s; value = sample steps/s x sampled fraction",
-            "sample_seconds": dt, "ms_per_sample_step": 1e3 * dt / steps}
+        orc.step(grads[t % len(grads)], lr)
+    return time.perf_counter() - t0
 
 
-def run_reference(args, w, avg_period, rank):
+def cpu_baseline(w, avg_period, seed, steps, warmup, wall_budget_s=200.0, sample_elems=40_000_000):
+    """The oracle, as it stands, on the host cores: whole steps of the workload at FULL size when the host can
+    hold it and (warmup + steps) of them fit the wall budget, otherwise on a bounded sample of whole tensors
+    (all K workers) scaled by the sampled fraction and marked as an extrapolation.  steps <= 0: as many
+    full-size steps as fit ~15 s, at least 2.  Used unchanged by the native arm's `cpu_baseline` and by
+    `--impl reference`, so the two cannot disagree about what was timed."""
+    import numpy as np
+    import psutil
+    K, sizes, d = w.num_workers, w.tensor_sizes, w.d
+    threads = _oracle_threads()
+    warmup = max(1, warmup)
+    # ---- a small sample first: the single-thread figure, the sampled estimate, and a guess of the full-size step time
+    js = sample_tensors(sizes, max(1, sample_elems // K))
+    sub = [sizes[j] for j in js]
+    n_sub = int(sum(sub))
+    frac = n_sub / d
+    x0s, gs = _sampled_inputs(w, seed, js)
+    orc = _oracle_for(w, avg_period, sub, x0s, threads)
+    orc.step(gs[0], w.lr)
+    dt_probe = _time_steps(orc, gs[1:] + gs[:1], w.lr, 2) / 2
+    n_s = int(max(2, min(200, 4.0 / max(dt_probe, 1e-4))))
+    dt_s = _time_steps(orc, gs, w.lr, n_s)
+    sampled = {"value": n_s / dt_s * frac, "unit": "steps/s", "cores": threads, "steps": n_s, "seconds": dt_s,
+               "sample": f"{len(js)} of {len(sizes)} whole tensors ({n_sub} of {d} params = {100 * frac:.2f}%), all {K} "
+                         f"workers; value = sample steps/s x sampled fraction (an extrapolation: small tensors sit in cache)"}
+    del orc
+    orc1 = _oracle_for(w, avg_period, sub, x0s, 1)
+    orc1.step(gs[0], w.lr)
+    n1 = int(max(1, min(n_s, 3.0 / max(dt_s / n_s * threads / 2, 1e-4))))
+    dt1 = _time_steps(orc1, gs[1:] + gs[:1], w.lr, n1)
+    single = {"value": n1 / dt1 * frac, "unit": "steps/s", "cores": 1, "steps": n1, "seconds": dt1,
+              "sample": "the same sample of whole tensors on one thread, scaled by the sampled fraction"}
+    del orc1
+    est_full_step = 2.0 * (dt_s / n_s) / frac          # (x2: the sample under-estimates, its small tensors sit in cache)
+    # ---- full size, if memory and time allow
+    sets = 1 if 4 * K * d > (4 << 30) else 2
+    need = 4 * (4 * K * d + sets * K * d + 8 * d)       # oracle state m, e, Delta, C(Delta) + gradient sets
+    avail = psutil.virtual_memory().available
+    want_steps = steps if steps > 0 else 2
+    reason = None
+    if need * 1.1 + (6 << 30) > avail:
+        reason = (f"host memory: the full-size oracle needs {need / 1e9:.1f} GB, {avail / 1e9:.1f} GB available "
+                  f"(short by {(need * 1.1 + (6 << 30) - avail) / 1e9:.1f} GB)")
+    elif est_full_step * (warmup + want_steps) + need / 2.5e9 > wall_budget_s:
+        reason = (f"time: a full-size step is estimated at {est_full_step:.1f} s, {warmup + want_steps} of them plus "
+                  f"set-up exceed the {wall_budget_s:.0f} s budget")
+    if reason is None:
+        x0, grads, how = _full_inputs(w, seed, sets)
+        orc = _oracle_for(w, avg_period, sizes, x0, threads)
+        warm_dt = _time_steps(orc, grads, w.lr, warmup) / warmup
+        if steps <= 0:
+            steps = int(max(2, min(1000, 15.0 / max(warm_dt, 1e-3))))
+        dt = _time_steps(orc, grads[::-1], w.lr, steps)
+        del orc, grads
+        return {"value": steps / dt, "unit": "steps/s", "cores": threads, "kind": "oracle", "full_size": True,
+                "extrapolated": False, "steps": steps, "warmup": warmup, "seconds": dt, "ms_per_step": 1e3 * dt / steps,
+                "sample": f"whole workload ({d} params x {K} workers), {steps} full-size steps in {dt:.2f} s after "
+                          f"{warmup} warm-up; {sets} gradient set(s) from the {how}",
+                "single_thread": single, "sampled_estimate": sampled}
+    # ---- bounded sample: K steps of a sample sized to fit the budget
+    if steps <= 0:
+        steps = n_s
+        dt = dt_s
+    else:
+        orc = _oracle_for(w, avg_period, sub, x0s, threads)
+        _time_steps(orc, gs, w.lr, warmup)
+        dt = _time_steps(orc, gs, w.lr, steps)
+        del orc
+    return {"value": steps / dt * frac, "unit": "steps/s", "cores": threads, "kind": "oracle", "full_size": False,
+            "extrapolated": True, "steps": steps, "warmup": warmup, "seconds": dt, "ms_per_step": 1e3 * dt / steps / frac,
+            "not_full_size_because": reason, "sample": sampled["sample"], "single_thread": single,
+            "sampled_estimate": sampled}
+
+
+def config_dict(w, p, args, world):
+    """The `config` object of the JSON line: the same for the native and the reference arm."""
+    from paper_2008_05823_b200 import configs
+    grad_bytes = 4 * w.num_workers * w.d
+    ring = ring_length(args, grad_bytes, p)
+    return {"workload": w.name, "num_workers": w.num_workers, "d": w.d, "num_tensors": w.num_tensors,
+            "compressor": {0: "identity", 1: "scaled_sign", 2: "topk"}[w.compressor],
+            "avg_period": p, "momentum": w.momentum, "lr": w.lr, "weight_decay": w.weight_decay,
+            "mode": "saef" if w.mode == configs.SAEF else "ef",
+            "server_compress": "double-way" if w.server_compress else "single-way",
+            "topk": f"{w.topk_num}/{w.topk_den}" if w.compressor == configs.TOPK else None,
+            "local_steps": args.local_steps,
+            "caller_reads_state_between_steps": False,
+            "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
+            "l2": l2_note(grad_bytes, ring)}
+
+
+def ring_length(args, grad_bytes, period=1):
+    """Gradient sets kept in HBM and cycled, at most 40 GB of them.  Large sets: four, or two.  Sets smaller than
+    L2: enough of them that the ring as a whole is twice L2 (a set is evicted before its turn comes again),
+    rounded up to a multiple of the step pattern's period -- lcm(4, p): scale buffers alternate, record
+    buffers rotate by four, every p-th step averages -- so that a given set always meets the same kind of step
+    and the library's cache of step graphs (keyed on the gradient pointer) stays small."""
+    import math
+    if args.ring:
+        return args.ring
+    if grad_bytes > L2_BYTES:
+        return 4 if 4 * grad_bytes <= (40 << 30) else 2     # (powers of two divide the step pattern's period)
+    pattern = math.lcm(4, max(1, period))
+    need = -(-2 * L2_BYTES // grad_bytes)
+    return int(-(-need // pattern) * pattern)
+
+
+def l2_note(grad_bytes, ring):
+    if grad_bytes > L2_BYTES:
+        return (f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient set "
+                f"(ring of {ring})")
+    return (f"inputs larger than L2: a ring of {ring} gradient sets of {grad_bytes / 1e6:.1f} MB = "
+            f"{ring * grad_bytes / 1e6:.0f} MB is cycled, so a set is evicted before it is read again; the K x d "
+            f"state of this workload is itself smaller than L2 and stays there")
+
+
+def run_reference(args, w, avg_period, rank, world):
     if rank != 0:
         return
     steps, warmup = max(1, args.steps), max(1, args.warmup)
-    cb = cpu_baseline(w, avg_period, args.seed, steps, warmup, target_elems=30_000_000)
+    cb = cpu_baseline(w, avg_period, args.seed, steps, warmup, wall_budget_s=300.0)
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": "steps/s", "n_gpus": args.gpus,
             "steps": steps, "warmup": warmup, "ms_per_step": 1e3 / cb["value"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "num_workers": w.num_workers, "d": w.d, "avg_period": avg_period,
-                       "note": "no reference implementation exists for this paper: this arm is the CPU oracle"},
+            "config": config_dict(w, avg_period, args, world),
+            "note": "no reference implementation exists for this paper: this arm is the CPU oracle on the host cores",
             "cpu_baseline": cb,
             "e2e": {"value": cb["value"], "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -218,6 +359,20 @@ def algorithmic_bytes(w, avg_period):
     return step, worker, variant
 
 
+def step_ahead_bytes(w, avg_period):
+    """Bytes a step must move when the caller reads the step-ahead point x - e^(k) after it (one vector).
+    p = 1: the averaged error needs every worker's scale (threshold), and a scale needs the worker's whole
+    tensor, so the K momentum rows are read a second time (or the K differences written and read back, which
+    is more): 16 W d; then ebar R+W, the server error R+W twice (the server's own scale separates forming
+    Delta from subtracting C(Delta)), x R+W, the point W.  Other periods: the general step plus x, one
+    worker's stored difference R and the point W."""
+    Wd, d = w.num_workers * w.d, w.d
+    if avg_period == 1:
+        return 16 * Wd + 36 * d, "16 W d + 36 d (g R, m R+W+R | ebar R+W, e_srv (R+W) x 2, x R+W, point W)"
+    step, _, _ = algorithmic_bytes(w, avg_period)
+    return step + 12 * d, "general step + 12 d (x R, one worker's difference R, point W)"
+
+
 def run_sharded(args, w, p, rank, local_rank, world):
     """One job whose K workers are split over the ranks (scaled sign).  Each rank runs the worker lines of
     its own workers; the server pass of every rank reads all K messages in place from their owners."""
@@ -245,7 +400,7 @@ def run_sharded(args, w, p, rank, local_rank, world):
     x0 = torch.empty(d, device=dev)
     gen.x0(x0, args.seed)
     grad_bytes = 4 * count * d
-    ring = args.ring or int(max(2, min(4, (40 << 30) // grad_bytes, args.steps + args.warmup)))
+    ring = args.ring or int(max(2, min(4, (40 << 30) // grad_bytes)))
     grads = []
     for t in range(ring):
         g = torch.empty(count, d, device=dev)
@@ -355,6 +510,9 @@ def main():
                     help="sharded operation: the workers are split over the ranks (strong scaling of one job); "
                          "with one rank it times the same two-phase, table-driven path on one GPU")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-step-ahead", action="store_true", help="skip the arm that reads the step-ahead point every step")
+    ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
+                    help="skip the short runs of every configuration under both schedules (default run only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
@@ -381,18 +539,19 @@ def main():
         w.tensor_sizes = configs.blockwise_sizes(w.tensor_sizes, args.block_size)
         w.name += f"_blk{args.block_size}"
     p = args.avg_period
+    overridden = (args.workers > 0 or args.mode is not None or args.single_way or args.momentum is not None or
+                  args.topk_percent is not None or args.block_size > 0 or args.local_steps != 1 or p != 1)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     if args.impl == "reference":
-        run_reference(args, w, p, rank)
+        run_reference(args, w, p, rank, world)
         return
     if args.sharded:
         run_sharded(args, w, p, rank, local_rank, world)
         return
 
-    import numpy as np
     import torch
     import torch.distributed as dist
     from paper_2008_05823_b200 import binding as sb
@@ -414,72 +573,144 @@ def main():
     # Everything runs on one non-default stream: on such a stream sae_step replays cached CUDA graphs.
     stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(stream)
-
-    K, d = w.num_workers, w.d
-    scales = synth.workload_scales(w, args.seed)
-    gen = synth.DeviceGenerator(w.tensor_sizes, scales, device=dev)
-    x0 = torch.empty(d, device=dev)
-    gen.x0(x0, args.seed)
-    grad_bytes = 4 * K * d
-    ring = args.ring or int(max(2, min(4, (40 << 30) // grad_bytes, args.steps + args.warmup)))
-    grads = []
-    for t in range(ring):
-        g = torch.empty(K, d, device=dev)
-        gen.grads(g, K, args.seed, t, w.outlier_per_65536, w.outlier_mult)
-        grads.append(g)
-
-    def make():
-        return sb.Sae(K, w.tensor_sizes, x0, compressor=w.compressor, server_compress=w.server_compress, mode=w.mode,
-                      avg_period=p, momentum=w.momentum, weight_decay=w.weight_decay, topk_num=w.topk_num,
-                      topk_den=w.topk_den, local_steps=args.local_steps)
-
-    # ---- device-resident throughput ------------------------------------------------------------------
-    sae = make()
-    for t in range(args.warmup):
-        sae.step(grads[t % ring], w.lr)
-    sae.sync()
-    sampler = ClockSampler(local_rank)
-    launches0 = sae.kernel_launches
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    sampler.start()
-    ev0.record()
-    for t in range(args.steps):
-        sae.step(grads[(args.warmup + t) % ring], w.lr)
-    ev1.record()
-    barrier()
-    clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    gpu_launches = sae.kernel_launches - launches0
-    sae.sync()                                    # raises if the device flagged a range error
-    ms_total = max_over_ranks(ms_total, dev)
-    ms_per_step = ms_total / args.steps
-    value = whole_job_value(args.steps, ms_total, world)
-
-    # ---- per-kernel times (same steps again, every launch bracketed by events on the library's stream) ----
-    sae.set_profiling(True)
-    for t in range(args.steps):
-        sae.step(grads[(args.warmup + t) % ring], w.lr)
-    ktimes = sae.get_kernel_times()
-    sae.set_profiling(False)
-    total_k = sum(ms for ms, _ in ktimes.values())
-    kernels = {name: {"launches": cnt, "ms_per_launch": ms / cnt, "share": ms / total_k}
-               for name, (ms, cnt) in ktimes.items()}
-    step_bytes, worker_bytes, variant = algorithmic_bytes(w, p)
     peak, peak_source = measured_peak()
+
+    def make_inputs(wl, n_sets):
+        scales = synth.workload_scales(wl, args.seed)
+        gen = synth.DeviceGenerator(wl.tensor_sizes, scales, device=dev)
+        x0 = torch.empty(wl.d, device=dev)
+        gen.x0(x0, args.seed)
+        grads = []
+        for t in range(n_sets):
+            g = torch.empty(wl.num_workers, wl.d, device=dev)
+            gen.grads(g, wl.num_workers, args.seed, t, wl.outlier_per_65536, wl.outlier_mult)
+            grads.append(g)
+        return gen, x0, grads
+
+    def make(wl, x0, period, local_steps=1):
+        return sb.Sae(wl.num_workers, wl.tensor_sizes, x0, compressor=wl.compressor, server_compress=wl.server_compress,
+                      mode=wl.mode, avg_period=period, momentum=wl.momentum, weight_decay=wl.weight_decay,
+                      topk_num=wl.topk_num, topk_den=wl.topk_den, local_steps=local_steps)
+
+    def measure(wl, x0, grads, period, steps, warmup, read_step_ahead=False, profile=True, local_steps=1):
+        """`steps` timed steps (CUDA events on the library's stream, max over ranks), then the same steps again
+        with every launch bracketed by events for the per-kernel shares.  read_step_ahead: the caller fetches
+        worker 0's step-ahead point x - e^(0) after every step, inside the timed region -- with p = 1 that one
+        vector is every worker's gradient point."""
+        ring = len(grads)
+        sae = make(wl, x0, period, local_steps)
+        out = torch.empty(wl.d, device=dev) if read_step_ahead else None
+
+        def one(t):
+            sae.step(grads[t % ring], wl.lr)
+            if read_step_ahead:
+                sae.get_step_ahead(0, out)
+
+        for t in range(warmup):
+            one(t)
+        sae.sync()
+        sampler = ClockSampler(local_rank)
+        launches0 = sae.kernel_launches
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        sampler.start()
+        ev0.record()
+        for t in range(steps):
+            one(warmup + t)
+        ev1.record()
+        barrier()
+        clocks = sampler.stop()
+        ms_total = ev0.elapsed_time(ev1)
+        launches = sae.kernel_launches - launches0
+        sae.sync()                                    # raises if the device flagged a range error
+        ms_total = max_over_ranks(ms_total, dev)
+        res = {"steps": steps, "ms_total": ms_total, "ms_per_step": ms_total / steps,
+               "steps_per_s": whole_job_value(steps, ms_total, world), "gpu_launches": launches, "clocks": clocks,
+               "kernels": None}
+        if profile:
+            sae.set_profiling(True)
+            for t in range(steps):
+                one(warmup + t)
+            ktimes = sae.get_kernel_times()
+            sae.set_profiling(False)
+            total_k = sum(ms for ms, _ in ktimes.values())
+            res["kernels"] = {name: {"launches": cnt, "ms_per_launch": ms / cnt, "share": ms / total_k}
+                              for name, (ms, cnt) in ktimes.items()}
+        sae.close()
+        return res
+
+    def fractions(nbytes, ms):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return gbs, gbs / peak, gbs / NOMINAL_HBM_GBS
+
+    # ---- headline: device-resident throughput, state not read between steps ------------------------------
+    K, d = w.num_workers, w.d
+    grad_bytes = 4 * K * d
+    ring = ring_length(args, grad_bytes, p)
+    gen, x0, grads = make_inputs(w, ring)
+    head = measure(w, x0, grads, p, args.steps, args.warmup, local_steps=args.local_steps)
+    ms_per_step, value, kernels = head["ms_per_step"], head["steps_per_s"], head["kernels"]
+    step_bytes, worker_bytes, variant = algorithmic_bytes(w, p)
     wk_ms = kernels["worker_pass"]["ms_per_launch"]
-    achieved = worker_bytes / (wk_ms * 1e-3) / 1e9
+    achieved, frac, frac_nom = fractions(worker_bytes, wk_ms)
     per = WORKER_PASS_DRAM_BYTES.get(variant)
+    sgbs, sfrac, sfrac_nom = fractions(step_bytes, ms_per_step)
     roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": (per[0] * K * d + per[1] * d) if per else None,
+                "frac": frac, "traffic": (per[0] * K * d + per[1] * d) if per else None,
+                "traffic_source": per[2] if per else None,
                 "algorithmic_bytes_per_launch": worker_bytes, "ms_per_launch": wk_ms, "peak_source": peak_source,
-                "frac_of_nominal_8TBs": achieved / 8000.0,
-                "step": {"algorithmic_bytes": step_bytes, "achieved_GBs": step_bytes / (ms_per_step * 1e-3) / 1e9,
-                         "frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
-                         "frac_of_nominal_8TBs": step_bytes / (ms_per_step * 1e-3) / 1e9 / 8000.0},
+                "frac_of_nominal_8TBs": frac_nom,
+                "step": {"algorithmic_bytes": step_bytes, "achieved_GBs": sgbs, "frac": sfrac,
+                         "frac_of_nominal_8TBs": sfrac_nom},
                 "kernels": kernels}
-    sae.close()
-    del sae
+
+    # ---- the loop of Algorithm 1 as the paper runs it: the gradient point is read after every step --------
+    with_step_ahead = None
+    if not args.no_step_ahead and args.local_steps == 1:
+        sa_steps = max(3, min(args.steps, 30))
+        sa = measure(w, x0, grads, p, sa_steps, args.warmup, read_step_ahead=True)
+        sa_bytes, sa_formula = step_ahead_bytes(w, p)
+        gbs, f_meas, f_nom = fractions(sa_bytes, sa["ms_per_step"])
+        with_step_ahead = {"steps_per_s": sa["steps_per_s"], "ms_per_step": sa["ms_per_step"], "steps": sa_steps,
+                           "algorithmic_bytes": sa_bytes, "algorithmic_bytes_formula": sa_formula,
+                           "achieved_GBs": gbs, "frac_of_measured": f_meas, "frac_of_nominal": f_nom,
+                           "gpu_launches": sa["gpu_launches"], "kernels": sa["kernels"], "clocks": sa["clocks"],
+                           "api": "sae_step + sae_get_step_ahead(worker 0) every step, device buffers"}
+
+    # ---- every benchmark configuration, both averaging schedules, a short timed region each ---------------
+    all_configs = None
+    if args.all_configs and world == 1 and args.workload == 4 and not overridden:
+        all_configs = []
+        for idx in range(configs.NUM_WORKLOADS):
+            wl = configs.workload(idx)
+            if idx == 4:
+                xs, gs = x0, grads
+            else:
+                gb = 4 * wl.num_workers * wl.d
+                _, xs, gs = make_inputs(wl, ring_length(args, gb, wl.avg_period_paper))
+            n_steps = {0: 400, 1: 400, 2: 100, 3: 100, 4: max(10, min(args.steps, 30))}[idx]
+            for period in (1, wl.avg_period_paper):
+                if idx == 4 and period == p:
+                    r = head
+                else:
+                    r = measure(wl, xs, gs, period, n_steps, max(args.warmup, 2 * period if period > 1 else 3))
+                sb_, wb_, _ = algorithmic_bytes(wl, period)
+                gbs, f_meas, f_nom = fractions(sb_, r["ms_per_step"])
+                wk = r["kernels"]["worker_pass"]["ms_per_launch"]
+                all_configs.append({"workload": wl.name, "avg_period": period, "steps": r["steps"],
+                                    "steps_per_s": r["steps_per_s"], "ms_per_step": r["ms_per_step"],
+                                    "step_algorithmic_bytes": sb_, "step_achieved_GBs": gbs,
+                                    "step_frac_of_measured": f_meas, "step_frac_of_nominal": f_nom,
+                                    "worker_pass_ms": wk, "worker_pass_algorithmic_bytes": wb_,
+                                    "worker_pass_frac": fractions(wb_, wk)[1],
+                                    "worker_pass_frac_of_nominal": fractions(wb_, wk)[2],
+                                    "kernels": {n: {"launches": v["launches"], "ms_per_launch": v["ms_per_launch"]}
+                                                for n, v in r["kernels"].items()},
+                                    "gpu_launches": r["gpu_launches"], "clocks": r["clocks"],
+                                    "l2": l2_note(4 * wl.num_workers * wl.d, len(gs))})
+            if idx != 4:
+                del xs, gs
+                torch.cuda.empty_cache()
 
     # ---- small workloads: the whole trajectory as ONE captured graph ----------------------------------
     # Configs 0-1 are bound by launch and pipeline latency; with all iterations' gradients resident their
@@ -488,13 +719,13 @@ def main():
     # is periodic: the number of steps is even (scale buffers alternate) and a multiple of p.
     whole_graph = None
     n_traj = w.iterations
-    if K * d <= (1 << 23) and n_traj % 2 == 0 and (p == 0 or n_traj % p == 0):
+    if K * d <= (1 << 23) and n_traj % 2 == 0 and (p == 0 or n_traj % p == 0) and args.local_steps == 1:
         g_all = []
         for t in range(n_traj):
             g = torch.empty(K, d, device=dev)
             gen.grads(g, K, args.seed, t, w.outlier_per_65536, w.outlier_mult)
             g_all.append(g)
-        sae = make()
+        sae = make(w, x0, p)
         for t in range(n_traj):                      # same phase of every schedule at the start of the capture
             sae.step(g_all[t], w.lr)
         sae.sync()
@@ -506,6 +737,7 @@ def main():
         for _ in range(3):
             graph.replay()
         torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
         for _ in range(reps):
             graph.replay()
@@ -526,7 +758,7 @@ def main():
             host_g = torch.empty(K, d, dtype=torch.float32, pin_memory=True)
             host_g.copy_(grads[0])
             host_x = torch.empty(d, dtype=torch.float32, pin_memory=True)
-            sae = make()
+            sae = make(w, x0, p, args.local_steps)
             e2e_steps = max(2, min(args.steps, int(4e9 // grad_bytes) + 2))
             for _ in range(2):
                 sae.step_host(host_g, w.lr)
@@ -548,6 +780,9 @@ def main():
         else:
             e2e = {"value": None, "unit": "steps/s", "skipped": "not enough host memory to pin one gradient set"}
 
+    # the device buffers are no longer needed; the oracle's inputs are generated afresh
+    del grads, x0
+    torch.cuda.empty_cache()
     cb = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cb = cpu_baseline(w, p, args.seed, steps=0, warmup=1)
@@ -556,17 +791,11 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": w.name, "num_workers": K, "d": d, "num_tensors": w.num_tensors,
-                           "compressor": {0: "identity", 1: "scaled_sign", 2: "topk"}[w.compressor],
-                           "avg_period": p, "momentum": w.momentum, "lr": w.lr, "weight_decay": w.weight_decay,
-                           "mode": "saef" if w.mode == configs.SAEF else "ef",
-                           "server_compress": "double-way" if w.server_compress else "single-way",
-                           "topk": f"{w.topk_num}/{w.topk_den}" if w.compressor == configs.TOPK else None,
-                           "local_steps": args.local_steps,
-                           "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
-                           "l2": f"inputs larger than L2: each step reads a fresh {grad_bytes / 1e9:.2f} GB gradient set "
-                                 f"(ring of {ring})"},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": gpu_launches, "roofline": roofline, "cpu_baseline": cb}
+                "config": config_dict(w, p, args, world),
+                "clocks": head["clocks"], "e2e": e2e, "gpu_launches": head["gpu_launches"], "roofline": roofline,
+                "cpu_baseline": cb, "with_step_ahead": with_step_ahead}
+        if all_configs is not None:
+            line["all_configs"] = all_configs
         if whole_graph is not None:
             line["whole_trajectory_graph"] = whole_graph
         print(json.dumps(line), flush=True)

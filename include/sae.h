@@ -228,7 +228,11 @@ int64_t sae_kernel_launches(const sae_handle *h);
  *   sae_shard_attach  makes the rows of one exported blob (any shard's, including this handle's own) known
  *                     to this handle.  Every handle must attach the blobs of all shards before stepping.
  *                     Buffers of another process are mapped with cudaIpcOpenMemHandle (peer access enabled
- *                     lazily) and unmapped by sae_shard_detach or sae_destroy.
+ *                     lazily) and unmapped by sae_shard_detach or sae_destroy.  Rows of the same process on
+ *                     ANOTHER device are taken by their raw pointers after peer access from this handle's
+ *                     device to theirs has been switched on here (cudaDeviceEnablePeerAccess; already on counts
+ *                     as success); if the two devices cannot reach each other the blob is refused with
+ *                     SAE_ERR_INVALID_ARG and nothing is attached, so no kernel ever reads an unmapped row.
  *   sae_shard_detach  forgets every attached row and unmaps other processes' buffers (waits for the stream
  *                     first).  An owner must not be destroyed while another process still maps its rows:
  *                     detach everywhere, synchronise the ranks, then destroy.

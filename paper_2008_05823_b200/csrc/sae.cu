@@ -136,7 +136,7 @@ struct sae_handle {
   const u32** d_tau_rows[2];
   std::vector<void*> ipc_opened;    // mappings of other processes' buffers, closed by sae_destroy
   // cached step graphs
-  int graphs_enabled, graph_misses;
+  int graphs_enabled, graph_misses, graph_pause;
   uint64_t graph_clock;
   std::vector<StepGraph> graphs;
   // profiling
@@ -757,18 +757,47 @@ int do_step(sae_handle* h, const float* grads, float lr) {
       return SAE_OK;
     }
   }
-  // Not seen before.  A caller whose key changes every step (say, a new learning rate each time) would
-  // only pay for captures: give up on graphs after a run of misses.
-  if (++h->graph_misses > 64) { h->graphs_enabled = 0; return do_step_direct(h, grads, lr); }
+  // Not seen before.  Capturing costs far more than a direct step, so a key is only captured when it can come
+  // back: the learning rate must have held still for a step (lr == the previous step's).  A schedule that
+  // changes lr every step (warm-up, cosine) therefore runs direct steps without paying for captures, and
+  // graphs come back by themselves once lr settles.  A run of captures that never hit pauses capturing for a
+  // while instead of switching it off for good.
+  const bool lr_settled = h->t == 0 || lr == h->eta_prev;
+  if (h->graph_pause > 0) { --h->graph_pause; return do_step_direct(h, grads, lr); }
+  if (!lr_settled) return do_step_direct(h, grads, lr);
+  if (++h->graph_misses > 64) { h->graph_misses = 0; h->graph_pause = 256; return do_step_direct(h, grads, lr); }
+  // The capture below runs the host side of the step (which advances the handle's small state) without any
+  // device work; if it fails, that state is put back and the step runs directly, so host and device agree.
+  struct HostState { int64_t t, launches; int esrc, last, rot, srv_pending, tail_pending, recs_srv_fresh; float eta_prev; };
+  const HostState before = {h->t, h->launches, h->esrc, h->last, h->rot, h->srv_pending, h->tail_pending,
+                            h->recs_srv_fresh, h->eta_prev};
+  auto restore = [&]() {
+    h->t = before.t; h->launches = before.launches; h->esrc = before.esrc; h->last = before.last; h->rot = before.rot;
+    h->srv_pending = before.srv_pending; h->tail_pending = before.tail_pending;
+    h->recs_srv_fresh = before.recs_srv_fresh; h->eta_prev = before.eta_prev;
+  };
+  auto fall_back = [&](cudaError_t ce) {
+    h->last_cuda_error = (int)ce; cudaGetLastError();
+    restore();
+    h->graph_pause = 256;
+    return do_step_direct(h, grads, lr);
+  };
   const int64_t launches0 = h->launches;
-  SAE_CUDA(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+  {
+    const cudaError_t cb = cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal);
+    if (cb != cudaSuccess) return fall_back(cb);
+  }
   int rc = do_step_direct(h, grads, lr);
   cudaGraph_t graph = nullptr;
   cudaError_t ce = cudaStreamEndCapture(h->stream, &graph);
   if (rc != SAE_OK || ce != cudaSuccess || !graph) {
     if (graph) cudaGraphDestroy(graph);
-    if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); }
-    return rc != SAE_OK ? rc : SAE_ERR_CUDA;
+    if (rc != SAE_OK) {                             // the step itself was refused; nothing ran on the device
+      if (ce != cudaSuccess) cudaGetLastError();
+      restore();
+      return rc;
+    }
+    return fall_back(ce != cudaSuccess ? ce : cudaErrorUnknown);
   }
   StepGraph e;
   e.key = key; e.exec = nullptr; e.kernels = (int)(h->launches - launches0);
@@ -777,9 +806,10 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   e.stamp = ++h->graph_clock;
   ce = cudaGraphInstantiate(&e.exec, graph, 0);
   cudaGraphDestroy(graph);
-  if (ce != cudaSuccess) { h->last_cuda_error = (int)ce; cudaGetLastError(); return SAE_ERR_CUDA; }
-  SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
-  if (h->graphs.size() >= 32) {               // evict the least recently used graph
+  if (ce != cudaSuccess) return fall_back(ce);
+  ce = cudaGraphLaunch(e.exec, h->stream);
+  if (ce != cudaSuccess) { cudaGraphExecDestroy(e.exec); return fall_back(ce); }
+  if (h->graphs.size() >= 128) {               // evict the least recently used graph
     size_t victim = 0;
     for (size_t q = 1; q < h->graphs.size(); ++q) if (h->graphs[q].stamp < h->graphs[victim].stamp) victim = q;
     cudaGraphExecDestroy(h->graphs[victim].exec);
@@ -896,7 +926,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f; h->local_steps = 1;
-  h->graphs_enabled = 1; h->graph_misses = 0; h->graph_clock = 0;
+  h->graphs_enabled = 1; h->graph_misses = 0; h->graph_pause = 0; h->graph_clock = 0;
   h->fused_ok = (!shard && cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
                  (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
   h->shard = shard ? 1 : 0; h->k0 = k0; h->K_total = cfg->num_workers; h->attached = 0; h->mid_step = 0;
@@ -1206,6 +1236,20 @@ int sae_shard_attach(sae_handle* h, const void* blob_host, size_t bytes) {
     if (h->h_word_rows[(size_t)b.worker_begin + q]) return SAE_ERR_INVALID_ARG;      // rows already attached
   void* base[kShardBufs];
   if (b.pid == (int32_t)getpid()) {
+    if (b.device != h->device) {
+      // rows of another GPU driven by this process: they are only readable from here once peer access is on
+      int can = 0;
+      if (b.device < 0 || cudaDeviceCanAccessPeer(&can, h->device, b.device) != cudaSuccess || !can) {
+        cudaGetLastError();
+        return SAE_ERR_INVALID_ARG;
+      }
+      const cudaError_t pe = cudaDeviceEnablePeerAccess(b.device, 0);
+      if (pe != cudaSuccess && pe != cudaErrorPeerAccessAlreadyEnabled) {
+        h->last_cuda_error = (int)pe; cudaGetLastError();
+        return SAE_ERR_CUDA;
+      }
+      cudaGetLastError();
+    }
     for (int q = 0; q < kShardBufs; ++q) base[q] = b.raw[q];
   } else {
     for (int q = 0; q < kShardBufs; ++q) {

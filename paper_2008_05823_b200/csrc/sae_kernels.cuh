@@ -363,7 +363,11 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 }
 
 // K3 (identity / Top-K): the same aggregation from the dense model differences.
-// COMP 0: C = identity, 2: Top-K with this step's thresholds.
+// COMP 0: C = identity, 2: Top-K with this step's thresholds, 1: scaled sign with this step's scales (the form
+// that closes a p = 1 scaled-sign step in one pass when the caller wants the state right after it: the messages
+// C(Delta^(k)) are re-formed from the momentum rows instead of unpacked from the sign words, so that the same
+// pass over the rows also yields the averaged error; with double-way compression it adds the server's exact
+// L1 partials and sign words like k_server_sign).
 // AVG: the next pre-step averages the local errors; they are functions of the same D^(k) and thresholds
 // this pass already reads, so ebar = (1/K) sum_k (D^(k) - C(D^(k))) is formed here, in k order, instead of
 // in a further pass over D.
@@ -372,7 +376,8 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 // operation that formed it, so the step moves 4 bytes per worker-element less.
 // LSRV != 0 (Top-K): the previous step left its server lines pending -- e = Delta - C(Delta), x = x - C(Delta)
 // and the server's selection words; they are carried out here on the fly with last step's server threshold
-// (LSRV 2) or with C = identity (LSRV 1, single-way), the same operations the apply kernel would have done.
+// (LSRV 2), with last step's server scale (LSRV 3, scaled sign) or with C = identity (LSRV 1, single-way), the
+// same operations the apply kernel would have done.
 // Full tiles are read through a ring of DENSE_RING thread-private 16-byte slots in shared memory filled by
 // asynchronous copies (cp.async): the reads of a thread -- per group of four parameters the server error,
 // (deferred lines) the parameters, (recompute) the old averaged error, then the K rows in k order -- form one
@@ -403,10 +408,14 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
   const bool emit = (COMP == 2) && A.emit_srv;
+  const bool sign_dc = (COMP == 1) && A.emit_srv;        // scaled sign, double-way: the server's L1 partials and words
   const u32 lo = emit ? window_lo(A.tau_srv_prev[ti.j]) : NO_GUESS;
   WarpStage stg; stg.buf = cstage + ((COMP == 2) ? (tid >> 5) * CAND_STAGE : 0); stg.n = 0;
-  if (COMP == 2 && !SUM) {                               // (SUM: no rows are read, so no worker thresholds either)
-    for (int k = tid; k < P.K; k += THREADS) t_k[k] = A.tau_cur[(long long)k * P.T + ti.j];
+  LaneAcc acc; lane_acc_init(acc);
+  if (COMP != 0 && !SUM) {                               // (SUM: no rows are read, so no worker thresholds either)
+    for (int k = tid; k < P.K; k += THREADS)
+      t_k[k] = (COMP == 2) ? A.tau_cur[(long long)k * P.T + ti.j]
+                           : __float_as_uint(A.scale_cur[(long long)k * P.T + ti.j]);
     __syncthreads();
   }
   const long long pbase = ti.poff + ti.t0;
@@ -417,6 +426,8 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   float* xp = A.x + pbase;                               // (LSRV only)
   u32* mwp = A.mask_srv + (pbase >> 5);                  // (LSRV 2 only)
   const u32 t_old = (LSRV == 2) ? A.tau_srv_prev[ti.j] : 0u;
+  const float s_old = (LSRV == 3) ? A.scale_srv_prev[ti.j] : 0.0f;
+  u32* wsp = A.words_srv + (pbase >> 5);                 // (scaled sign, double-way)
   const int lane = tid & 31, warp = tid >> 5;
   if (ti.cnt == TILE) {
     constexpr int NPRE = 1 + (LSRV != 0 ? 1 : 0) + ((RECOMP || SUM) ? 1 : 0);   // reads ahead of the rows, per iteration
@@ -456,9 +467,10 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
       float4 e = take();
       if (LSRV != 0) {
         float4 xv = take();
-        const bool q0 = LSRV == 1 || topk_selected(e.x, t_old), q1 = LSRV == 1 || topk_selected(e.y, t_old);
-        const bool q2 = LSRV == 1 || topk_selected(e.z, t_old), q3 = LSRV == 1 || topk_selected(e.w, t_old);
-        const float c0 = q0 ? e.x : 0.0f, c1 = q1 ? e.y : 0.0f, c2 = q2 ? e.z : 0.0f, c3 = q3 ? e.w : 0.0f;
+        const bool q0 = LSRV != 2 || topk_selected(e.x, t_old), q1 = LSRV != 2 || topk_selected(e.y, t_old);
+        const bool q2 = LSRV != 2 || topk_selected(e.z, t_old), q3 = LSRV != 2 || topk_selected(e.w, t_old);
+        float c0 = q0 ? e.x : 0.0f, c1 = q1 ? e.y : 0.0f, c2 = q2 ? e.z : 0.0f, c3 = q3 ? e.w : 0.0f;
+        if (LSRV == 3) { c0 = sign_code(e.x, s_old); c1 = sign_code(e.y, s_old); c2 = sign_code(e.z, s_old); c3 = sign_code(e.w, s_old); }
         xv.x = __fsub_rn(xv.x, c0); xv.y = __fsub_rn(xv.y, c1); xv.z = __fsub_rn(xv.z, c2); xv.w = __fsub_rn(xv.w, c3);
         st4(xp + i, xv);
         e.x = __fsub_rn(e.x, c0); e.y = __fsub_rn(e.y, c1); e.z = __fsub_rn(e.z, c2); e.w = __fsub_rn(e.w, c3);
@@ -479,11 +491,17 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
           v.x = __fmaf_rn(A.eta, v.x, eold.x); v.y = __fmaf_rn(A.eta, v.y, eold.y);
           v.z = __fmaf_rn(A.eta, v.z, eold.z); v.w = __fmaf_rn(A.eta, v.w, eold.w);
         }
-        const u32 t = (COMP == 2) ? t_k[k] : 0u;
-        const float c0 = (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f;
-        const float c1 = (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f;
-        const float c2 = (COMP == 0 || topk_selected(v.z, t)) ? v.z : 0.0f;
-        const float c3 = (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f;
+        const u32 t = (COMP != 0) ? t_k[k] : 0u;
+        float c0, c1, c2, c3;
+        if (COMP == 1) {
+          const float sk = __uint_as_float(t);
+          c0 = sign_code(v.x, sk); c1 = sign_code(v.y, sk); c2 = sign_code(v.z, sk); c3 = sign_code(v.w, sk);
+        } else {
+          c0 = (COMP == 0 || topk_selected(v.x, t)) ? v.x : 0.0f;
+          c1 = (COMP == 0 || topk_selected(v.y, t)) ? v.y : 0.0f;
+          c2 = (COMP == 0 || topk_selected(v.z, t)) ? v.z : 0.0f;
+          c3 = (COMP == 0 || topk_selected(v.w, t)) ? v.w : 0.0f;
+        }
         a0 = __fadd_rn(a0, c0); a1 = __fadd_rn(a1, c1); a2 = __fadd_rn(a2, c2); a3 = __fadd_rn(a3, c3);
         if (AVG) {
           b0 = __fadd_rn(b0, __fsub_rn(v.x, c0)); b1 = __fadd_rn(b1, __fsub_rn(v.y, c1));
@@ -501,6 +519,11 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
         if (stg.n > CAND_STAGE - 128) stage_flush(stg, A.cand_srv, 0, ti.j);
         stage_row4(stg, lo, mag_key(ds.x), mag_key(ds.y), mag_key(ds.z), mag_key(ds.w));
       }
+      if (COMP == 1 && sign_dc) {                          // (uniform over the block)
+        lane_add4(acc, ds);
+        const u32 w = pack_row4(ds.x >= 0.0f, ds.y >= 0.0f, ds.z >= 0.0f, ds.w >= 0.0f);
+        if ((lane & 7) == 0) wsp[i >> 5] = w;
+      }
     }
     cp_async_wait<0>();
   } else {
@@ -514,24 +537,30 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
         for (int k = 0; k < (SUM ? 0 : P.K); ++k) {
           float v = dp[(long long)k * P.dpad + i];
           if (RECOMP) v = __fmaf_rn(A.eta, v, ebo);
-          const float c = (COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f;
+          const float c = (COMP == 1) ? sign_code(v, __uint_as_float(t_k[k]))
+                                      : ((COMP == 0 || topk_selected(v, t_k[k])) ? v : 0.0f);
           a = __fadd_rn(a, c);
           if (AVG) b = __fadd_rn(b, __fsub_rn(v, c));
         }
         if (AVG) A.ebar[pbase + i] = div_by_k(P, b);
         float eold = ep[i];
         if (LSRV != 0) {
-          qs = LSRV == 1 || topk_selected(eold, t_old);
-          const float cs = qs ? eold : 0.0f;
+          qs = LSRV != 2 || topk_selected(eold, t_old);
+          const float cs = (LSRV == 3) ? sign_code(eold, s_old) : (qs ? eold : 0.0f);
           xp[i] = __fsub_rn(xp[i], cs);
           eold = __fsub_rn(eold, cs);
         }
         ds = __fadd_rn(eold, div_by_k(P, a));
         ep[i] = ds;
+        if (COMP == 1 && sign_dc) lane_add(acc, ds);
       }
       if (LSRV == 2) {
         const u32 w = __ballot_sync(0xffffffffu, qs);
         if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) mwp[(r * THREADS + warp * 32) >> 5] = w;
+      }
+      if (COMP == 1 && sign_dc) {
+        const u32 w = __ballot_sync(0xffffffffu, i < ti.cnt && ds >= 0.0f);
+        if (lane == 0 && (r * THREADS + warp * 32) < ti.cnt) wsp[(r * THREADS + warp * 32) >> 5] = w;
       }
       if (COMP == 2 && lo != NO_GUESS) {
         if (stg.n > CAND_STAGE - 32) stage_flush(stg, A.cand_srv, 0, ti.j);
@@ -540,6 +569,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
     }
   }
   if (COMP == 2) stage_flush(stg, A.cand_srv, 0, ti.j);
+  if (COMP == 1 && sign_dc) warp_commit(acc, A.recs_srv + ti.j, A.status);
 }
 
 // Between the worker pass and the server pass: one thread per (worker, tensor) record turns the exact
@@ -631,6 +661,8 @@ struct ApplyArgs {
   u32* mask_srv;           // [nwords] Top-K: server selection of this step
 
   float eta;
+  float* out;              // (OUT) [d], caller layout: the re-updated parameters, or the step-ahead point x - ebar
+  const float* ebar_out;   // (OUT 2) [dpad] the uniform local error the point is taken at
 };
 
 constexpr int AVG_NONE = 0;
@@ -656,7 +688,10 @@ __device__ __forceinline__ float worker_err(float dk, float s, u32 t) {
 }
 
 // K5: server error, re-update, and (when the next pre-step averages) the averaged worker error.
-template <int COMP, int SRV, int AVG>
+// OUT (a getter that finds the server lines pending and the local errors uniform): the same pass also writes,
+// in the caller's layout, what the getter asked for -- 1: the re-updated parameters x_{t+1}; 2: the step-ahead
+// point x_{t+1} - ebar (Algorithm 1, "One step ahead"; the same single subtraction the export kernel does).
+template <int COMP, int SRV, int AVG, int OUT = 0>
 __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
   __shared__ float s_k[MAX_WORKERS];
   __shared__ u32 t_k[MAX_WORKERS];
@@ -687,6 +722,9 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
   float* ebp = A.ebar + pbase;
   const float* __restrict__ src = (AVG == AVG_RECOMPUTE) ? A.m + pbase : A.D + pbase;
   u32* mwp = A.mask_srv + (pbase >> 5);
+  float* op = (OUT != 0) ? A.out + ti.off + ti.t0 : nullptr;              // caller layout: any 4-byte alignment
+  const float* __restrict__ eop = (OUT == 2) ? A.ebar_out + pbase : nullptr;
+  const bool out_vec = (OUT != 0) && (reinterpret_cast<uintptr_t>(op) & 15) == 0;
 
   if (ti.cnt == TILE) {
 #pragma unroll 2
@@ -701,6 +739,15 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
       apply_elem<COMP, SRV, AVG>(ds.w, x.w, es.w, q3, s_srv, t_srv);
       st4(ep + i, es);
       st4(xp + i, x);
+      if (OUT != 0) {
+        float4 o = x;
+        if (OUT == 2) {
+          const float4 eb = ld4(eop + i);
+          o.x = __fsub_rn(x.x, eb.x); o.y = __fsub_rn(x.y, eb.y); o.z = __fsub_rn(x.z, eb.z); o.w = __fsub_rn(x.w, eb.w);
+        }
+        if (out_vec) st4(op + i, o);
+        else { op[i] = o.x; op[i + 1] = o.y; op[i + 2] = o.z; op[i + 3] = o.w; }
+      }
       if (SRV == 2) {
         u32 w = pack_row4(q0, q1, q2, q3);
         if ((lane & 7) == 0) mwp[i >> 5] = w;
@@ -736,6 +783,8 @@ __global__ void __launch_bounds__(THREADS) k_apply(Plan P, ApplyArgs A) {
         apply_elem<COMP, SRV, AVG>(ep[i], x, es, q, s_srv, t_srv);
         ep[i] = es;
         xp[i] = x;
+        if (OUT == 1) op[i] = x;
+        if (OUT == 2) op[i] = __fsub_rn(x, eop[i]);
         if (AVG != AVG_NONE) {
           const float eb = (AVG == AVG_RECOMPUTE) ? ebp[i] : 0.0f;
           float a = 0.f;

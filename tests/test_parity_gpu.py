@@ -263,6 +263,31 @@ def test_graph_replay_on_a_side_stream(comp, p):
         gpu.close()
 
 
+@pytest.mark.parametrize("comp,p", [(so.SIGN, 1), (so.TOPK, 0)])
+def test_learning_rate_schedule_then_constant_on_a_side_stream(comp, p):
+    """A learning rate that changes on every step (warm-up, then decay) for more steps than the graph cache
+    tolerates misses, then held constant: steps run directly while it moves and as replayed graphs once it
+    has settled -- the same bits as the oracle either way."""
+    import torch
+    K, sizes = 4, [33, 4096, 5000]
+    d = sum(sizes)
+    scales = synth.tensor_scales(5, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(5, d)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        orc = so.Oracle(K, sizes, x0, compressor=comp, avg_period=p, topk_den=20, threads=4)
+        gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), compressor=comp, avg_period=p, topk_den=20)
+        gs = [synth.grads_numpy(5, t, K, sizes, scales) for t in range(2)]
+        bufs = [torch.from_numpy(g).cuda() for g in gs]
+        lrs = [0.1 * (t + 1) / 40 for t in range(40)] + [0.1 * 0.97 ** t for t in range(40)] + [0.01] * 12
+        for t, lr in enumerate(lrs):
+            orc.step(gs[t % 2], lr)
+            gpu.step(bufs[t % 2], lr)
+            if t in (39, 79, 85, len(lrs) - 1):
+                compare_state(gpu, orc, comp, tag=f"schedule comp={comp} t={t + 1}")
+        gpu.close()
+
+
 @pytest.mark.parametrize("comp", [so.SIGN, so.TOPK])
 def test_two_runs_give_identical_bytes(comp):
     """Run-to-run determinism: the exact L1 is an integer sum (atomics in any order), histograms are integer

@@ -104,7 +104,20 @@ def test_sharded_handle_checks_its_arguments():
     other = sb.Sae(4, SIZES + [5], torch.zeros(d + 5, device="cuda"), shard=(2, 2))
     with pytest.raises(sb.SaeError):
         a.shard_attach(other.shard_export())                             # a different parameter list
+    # rows of the same process on a device this handle's device cannot reach (here: one that does not exist):
+    # refused on the host, nothing attached, no kernel ever sees the pointers
+    peer = sb.Sae(4, SIZES, x0, shard=(2, 2))
+    foreign = bytearray(peer.shard_export())
+    assert int.from_bytes(foreign[12:16], "little", signed=True) == torch.cuda.current_device()
+    foreign[12:16] = int(torch.cuda.device_count()).to_bytes(4, "little", signed=True)
+    with pytest.raises(sb.SaeError) as err:
+        a.shard_attach(bytes(foreign))
+    assert err.value.status == sb.ERR_INVALID_ARG
+    with pytest.raises(sb.SaeError):
+        a.step_begin(g, 0.1)                                             # still not every worker attached
+    a.shard_attach(peer.shard_export())                                  # the untouched blob is accepted
     a.close()
+    peer.close()
     other.close()
 
 
