@@ -189,7 +189,16 @@ int64_t sae_iteration(const sae_handle *h);
 int64_t sae_num_params(const sae_handle *h);
 int64_t sae_num_words(const sae_handle *h);
 
-/* Waits for the stream; returns and clears the sticky device status (SAE_OK or SAE_ERR_RANGE...). */
+/* Waits for the stream; returns and clears the sticky device status (SAE_OK or SAE_ERR_RANGE...).
+ *
+ * SAE_ERR_TIMEOUT: the worker and server passes move tiles into shared memory with asynchronous bulk copies
+ * and wait for them on shared-memory barriers.  Every such wait is bounded in time: a warp that has polled
+ * for longer than the handle's limit raises the status and the kernel returns (after the copying warp has
+ * waited, under the same limit, for the copies it still had in flight) -- it never traps and never spins
+ * without a bound.  The limit is one second unless the environment variable SAE_WAIT_LIMIT_US (microseconds,
+ * 1 .. 60 000 000, read by sae_init) sets another; a kernel in which a copy was lost therefore ends within
+ * about twice the limit.  After SAE_ERR_TIMEOUT the handle's state is that of a half-finished step: destroy it
+ * (or restore a checkpoint); the CUDA context and other handles are unaffected. */
 int sae_sync(sae_handle *h);
 
 /*

@@ -9,6 +9,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <unistd.h>
 #include <new>
@@ -36,7 +37,7 @@ const char* const kSlotNames[SAE_NUM_KERNELS] = {"worker_pass", "server_aggregat
 
 struct EventPair { int slot; cudaEvent_t a, b; };
 
-struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm, tail, fresh; const float* grads; float lr, eta_prev; };
+struct StepGraphKey { int esrc, last, avg_after, srv_pending, rot, comm, tail, fresh, reader; const float* grads; float lr, eta_prev; };
 struct StepGraph { StepGraphKey key; cudaGraphExec_t exec; int kernels, esrc_after, last_after, pending_after, rot_after, tail_after, fresh_after; uint64_t stamp; };
 
 }  // namespace
@@ -52,7 +53,6 @@ struct sae_handle {
   long long *d_off, *d_poff;
   // state
   float *x, *e_srv, *ebar, *m, *D;
-  float* etmp;           // [dpad] the pending average, materialised for getters only
   CUtensorMap tm_m;      // momentum rows [K][dpad] as a tensor map (folded-averaging worker pass)
   CUtensorMap tm_D;      // stored model differences [K][dpad] (folded Top-K tail with stored differences)
   int fused_gen_ok;      // Top-K, p != 1, K = 8 or 16: the tail of a non-averaging step is folded into the next worker pass
@@ -90,6 +90,7 @@ struct sae_handle {
   long long cand_stride;
   u32* status;
   u32* status_host;      // pinned
+  WaitCfg wc;            // how long device waits poll before they give up (and the test-only dropped copy)
   float* staging;        // sae_step_host
   float* out_stage;      // sae_get_params_host
   double* mismatch;      // sae_get_mismatch
@@ -115,6 +116,8 @@ struct sae_handle {
   // server lines) is left to the worker pass of the next step, which reads the same momentum rows anyway
   int fused_topk_ok;
   int tail_pending;                 // the last step stopped after its threshold select (scaled sign: after its scales)
+  int reader;                       // the caller has been reading x / e between steps: a p = 1 scaled-sign step then
+                                    // stops after its scales whatever K is, and the getter closes it in one pass
   int recs_srv_fresh;               // a server pass has added to the server's L1 records since they were last finalized
   float* ssum;                      // [dpad] ordered worker-axis sum of the selected entries (folded form)
   int avg_external;                 // the averaging sum is all-reduced by the caller instead of pulled in k order
@@ -219,7 +222,7 @@ cudaError_t dalloc(T** p, size_t count) {
 }
 
 void free_all(sae_handle* h) {
-  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->ebar_alt, h->m, h->D, h->etmp,
+  void* ptrs[] = {h->d_tile_tensor, h->d_first_tile, h->d_n, h->d_off, h->d_poff, h->x, h->e_srv, h->ebar, h->ebar_alt, h->m, h->D,
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
                   h->tau_srv, h->recs, h->recs_alt, h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
@@ -301,24 +304,28 @@ int flush_tail(sae_handle* h) {
   const bool dc = h->cfg.server_compress != 0;
   ServerArgs sa;
   memset(&sa, 0, sizeof(sa));
+  sa.wc = h->wc;
   if (h->cfg.compressor == SAE_COMPRESSOR_SIGN) {
-    // scaled sign, p = 1: the open tail is the server pass over the last step's message words (still in place)
+    // Scaled sign, p = 1: the open tail is the whole server pass of the last step, and the average of the local
+    // errors is pending with it.  One pass over the K momentum rows does both: it re-forms every message
+    // C(Delta^(k)) = +-s_k from Delta^(k) = fma(eta, m^(k), ebar) (the bits the worker pass packed), adds them
+    // and the errors Delta^(k) - C(Delta^(k)) up in k order, and writes the server's Delta, its L1 partials and
+    // sign words and the averaged error -- which thereby becomes the plain uniform error of the next step.
+    if (h->esrc != ESRC_PENDING_AVG) return SAE_ERR_INVALID_ARG;
     const bool pending = h->srv_pending != 0;
     LAUNCH(h, S_FINALIZE, k_finalize_scales, (P.T + THREADS - 1) / THREADS, 0, P.T, h->d_n, h->recs, h->scale[h->last],
            h->recs_srv, (pending && dc && h->recs_srv_fresh) ? h->scale_srv : nullptr);
-    sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[h->last]; sa.words_srv = h->words_srv;
-    sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv; sa.status = h->status; sa.x = h->x;
-    sa.scale_srv_prev = h->scale_srv;
-    const int tpb = std::max(1, std::min(8, P.ntiles / (h->num_sms * 16)));
-    const int nblk = (P.ntiles + tpb - 1) / tpb;
-    if (pending) {
-      if (dc) LAUNCH(h, S_SERVER, (k_server_sign<true, false, false, true>), nblk, P, sa, tpb);
-      else LAUNCH(h, S_SERVER, (k_server_sign<false, false, false, true>), nblk, P, sa, tpb);
-    } else if (dc) LAUNCH(h, S_SERVER, k_server_sign<true>, nblk, P, sa, tpb);
-    else LAUNCH(h, S_SERVER, k_server_sign<false>, nblk, P, sa, tpb);
+    sa.e_srv = h->e_srv; sa.scale_cur = h->scale[h->last]; sa.words_srv = h->words_srv; sa.recs_srv = h->recs_srv;
+    sa.status = h->status; sa.x = h->x; sa.scale_srv_prev = h->scale_srv; sa.emit_srv = dc ? 1 : 0;
+    sa.m = h->m; sa.ebar_in = h->ebar; sa.ebar = h->ebar; sa.eta = h->eta_prev;
+    const int lsrv = pending ? (dc ? 3 : 1) : 0;
+    if (lsrv == 0) LAUNCH_DENSE(h, (k_server_dense<1, true, true, 0>), P.ntiles, P, sa);
+    else if (lsrv == 1) LAUNCH_DENSE(h, (k_server_dense<1, true, true, 1>), P.ntiles, P, sa);
+    else LAUNCH_DENSE(h, (k_server_dense<1, true, true, 3>), P.ntiles, P, sa);
     h->recs_srv_fresh = 1;
     h->srv_pending = 1;
     h->tail_pending = 0;
+    h->esrc = ESRC_UNIFORM;
     return check_launch(h);
   }
   sa.e_srv = h->e_srv; sa.tau_cur = h->tau[h->last]; sa.status = h->status;
@@ -341,11 +348,21 @@ int flush_tail(sae_handle* h) {
   return check_launch(h);
 }
 
-int flush_server(sae_handle* h) {
+template <int COMP, int SRV>
+void launch_apply_out(sae_handle* h, int out_kind, const ApplyArgs& aa) {
+  if (out_kind == 0) LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_NONE>), h->P.ntiles, h->P, aa);
+  else if (out_kind == 1) LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_NONE, 1>), h->P.ntiles, h->P, aa);
+  else LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_NONE, 2>), h->P.ntiles, h->P, aa);
+}
+
+// out_kind 1 / 2: the apply kernel also writes the re-updated parameters / the step-ahead point x - ebar
+// (uniform local errors) to `out`, caller layout, so that a getter needs no export pass of its own.
+int flush_server(sae_handle* h, int out_kind = 0, float* out = nullptr) {
   { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
   if (!h->srv_pending) return SAE_OK;
   ApplyArgs aa;
   memset(&aa, 0, sizeof(aa));
+  aa.out = out; aa.ebar_out = ebar_now(h);
   aa.e_srv = h->e_srv; aa.x = h->x; aa.ebar = h->ebar; aa.scale_srv = h->scale_srv; aa.recs_srv = h->recs_srv;
   if (h->inline_fin) {      // the last step accumulated into the buffer before the current rotation index
     L1Record* rs[4] = {h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3};
@@ -354,10 +371,9 @@ int flush_server(sae_handle* h) {
   aa.tau_srv = h->tau_srv; aa.mask_srv = h->mask_srv;
   const bool dcs = h->cfg.server_compress != 0;
   if (h->cfg.compressor == SAE_COMPRESSOR_TOPK) {
-    if (dcs) LAUNCH(h, S_APPLY, (k_apply<2, 2, AVG_NONE>), h->P.ntiles, h->P, aa);
-    else LAUNCH(h, S_APPLY, (k_apply<2, 0, AVG_NONE>), h->P.ntiles, h->P, aa);
-  } else if (dcs) LAUNCH(h, S_APPLY, (k_apply<1, 1, AVG_NONE>), h->P.ntiles, h->P, aa);
-  else LAUNCH(h, S_APPLY, (k_apply<1, 0, AVG_NONE>), h->P.ntiles, h->P, aa);
+    if (dcs) launch_apply_out<2, 2>(h, out_kind, aa); else launch_apply_out<2, 0>(h, out_kind, aa);
+  } else if (dcs) launch_apply_out<1, 1>(h, out_kind, aa);
+  else launch_apply_out<1, 0>(h, out_kind, aa);
   h->srv_pending = 0;
   return check_launch(h);
 }
@@ -498,12 +514,14 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
   sp.mu = c.momentum; sp.eta = lr; sp.lambda = c.weight_decay;
   sp.saef = (c.mode == SAE_MODE_SAEF); sp.wd = (c.weight_decay != 0.0f);
   WorkerArgs wa;
+  wa.wc = h->wc;
   wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = ebar_now(h); wa.x = h->x;
   wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
   wa.cand = cand_args(h, false);
   ServerArgs sa;
   memset(&sa, 0, sizeof(sa));
+  sa.wc = h->wc;
   sa.e_srv = h->e_srv; sa.words = h->words; sa.scale_cur = h->scale[cur]; sa.D = h->D; sa.tau_cur = h->tau[cur];
   // inline_fin: rotating record buffers (see the handle)
   L1Record* rs3[4] = {h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3};
@@ -539,6 +557,8 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     return check_launch(h);
   }
   if (c.compressor == SAE_COMPRESSOR_SIGN) {
+    // an open tail that the next worker pass cannot take over (no sum vector, or this step does not fold): close it
+    if (h->tail_pending && (h->ssum == nullptr || sp.wd)) { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
     // The model differences need not be stored when the previous error was uniform and the next
     // pre-step averages: the averaging pass recomputes them from m and ebar with the same fused op.
     const bool pending_in = h->esrc == ESRC_PENDING_AVG;
@@ -555,11 +575,15 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // (Worth it from 32 workers on: the unpacking server pass costs K additions per parameter, the streaming
     // one and the extra vector the worker pass writes do not depend on K -- config 4: 7.82 -> 7.62 ms per step,
     // config 2 with 16 workers: 0.931 ms either way.)
-    const bool fold_sign = defer_avg && lazy_ok && !h->inline_fin && h->local_steps <= 1 && h->ssum != nullptr;
-    if (h->tail_pending && !(pending_in && fold_sign)) return SAE_ERR_INVALID_ARG;
+    // The same open form, at any K, for a caller that reads the state between steps: the getter closes the step
+    // in one pass over the momentum rows (flush_tail), which leaves the plain uniform error behind.
+    const bool fold_sign = defer_avg && lazy_ok && !h->inline_fin && h->local_steps <= 1 &&
+                           (h->ssum != nullptr || h->reader);
+    if (h->tail_pending && !(pending_in && fold_sign && h->ssum != nullptr)) return SAE_ERR_INVALID_ARG;
     if (pending_in) {
       FusedArgs fa;
       memset(&fa, 0, sizeof(fa));
+      fa.wc = h->wc;
       fa.g = grads; fa.m = h->m; fa.ebar = ebar_now(h); fa.x = h->x; fa.scale_prev = h->scale[h->last];
       fa.words = h->words; fa.recs = recs_now; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
       fa.ssum = h->tail_pending ? h->ssum : nullptr;
@@ -645,6 +669,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
       if (!lazy_ok || (!nod && h->esrc != ESRC_LAZY_TOPK)) return SAE_ERR_INVALID_ARG;
       FusedArgs fa;
       memset(&fa, 0, sizeof(fa));
+      fa.wc = h->wc;
       fa.g = grads; fa.m = h->m; fa.ebar = ebar_other(h); fa.ebar_out = ebar_now(h); fa.x = h->x; fa.D = h->D;
       fa.tau_prev = h->tau[h->last]; fa.ssum = h->ssum; fa.cand = wa.cand; fa.status = h->status;
       fa.eta_prev = h->eta_prev;
@@ -727,6 +752,7 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
 // the gradient pointer and the learning rate; a step with a key seen before is replayed with a single
 // cudaGraphLaunch, which takes the per-kernel launch cost off the host (small workloads are bound by it).
 int do_step(sae_handle* h, const float* grads, float lr) {
+  if (h->esrc == ESRC_PENDING_AVG) h->reader = 0;       // nobody looked at the state since the last step
   bool usable = h->graphs_enabled && !h->profiling && h->stream != nullptr && h->stream != cudaStreamLegacy &&
                 h->stream != cudaStreamPerThread;
   if (usable) {
@@ -740,13 +766,13 @@ int do_step(sae_handle* h, const float* grads, float lr) {
 
   StepGraphKey key;
   key.esrc = h->esrc; key.last = h->last; key.srv_pending = h->srv_pending; key.rot = h->rot;
-  key.comm = communicates(h) ? 1 : 0; key.tail = h->tail_pending; key.fresh = h->recs_srv_fresh;
+  key.comm = communicates(h) ? 1 : 0; key.tail = h->tail_pending; key.fresh = h->recs_srv_fresh; key.reader = h->reader;
   key.avg_after = (h->cfg.avg_period > 0 && ((h->t + 2) % h->cfg.avg_period == 0)) ? 1 : 0;
   key.grads = grads; key.lr = lr; key.eta_prev = h->eta_prev;     // every value a captured kernel argument depends on
   for (size_t q = 0; q < h->graphs.size(); ++q) {
     StepGraph& e = h->graphs[q];
     if (e.key.esrc == key.esrc && e.key.last == key.last && e.key.avg_after == key.avg_after &&
-        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.tail == key.tail && e.key.fresh == key.fresh && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
+        e.key.srv_pending == key.srv_pending && e.key.rot == key.rot && e.key.comm == key.comm && e.key.tail == key.tail && e.key.fresh == key.fresh && e.key.reader == key.reader && e.key.grads == key.grads && e.key.lr == key.lr && e.key.eta_prev == key.eta_prev) {
       SAE_CUDA(h, cudaGraphLaunch(e.exec, h->stream));
       h->launches += e.kernels;
       h->esrc = e.esrc_after; h->last = e.last_after; h->srv_pending = e.pending_after; h->rot = e.rot_after;
@@ -820,25 +846,44 @@ int do_step(sae_handle* h, const float* grads, float lr) {
   return SAE_OK;
 }
 
-ExportArgs export_args(sae_handle* h, int what, int k, bool need_error) {
+// The pending average of a p = 1 scaled-sign step whose server pass is already done, formed in place: the
+// averaged error becomes the plain uniform error (what the next worker pass would have formed, same bits).
+int close_pending_avg(sae_handle* h) {
+  if (h->esrc != ESRC_PENDING_AVG) return SAE_OK;
+  { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }          // (an open tail closes the average with it)
+  if (h->esrc != ESRC_PENDING_AVG) return SAE_OK;
+  LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, h->ebar, h->scale[h->last], h->eta_prev, h->ebar);
+  h->esrc = ESRC_UNIFORM;
+  return check_launch(h);
+}
+
+ExportArgs export_args(sae_handle* h, int what, int k) {
   ExportArgs ea;
   ea.x = h->x; ea.e_srv = h->e_srv; ea.m = h->m; ea.D = h->D; ea.ebar = ebar_now(h);
   ea.scale_last = h->scale[h->last]; ea.tau_last = h->tau[h->last];
   ea.esrc = h->esrc; ea.what = what; ea.k = k; ea.saef = (h->cfg.mode == SAE_MODE_SAEF);
-  if (h->esrc == ESRC_PENDING_AVG) {
-    // the averaged error exists only implicitly: form it in a scratch vector, leave the state alone
-    if (need_error)
-      LAUNCH(h, S_EXPORT, k_materialize_avg, h->P.ntiles, h->P, h->m, ebar_now(h), h->scale[h->last], h->eta_prev, h->etmp);
-    ea.ebar = h->etmp;
-    ea.esrc = ESRC_UNIFORM;
-  }
   return ea;
 }
 
 int export_vec(sae_handle* h, int what, int k, float* out) {
-  if (what != EXP_M) { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }     // x and e must be up to date
-  else { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
-  const ExportArgs ea = export_args(h, what, k, what == EXP_WERR || what == EXP_STEP_AHEAD);
+  if (what == EXP_M) {
+    int rct = flush_tail(h);
+    if (rct != SAE_OK) return rct;
+  } else {
+    h->reader = 1;                                       // x and e must be up to date, and will be asked for again
+    const bool saef = h->cfg.mode == SAE_MODE_SAEF;
+    const bool need_error = what == EXP_WERR || (what == EXP_STEP_AHEAD && saef);
+    if (need_error) { int rca = close_pending_avg(h); if (rca != SAE_OK) return rca; }
+    { int rct = flush_tail(h); if (rct != SAE_OK) return rct; }
+    // the pending server lines and the answer in one pass where the answer is x, or x minus a uniform error
+    int out_kind = 0;
+    if (what == EXP_X || (what == EXP_STEP_AHEAD && !saef)) out_kind = 1;
+    else if (what == EXP_STEP_AHEAD && h->esrc == ESRC_UNIFORM) out_kind = 2;
+    if (h->srv_pending && out_kind != 0) return flush_server(h, out_kind, out);
+    int rcf = flush_server(h);
+    if (rcf != SAE_OK) return rcf;
+  }
+  const ExportArgs ea = export_args(h, what, k);
   LAUNCH(h, S_EXPORT, k_export, h->P.ntiles, h->P, ea, out);
   return check_launch(h);
 }
@@ -926,6 +971,12 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f; h->local_steps = 1;
+  // Device waits give up after SAE_WAIT_LIMIT_US microseconds of polling (default: one second).
+  // SAE_DEBUG_DROP_COPY=<item> (testing only) makes the producer of the worker / server passes announce the
+  // copies of that work item without issuing them, so that the waits on it run out and SAE_ERR_TIMEOUT is raised.
+  h->wc.limit_us = 0; h->wc.drop_item = 0;
+  if (const char* ev = getenv("SAE_WAIT_LIMIT_US")) { const long v = atol(ev); if (v > 0 && v <= 60000000L) h->wc.limit_us = (u32)v; }
+  if (const char* ev = getenv("SAE_DEBUG_DROP_COPY")) { const long v = atol(ev); if (v >= 0 && v < (1L << 31) - 1) h->wc.drop_item = (u32)v + 1u; }
   h->graphs_enabled = 1; h->graph_misses = 0; h->graph_pause = 0; h->graph_clock = 0;
   h->fused_ok = (!shard && cfg->compressor == SAE_COMPRESSOR_SIGN && cfg->avg_period == 1 && cfg->num_workers <= 32 &&
                  (cfg->num_workers & (cfg->num_workers - 1)) == 0) ? 1 : 0; h->last_cuda_error = 0; h->launches = 0; h->profiling = 0;
@@ -969,11 +1020,10 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->d_off, T); ALLOC0(h->d_poff, T);
   ALLOC0(h->x, dpad); ALLOC0(h->e_srv, dpad); ALLOC0(h->ebar, dpad);
   if (!h->mu0) ALLOC0(h->m, (size_t)K * dpad);
-  if (h->fused_ok) ALLOC0(h->etmp, dpad);
   if (need_D) ALLOC0(h->D, (size_t)K * dpad);
   if (h->topk_nod) ALLOC0(h->ebar_alt, dpad);
   h->fused_topk_ok = (h->topk_nod && (K == 8 || K == 16) && dpad < (1ll << 31) && d < (1ll << 31)) ? 1 : 0;
-  h->tail_pending = 0; h->recs_srv_fresh = 0;
+  h->tail_pending = 0; h->recs_srv_fresh = 0; h->reader = 0;
   h->fused_gen_ok = (!shard && topk && cfg->avg_period != 1 && (K == 8 || K == 16) && dpad < (1ll << 31) &&
                      d < (1ll << 31)) ? 1 : 0;
   // (scaled sign: the folded server pass is for large problems, p = 1, K a power of two up to 32)
@@ -1107,6 +1157,7 @@ int shard_begin(sae_handle* h, const float* grads, float lr) {
   sp.mu = c.momentum; sp.eta = lr; sp.lambda = c.weight_decay;
   sp.saef = (c.mode == SAE_MODE_SAEF); sp.wd = (c.weight_decay != 0.0f);
   WorkerArgs wa;
+  wa.wc = h->wc;
   wa.g = grads; wa.m = h->m; wa.D = h->D; wa.ebar = h->ebar; wa.x = h->x;
   wa.scale_prev = h->scale[h->last]; wa.tau_prev = h->tau[h->last];
   wa.words = h->words; wa.scale_cur = h->scale[cur]; wa.recs = h->recs; wa.status = h->status;
@@ -1141,6 +1192,7 @@ int shard_end(sae_handle* h) {
   const bool avg_after = c.avg_period > 0 && ((h->t + 2) % c.avg_period == 0);
   ServerArgs sa;
   memset(&sa, 0, sizeof(sa));
+  sa.wc = h->wc;
   sa.e_srv = h->e_srv; sa.words_srv = h->words_srv; sa.scale_srv = h->scale_srv; sa.recs_srv = h->recs_srv;
   sa.status = h->status; sa.word_rows = h->d_word_rows; sa.scale_rows = h->d_scale_rows[cur];
   ApplyArgs aa;
@@ -1525,7 +1577,8 @@ int sae_get_mismatch(sae_handle* h, double* out_host) {
   { int rcf = flush_server(h); if (rcf != SAE_OK) return rcf; }
   if (!h->mismatch) SAE_CUDA(h, dalloc(&h->mismatch, 2));
   SAE_CUDA(h, cudaMemsetAsync(h->mismatch, 0, 2 * sizeof(double), h->stream));
-  const ExportArgs ea = export_args(h, EXP_WERR, 0, true);
+  { int rca = close_pending_avg(h); if (rca != SAE_OK) return rca; }
+  const ExportArgs ea = export_args(h, EXP_WERR, 0);
   LAUNCH(h, S_EXPORT, k_mismatch, h->P.ntiles, h->P, ea, h->mismatch);
   int rc = check_launch(h);
   if (rc != SAE_OK) return rc;

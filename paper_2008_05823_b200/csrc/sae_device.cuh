@@ -279,10 +279,18 @@ __device__ __forceinline__ u32 pack_row4(bool p0, bool p1, bool p2, bool p3) {
 }
 
 // ---- mbarrier / bulk-copy (TMA) primitives ----------------------------------------------------------
-// Every wait on an mbarrier is bounded: after WAIT_LIMIT polls the waiter gives up and the caller raises
-// STATUS_TIMEOUT in the handle's status word.
-constexpr u32 WAIT_LIMIT = 1u << 24;
+// Every wait on an mbarrier is bounded in time: a waiter that has polled for longer than the limit (the
+// handle's, one second unless set otherwise) gives up, the caller raises STATUS_TIMEOUT in the handle's status
+// word and the kernel returns; nothing traps and nothing spins without a limit.
+constexpr u32 DEFAULT_WAIT_US = 1000000u;
 constexpr u32 STATUS_TIMEOUT = 2u;
+
+// How the kernels wait, passed by value with their arguments.
+struct WaitCfg {
+  u32 limit_us;       // 0 = DEFAULT_WAIT_US
+  u32 drop_item;      // testing only: 1 + index of the work item whose copies the producer announces (expect_tx)
+                      // but does not issue, so that the waits on it run out; 0 = none
+};
 
 __device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
 
@@ -295,10 +303,18 @@ __device__ __forceinline__ void mbar_arrive(u64* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(u64* bar, u32 bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Bounded wait for the completion of the phase with the given parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity) {
+__device__ __forceinline__ u64 global_ns() {
+  u64 t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait for the completion of the phase with the given parity; false = gave up.  The clock is read once
+// per 256 polls (the first reading starts the interval), so the common case -- done within a few polls -- pays
+// nothing for the bound.
+__device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity, const WaitCfg& wc) {
   const u32 addr = smem_u32(bar);
-  for (u32 it = 0; it < WAIT_LIMIT; ++it) {
+  u64 t0 = 0;
+  for (u32 it = 0;; ++it) {
     u32 done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -308,8 +324,12 @@ __device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity) {
         : "r"(addr), "r"(parity)
         : "memory");
     if (done) return true;
+    if ((it & 255u) == 255u) {
+      const u64 now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > (u64)(wc.limit_us ? wc.limit_us : DEFAULT_WAIT_US) * 1000ull) return false;
+    }
   }
-  return false;
 }
 // 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on `bar`.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {

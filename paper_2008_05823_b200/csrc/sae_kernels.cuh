@@ -55,6 +55,7 @@ struct WorkerArgs {
   float* scale_cur;       // [K][T]
   L1Record* recs;         // [K][T]
   u32* status;
+  WaitCfg wc;
 };
 
 // ---------------------------------------------------------------------------------------------------
@@ -90,6 +91,7 @@ struct ServerArgs {
   float* x;                        // [dpad]
   const float* scale_srv_prev;     // [T] server scales of the previous step (double-way)
   u32* mask_srv;                   // [nwords] Top-K: the server's selection of the previous step (written when pending)
+  WaitCfg wc;
 };
 
 // K3 (scaled sign): Delta = e + (1/K) sum_k C(Delta^(k)) from the packed messages; with double-way
@@ -218,8 +220,10 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         __syncthreads();                          // nobody still reads the previous tile's staged rows
         if (tid == 0) {
           mbar_arrive_expect_tx(&s_bar, (LAZY ? 2u : 1u) * TILE * (u32)sizeof(float));
-          bulk_load(s_e, ep, TILE * (u32)sizeof(float), &s_bar);
-          if (LAZY) bulk_load(s_x, xp, TILE * (u32)sizeof(float), &s_bar);
+          if (A.wc.drop_item != (u32)tile + 1u) {
+            bulk_load(s_e, ep, TILE * (u32)sizeof(float), &s_bar);
+            if (LAZY) bulk_load(s_x, xp, TILE * (u32)sizeof(float), &s_bar);
+          }
         }
       }
       const int i = tid * SRV_E;
@@ -277,7 +281,7 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         }
       }
       if constexpr (STAGE) {
-        if (!mbar_wait(&s_bar, phase)) {           // gave up: flag it and leave (the whole block does)
+        if (!mbar_wait(&s_bar, phase, A.wc)) {           // gave up: flag it and leave (the whole block does)
           if (tid == 0) atomicOr(A.status, STATUS_TIMEOUT);
           return;
         }
@@ -421,7 +425,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   const long long pbase = ti.poff + ti.t0;
   float* ep = A.e_srv + pbase;
   const float* __restrict__ dp = (RECOMP ? A.m : A.D) + pbase;
-  const float* __restrict__ eo = A.ebar_in + pbase;      // read only when RECOMP
+  const float* eo = A.ebar_in + pbase;                   // read only when RECOMP (may be the buffer A.ebar writes)
   const float* __restrict__ sump = A.ssum + pbase;       // read only when SUM
   float* xp = A.x + pbase;                               // (LSRV only)
   u32* mwp = A.mask_srv + (pbase >> 5);                  // (LSRV 2 only)

@@ -122,6 +122,7 @@ struct FusedArgs {
   u32* status;
   float eta_prev;
   int g_tma_ok;            // the gradient buffer admits a tensor map (16-byte aligned base and row pitch)
+  WaitCfg wc;
 };
 
 template <int K, int MODE>
@@ -215,24 +216,34 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
           const int s = i % FW_STAGES;
           int ok = 1;
           if (lane == 0) {
-            if (i >= FW_STAGES && !mbar_wait(&S.empty[s], ((i / FW_STAGES) - 1) & 1)) {
+            if (i >= FW_STAGES && !mbar_wait(&S.empty[s], ((i / FW_STAGES) - 1) & 1, A.wc)) {
               atomicOr(A.status, STATUS_TIMEOUT);
               ok = 0;
             }
           }
-          if (!__shfl_sync(0xffffffffu, ok, 0)) return;
+          if (!__shfl_sync(0xffffffffu, ok, 0)) {
+            // Gave up on item i: nobody releases a stage again.  Before this warp returns it waits (bounded) for
+            // the copies it already issued into each stage.
+            if (lane < FW_STAGES) {
+              const int last = i - 1;
+              const int j = last - ((last - lane) % FW_STAGES + FW_STAGES) % FW_STAGES;
+              if (last >= 0 && j >= 0) mbar_wait(&S.full[lane], (j / FW_STAGES) & 1, A.wc);
+            }
+            return;
+          }
           if (lane == l) { FwItem t = cur; t.h = hh; S.item[s] = t; }
           if (lane < G::KH) S.sc[s][lane] = scale_k;
           __syncwarp();
           if (cnt == 0) {
             if (lane == 0) mbar_arrive(&S.full[s]);
           } else if (lane == 0) {
+            const bool drop = A.wc.drop_item == (u32)fw_range_of(p0 + l, chunk_log2) + 1u;   // (testing only)
             const u32 ebytes = (hh == 0 && !GEN) ? (u32)((cnt + 31) & ~31) * 4u : 0u;    // rows are padded to 32 elements
             const int chunks = (cnt + FW_BOX - 1) / FW_BOX;
             constexpr u32 BOXB = (u32)(G::KH * FW_BOX * 4);
             mbar_arrive_expect_tx(&S.full[s], ebytes + (u32)chunks * BOXB * ((gtma ? 2u : 1u) + (GEN ? 1u : 0u)));
-            if (hh == 0 && !GEN) bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);  // the old ebar travels with the first group
-            for (int c = 0; c < chunks; ++c) {
+            if (hh == 0 && !GEN && !drop) bulk_load(S.e[s], A.ebar + pbase, ebytes, &S.full[s]);  // the old ebar travels with the first group
+            for (int c = 0; c < (drop ? 0 : chunks); ++c) {
               tma_load_2d(&S.m[s][c * G::KH * FW_BOX], &tm_m, (int)pbase + c * FW_BOX, hh * G::KH, &S.full[s]);
               if (GEN) tma_load_2d(&S.dd[s][c * G::KH * FW_BOX], &tm_d, (int)pbase + c * FW_BOX, hh * G::KH, &S.full[s]);
               if (gtma) tma_load_2d(&S.g[s][c * G::KH * FW_BOX], &tm_g, (int)goff + c * FW_BOX, hh * G::KH, &S.full[s]);
@@ -265,7 +276,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
     for (int i = 0; i < nmine * G::HALVES; ++i) {
       const int hh = i % G::HALVES;
       const int s = i % FW_STAGES;
-      if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
+      if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1, A.wc)) {
         if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
         return;
       }
@@ -340,7 +351,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   for (int i = 0; i < nmine * G::HALVES; ++i) {
     const int hh = i % G::HALVES;
     const int s = i % FW_STAGES;
-    if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1)) {
+    if (!mbar_wait(&S.full[s], (i / FW_STAGES) & 1, A.wc)) {
       if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
       return;
     }
@@ -367,7 +378,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
       const u32 tk = TOPK ? __float_as_uint(S.sc[s][kl0]) : 0u;
       // ebar' of this range comes from the averager warps (MODE 2: nothing is handed over, but the averagers
       // must be done with the stage before the workers release it)
-      if (!mbar_wait(&S.avgd[s], (i / FW_STAGES) & 1)) {
+      if (!mbar_wait(&S.avgd[s], (i / FW_STAGES) & 1, A.wc)) {
         if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
         return;
       }
@@ -462,11 +473,11 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
   }
 }
 
-// The pending average on its own (getters): etmp = (1/K) sum_k ( fma(eta, m_k, ebar) - C(...) ).
-__global__ void __launch_bounds__(THREADS) k_materialize_avg(Plan P, const float* __restrict__ m,
-                                                              const float* __restrict__ ebar,
+// The pending average on its own (getters): etmp = (1/K) sum_k ( fma(eta, m_k, ebar) - C(...) ).  etmp may be
+// ebar itself: a thread reads its element of ebar before it writes it.
+__global__ void __launch_bounds__(THREADS) k_materialize_avg(Plan P, const float* __restrict__ m, const float* ebar,
                                                               const float* __restrict__ scale_prev, float eta_prev,
-                                                              float* __restrict__ etmp) {
+                                                              float* etmp) {
   const TileInfo ti = tile_info(P, blockIdx.x);
   for (int i = threadIdx.x; i < ti.cnt; i += THREADS) {
     const long long p = ti.poff + ti.t0 + i;

@@ -16,8 +16,9 @@
 // Ragged tails and gradient rows that are not 16-byte aligned cannot use bulk copies; for those items
 // the producer only publishes the tile description and the consumers load from global memory.
 //
-// Every wait on an mbarrier is bounded: after WAIT_LIMIT polls the waiter raises STATUS_TIMEOUT in
-// the status word and leaves the loop.
+// Every wait on an mbarrier is bounded: a waiter that has polled for longer than the handle's limit raises
+// STATUS_TIMEOUT in the status word and leaves the loop; the producer, the last to leave, first waits (with the same
+// bound) for the copies it still has in flight.
 #pragma once
 #include "sae_kernels.cuh"
 
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
         if (lane == l && cur.cnt > 0) {
           const int i = i0 + l;
           const int s = i % WT_STAGES;
-          if (i >= WT_STAGES && !mbar_wait(&S.empty[s], ((i / WT_STAGES) - 1) & 1)) {
+          if (i >= WT_STAGES && !mbar_wait(&S.empty[s], ((i / WT_STAGES) - 1) & 1, A.wc)) {
             atomicOr(A.status, STATUS_TIMEOUT);
             ok = false;
           } else {
@@ -120,17 +121,28 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
             if (cur.vec) {
               constexpr u32 B = TILE * sizeof(float);
               mbar_arrive_expect_tx(&S.full[s], (MU0 ? 2 : 3) * B);
-              bulk_load(S.buf[s][0], A.g + cur.gofs, B, &S.full[s]);
-              if (!MU0) bulk_load(S.buf[s][1], A.m + cur.wbase, B, &S.full[s]);
-              bulk_load(S.buf[s][2], (ESRC == ESRC_UNIFORM) ? (A.ebar + cur.pbase) : (A.D + cur.wbase), B,
-                        &S.full[s]);
+              if (A.wc.drop_item != (u32)(wb + l * G) + 1u) {
+                bulk_load(S.buf[s][0], A.g + cur.gofs, B, &S.full[s]);
+                if (!MU0) bulk_load(S.buf[s][1], A.m + cur.wbase, B, &S.full[s]);
+                bulk_load(S.buf[s][2], (ESRC == ESRC_UNIFORM) ? (A.ebar + cur.pbase) : (A.D + cur.wbase), B,
+                          &S.full[s]);
+              }
             } else {
               mbar_arrive(&S.full[s]);
             }
           }
         }
         __syncwarp();
-        if (!__all_sync(0xffffffffu, ok)) return;
+        if (!__all_sync(0xffffffffu, ok)) {
+          // Gave up on item i0 + l.  The consumers never release a stage again; before this warp -- the last
+          // one to leave -- returns, it waits (bounded) for the copies already on their way into each stage.
+          if (lane < WT_STAGES) {
+            const int last = i0 + l - 1;                           // last item issued
+            const int j = last - ((last - lane) % WT_STAGES + WT_STAGES) % WT_STAGES;   // ... into stage `lane`
+            if (last >= 0 && j >= 0) mbar_wait(&S.full[lane], (j / WT_STAGES) & 1, A.wc);
+          }
+          return;
+        }
       }
     }
     return;
@@ -149,7 +161,7 @@ __global__ void __launch_bounds__(WT_THREADS, SAE_WT_BLOCKS_PER_SM) k_worker_tma
   long long w = blockIdx.x;
   for (int i = 0; w < nitems; ++i, w += gridDim.x) {
     const int s = i % WT_STAGES;
-    if (!mbar_wait(&S.full[s], (i / WT_STAGES) & 1)) {
+    if (!mbar_wait(&S.full[s], (i / WT_STAGES) & 1, A.wc)) {
       if (lane == 0) atomicOr(A.status, STATUS_TIMEOUT);
       return;
     }

@@ -134,3 +134,52 @@ def test_config4_embedding_scale_first_step():
         words = gpu.get_state(sb.STATE_WORKER_WORDS, k).cpu().numpy().view(np.uint32)[: (n0 + 31) // 32]
         assert_same(f"embedding words[{k}]", words, so.pack_signs(delta, [n0]))
     gpu.close()
+
+
+@pytest.mark.parametrize("p,steps", [(1, 8), (2, 6)])
+def test_one_embedding_sized_tensor_whole_trajectory(p, steps):
+    """The one shape a sample of whole tensors cannot reach at full worker count: a single tensor of
+    23 440 896 elements (config 4's embedding) for 32 workers -- 5723 tiles per worker feeding one L1 record,
+    the folded two-halves ring of the 32-worker pass on a tensor that never ends, the open server pass of the
+    p = 1 form and (p = 2) stored and recomputed differences in turn.  Every step: parameters, server error,
+    all 32 scales; first, middle and last step: every worker's momentum, error, step-ahead point and sign
+    words, and the server's message."""
+    import psutil
+    import torch
+    from parity_util import compare_state, compare_server_messages
+    K, n = 32, 30522 * 768
+    if psutil.virtual_memory().available < 6 * K * n * 4 + (8 << 30):
+        pytest.skip("the oracle's arrays for this case need about 20 GB of host memory")
+    sizes = [n]
+    scales = synth.tensor_scales(4, 1, -5.0, -2.0)
+    gen = synth.DeviceGenerator(sizes, scales)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        x0 = torch.empty(n, device="cuda")
+        gen.x0(x0, 4)
+        kw = dict(compressor=so.SIGN, avg_period=p, momentum=0.9)
+        gpu = sb.Sae(K, sizes, x0, **kw)
+        orc = so.Oracle(K, sizes, x0.cpu().numpy(), threads=so.max_threads(), **kw)
+        gbuf = [torch.empty(K, n, device="cuda") for _ in range(2)]
+        for t in range(steps):
+            g = gbuf[t % 2]
+            gen.grads(g, K, 4, t)
+            gpu.step(g, 0.1)
+            gh = g.cpu().numpy()
+            if t == 0:
+                assert_same("generator row", gh[K - 1, -5000:],
+                            synth.grads_numpy_range(4, 0, K - 1, n - 5000, 5000, scales[0]))
+            orc.step(gh, 0.1)
+            del gh
+            tag = f"one tensor p={p} t={t + 1}"
+            if t in (0, steps // 2, steps - 1):
+                compare_state(gpu, orc, so.SIGN, tag=tag)
+                compare_server_messages(gpu, orc, so.SIGN, 1, tag=tag)
+            else:
+                gpu.sync()
+                assert_same(f"{tag} x", gpu.get_params().cpu().numpy(), orc.get(orc.X))
+                assert_same(f"{tag} e_srv", gpu.get_state(sb.STATE_SERVER_ERROR).cpu().numpy(), orc.get(orc.E_SRV))
+                for k in range(K):
+                    assert_same(f"{tag} scale[{k}]", gpu.get_state(sb.STATE_WORKER_SCALES, k).cpu().numpy(),
+                                orc.get(orc.SCALES, k))
+        assert not orc.range_flag
+        gpu.close()

@@ -563,3 +563,43 @@ def test_sign_folded_server_pass_checkpoint_and_graphs():
         compare_server_messages(a, orc, so.SIGN, 1, tag="continued")
         compare_server_messages(b, orc, so.SIGN, 1, tag="restored")
         a.close(); b.close()
+
+
+@pytest.mark.parametrize("K,comp,dc,mode", [(32, so.SIGN, 1, so.SAEF), (16, so.SIGN, 1, so.SAEF), (4, so.SIGN, 0, so.SAEF),
+                                            (8, so.SIGN, 1, so.EF), (8, so.TOPK, 1, so.SAEF), (16, so.TOPK, 0, so.SAEF)])
+def test_step_ahead_point_read_after_every_step(K, comp, dc, mode):
+    """Algorithm 1 as the paper runs it (p = 1): after every step the caller fetches the point where the next
+    gradient is evaluated, x_{t+1} - e_{t+1}^(k).  Above the small-problem limit, on a side stream (step
+    graphs), with unaligned output buffers; the caller also stops reading for a few steps and resumes, and
+    reads the plain parameters in between.  Every fetched vector and, at the end, the whole state against
+    the oracle."""
+    import torch
+    big = (1 << 24) // K + 40_000
+    sizes = [33, 4096, big - 70_000, 5000, 3 * 4096 + 7, 60_000]
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(21, len(sizes), -4.0, -1.0)
+    x0 = synth.x0_numpy(21, d)
+    kw = dict(compressor=comp, server_compress=dc, mode=mode, avg_period=1, momentum=0.9, topk_den=50)
+    orc = so.Oracle(K, sizes, x0, threads=8, **kw)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
+        gs = [synth.grads_numpy(21, t, K, sizes, scales) for t in range(2)]
+        bufs = [torch.from_numpy(g).cuda() for g in gs]
+        raw = torch.empty(d + 3, device="cuda")
+        quiet = {5, 6, 7}                                   # steps after which nobody reads
+        for t in range(12):
+            lr = 0.1 if t < 9 else 0.05
+            orc.step(gs[t % 2], lr)
+            gpu.step(bufs[t % 2], lr)
+            if t in quiet:
+                continue
+            out = raw[t % 4:t % 4 + d]                      # any 4-byte alignment
+            w = t % K
+            gpu.get_step_ahead(w, out)
+            assert_same(f"step-ahead point t={t + 1} worker {w}", out.cpu().numpy(), orc.step_ahead(w))
+            if t % 3 == 0:
+                gpu.get_params(out)
+                assert_same(f"x t={t + 1}", out.cpu().numpy(), orc.get(orc.X))
+        compare_state(gpu, orc, comp, tag="read every step, end")
+        compare_server_messages(gpu, orc, comp, dc, tag="read every step, end")
+        gpu.close()
