@@ -8,6 +8,7 @@
 
 #include <cuda.h>
 #include <cudaTypedefs.h>
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -106,6 +107,7 @@ struct sae_handle {
   int topk_nod;            // Top-K with p = 1: model differences never stored, two uniform-error buffers
   float* ebar_alt;
   int64_t launches;
+  long long max_n;         // largest tensor
   // sharded operation: this handle owns workers k0 .. k0+P.K-1 of K_total; the server lines run on every shard
   int shard, k0, K_total;
   Plan P_all;                       // the plan with K = K_total (server pass, averaging)
@@ -257,15 +259,24 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   int2* work = own ? h->work_srv : h->work;
   u32* work_count = own ? h->work_count_srv : h->work_count;
   u32* cand_n = own ? h->cand_n_srv : h->cand_n;
-  LAUNCH(h, S_TOPK_SELECT, k_topk_decide, (pairs + THREADS - 1) / THREADS, cand, rows, h->d_n, h->cfg.topk_num,
-         h->cfg.topk_den, tau_guess, cand_n, fb, fb_total, work, work_count);
+  // One launch settles every pair whose candidate list holds the threshold, and small tensors whose window
+  // failed; the server's single row is settled there entirely.  For the workers, large tensors whose window
+  // failed (all of them at the first step) go through the distributed three-level select, whose launches
+  // find an empty work list otherwise.
+  // (A server row with a tensor of more than 2^22 elements keeps the distributed select as well: one block
+  // would take too long over it.)
+  const bool distributed = fb != h->fb_srv || h->max_n > (1ll << 22);
+  const int inline_max = distributed ? (1 << 16) : 0x7fffffff;
+  LAUNCH(h, S_TOPK_SELECT, k_topk_select_window, pairs, P, cand, rows, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess,
+         tau_out, fb, fb_total, inline_max);
+  if (!distributed) return;
   const long long items = (long long)P.ntiles * rows;
   LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, work, work_count);
   const long long hist_grid = 8LL * h->persistent_blocks;
   for (int level = 0; level < 3; ++level) {
     LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, src, cand_n, sel, hist, work, work_count);
     LAUNCH(h, S_TOPK_SELECT, k_topk_select, pairs, P.T, level, h->d_n, h->cfg.topk_num, h->cfg.topk_den, hist, sel,
-           tau_out, work_count);
+           tau_out, work_count, fb);
   }
 }
 
@@ -968,6 +979,8 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   h->cfg = *cfg;
   h->sizes.assign(cfg->tensor_sizes, cfg->tensor_sizes + T);
   h->cfg.tensor_sizes = h->sizes.data();
+  h->max_n = 0;
+  for (int j = 0; j < T; ++j) h->max_n = std::max<long long>(h->max_n, h->sizes[j]);
   h->device = cfg->device;
   h->stream = (cudaStream_t)cfg->stream;
   h->t = 0; h->esrc = ESRC_UNIFORM; h->last = 0; h->eta_prev = 0.0f; h->local_steps = 1;

@@ -13,6 +13,14 @@
 //
 // Fallback -- the select reads the values themselves, only for the (row, tensor) pairs whose window
 // failed (first step, a jump of the threshold, ties, zeros).  Both paths give the same exact key.
+//
+// One launch settles the common case (k_topk_select_window: one block per (row, tensor)): a list that holds the
+// threshold is resolved by two histogram passes over it in shared memory -- the keys of a list lie in a narrow
+// window above `lo`, so they are binned by their distance from `lo` and spread evenly over the bins -- and a
+// pair whose window failed is resolved by the same block with the three-level radix select over its values
+// when the tensor is small.  Only large tensors whose window failed go to the work list of the distributed
+// three-level select (k_topk_worklist, then k_topk_hist / k_topk_select per level), whose launches find the
+// list empty otherwise.
 #pragma once
 #include "sae_device.cuh"
 
@@ -266,12 +274,15 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
 // One block per (row, tensor): find the bin holding the rank-th largest key, update prefix/rank, clear
 // the histogram.  After level 2 the prefix is the threshold key itself (and the work list is released).
 __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const int* __restrict__ n, u32 num, u32 den,
-                                                          u32* hist, SelectState* st, u32* tau, u32* work_count) {
+                                                          u32* hist, SelectState* st, u32* tau, u32* work_count,
+                                                          const u32* __restrict__ fallback) {
   __shared__ u32 part[THREADS];
   __shared__ u32 above[THREADS];
   __shared__ u32 sh_bin, sh_rank;
   const int rj = blockIdx.x;              // row * T + j
   const int j = rj % T;
+  if (level == 2 && rj == 0 && threadIdx.x == 0) *work_count = 0u;      // (nobody reads the list any more)
+  if (!fallback[rj]) return;              // settled by k_topk_select_window: nothing was queued for this pair
   const u32 rank = (level == 0) ? topk_count_of(n[j], num, den) : st[rj].rank;
   const u32 old_prefix = (level == 0) ? 0u : st[rj].prefix;
   __syncthreads();
@@ -280,11 +291,100 @@ __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const
     const u32 prefix = (level == 0) ? sh_bin : ((old_prefix << 10) | sh_bin);
     st[rj].prefix = prefix;
     st[rj].rank = sh_rank;
-    if (level == 2) {
-      tau[rj] = prefix;
-      if (rj == 0) *work_count = 0u;
+    if (level == 2) tau[rj] = prefix;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// The whole select of one (row, tensor) in one block.
+//
+// Window path (the list did not overflow and holds at least k keys, so the k-th largest key of the tensor is
+// the k-th largest key of the list): every key of the list is >= lo.  Pass 1 bins rel = key - lo in steps of
+// 2^WIN_SHIFT over WIN_BINS bins and counts the keys above that range (the bulk of the selected entries: a
+// heavy tail, counted per thread and reduced, not binned); the rank that is left is located from the top of
+// the histogram.  Pass 2 bins the keys of that one bin by their low WIN_SHIFT bits, which gives the exact key.
+// If the k-th largest key lies above the binned range (the threshold rose by more than the range in one step)
+// the pair is treated like a failed window.
+//
+// Failed window: tensors of at most inline_max elements are settled here by the three-level radix select
+// (11 + 10 + 10 bits) over their values, read by this block alone; larger ones raise their fallback flag for
+// the distributed select that follows.
+constexpr int WIN_SHIFT = 8;
+constexpr int WIN_BINS = 2048;            // covers 2^19 key units above lo: twice the window below the old threshold
+
+__global__ void __launch_bounds__(THREADS) k_topk_select_window(Plan P, CandArgs C, int rows, u32 num, u32 den,
+                                                                 DeltaSrc src, const u32* tau_guess, u32* tau_out,
+                                                                 u32* fallback, u32* fallback_total, int inline_max) {
+  __shared__ u32 sh[HIST_BINS];
+  __shared__ u32 part[THREADS];
+  __shared__ u32 above[THREADS];
+  __shared__ u32 sh_bin, sh_rank, sh_above;
+  const int tid = threadIdx.x;
+  const int rj = blockIdx.x;              // row * T + j
+  const int row = rj / C.T, j = rj - row * C.T;
+  const int n = P.n[j];
+  const u32 kk = topk_count_of(n, num, den);
+  const u32 cnt = C.count[rj];
+  const u32 lo = window_lo(tau_guess[rj]);
+  bool ok = lo != NO_GUESS && cnt <= (u32)C.cap[j] && cnt >= kk;
+  for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
+  if (tid == 0) sh_above = 0u;
+  __syncthreads();
+  if (tid == 0) C.count[rj] = 0u;         // (every thread has read the cursor: the barrier above)
+  if (ok) {
+    const u32* __restrict__ keys = C.keys + (long long)row * C.stride + C.off[j];
+    u32 mine = 0;
+    for (u32 i = tid; i < cnt; i += THREADS) {
+      const u32 rel = keys[i] - lo;
+      if (rel >= ((u32)WIN_BINS << WIN_SHIFT)) ++mine;
+      else atomicAdd(sh + (rel >> WIN_SHIFT), 1u);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if ((tid & 31) == 0 && mine) atomicAdd(&sh_above, mine);
+    __syncthreads();
+    const u32 over = sh_above;
+    if (kk <= over) {
+      ok = false;                         // (uniform: every thread reads the same count)
+      __syncthreads();
+      for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
+      __syncthreads();
+    } else {
+      walk_from_top(sh, WIN_BINS, kk - over, part, above, &sh_bin, &sh_rank);     // (clears the bins)
+      const u32 bin = sh_bin, rank = sh_rank;
+      for (u32 i = tid; i < cnt; i += THREADS) {
+        const u32 rel = keys[i] - lo;
+        if ((rel >> WIN_SHIFT) == bin) atomicAdd(sh + (rel & ((1u << WIN_SHIFT) - 1u)), 1u);
+      }
+      __syncthreads();
+      walk_from_top(sh, 1024, rank, part, above, &sh_bin, &sh_rank);
+      if (tid == 0) {
+        tau_out[rj] = lo + (bin << WIN_SHIFT) + sh_bin;
+        fallback[rj] = 0u;
+      }
+      return;
     }
   }
+  // ---- the window failed ----
+  if (tid == 0) atomicAdd(fallback_total, 1u);
+  if (n > inline_max) {
+    if (tid == 0) fallback[rj] = 1u;      // a large tensor: left to the distributed select
+    return;
+  }
+  if (tid == 0) fallback[rj] = 0u;
+  const float* __restrict__ bp = (src.recompute ? src.m : src.buf) + (long long)row * P.dpad + P.poff[j];
+  const float* __restrict__ eb = src.ebar + P.poff[j];               // read only when recomputing
+  u32 prefix = 0u, rank = kk;
+  for (int level = 0; level < 3; ++level) {
+    for (int i = tid; i < n; i += THREADS)
+      hist_elem(mag_key(src.recompute ? __fmaf_rn(src.eta, bp[i], eb[i]) : bp[i]), level, prefix, sh);
+    __syncthreads();
+    walk_from_top(sh, level == 0 ? HIST_BINS : 1024, rank, part, above, &sh_bin, &sh_rank);
+    prefix = (level == 0) ? sh_bin : ((prefix << 10) | sh_bin);
+    rank = sh_rank;
+    __syncthreads();                      // (sh_bin / sh_rank are rewritten by the next level)
+  }
+  if (tid == 0) tau_out[rj] = prefix;
 }
 
 }  // namespace sae
