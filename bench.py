@@ -609,6 +609,8 @@ def main():
         for t in range(warmup):
             one(t)
         sae.sync()
+        topk = wl.compressor == configs.TOPK
+        fb0 = sae.get_state(sb.STATE_TOPK_FALLBACKS).cpu().tolist() if topk else None
         sampler = ClockSampler(local_rank)
         launches0 = sae.kernel_launches
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -627,6 +629,11 @@ def main():
         res = {"steps": steps, "ms_total": ms_total, "ms_per_step": ms_total / steps,
                "steps_per_s": whole_job_value(steps, ms_total, world), "gpu_launches": launches, "clocks": clocks,
                "kernels": None}
+        if topk:     # (row, tensor) pairs whose candidate window missed the threshold during the timed steps
+            fb1 = sae.get_state(sb.STATE_TOPK_FALLBACKS).cpu().tolist()
+            res["topk_window_misses_per_step"] = {"workers": (fb1[0] - fb0[0]) / steps, "server": (fb1[1] - fb0[1]) / steps,
+                                                  "pairs": {"workers": wl.num_workers * wl.num_tensors,
+                                                            "server": wl.num_tensors}}
         if profile:
             sae.set_profiling(True)
             for t in range(steps):
@@ -656,6 +663,7 @@ def main():
     per = WORKER_PASS_DRAM_BYTES.get(variant)
     sgbs, sfrac, sfrac_nom = fractions(step_bytes, ms_per_step)
     roofline = {"bound": "hbm", "kernel": "worker_pass", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "topk_window_misses_per_step": head.get("topk_window_misses_per_step"),
                 "frac": frac, "traffic": (per[0] * K * d + per[1] * d) if per else None,
                 "traffic_source": per[2] if per else None,
                 "algorithmic_bytes_per_launch": worker_bytes, "ms_per_launch": wk_ms, "peak_source": peak_source,
@@ -708,6 +716,8 @@ def main():
                                                 for n, v in r["kernels"].items()},
                                     "gpu_launches": r["gpu_launches"], "clocks": r["clocks"],
                                     "l2": l2_note(4 * wl.num_workers * wl.d, len(gs))})
+                if "topk_window_misses_per_step" in r:
+                    all_configs[-1]["topk_window_misses_per_step"] = r["topk_window_misses_per_step"]
             if idx != 4:
                 del xs, gs
                 torch.cuda.empty_cache()

@@ -77,6 +77,9 @@ struct sae_handle {
   u32 *cand_keys, *cand_keys_srv, *cand_count, *cand_count_srv, *fb, *fb_srv, *fb_total;
   long long* d_cand_off;
   int* d_cand_cap;
+  int* d_sel_list;       // [T] the order in which the one-launch select takes the tensors
+  int n_sel_long;        // how many of them (the first ones) have long candidate regions
+  int* d_wlog2;          // [T] width of each tensor's candidate window (log2 of key units; WINDOW_ALL: whole tensor)
   int2* work;            // work list of the radix select: data items and candidate chunks
   u32* work_count;
   u32* cand_n;           // [K][T] candidates captured for this step's select
@@ -228,7 +231,7 @@ void free_all(sae_handle* h) {
                   h->words, h->words_srv, h->mask_srv, h->scale[0], h->scale[1], h->scale_srv, h->tau[0], h->tau[1],
                   h->tau_srv, h->recs, h->recs_alt, h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3, h->hist, h->sel, h->status, h->staging, h->out_stage, h->mismatch,
                   h->cand_keys, h->cand_keys_srv, h->cand_count, h->cand_count_srv, h->fb, h->fb_srv, h->fb_total,
-                  h->d_cand_off, h->d_cand_cap, h->work, h->work_count, h->cand_n, h->ssum};
+                  h->d_cand_off, h->d_cand_cap, h->d_wlog2, h->d_sel_list, h->work, h->work_count, h->cand_n, h->ssum};
   for (void* p : ptrs) if (p) cudaFree(p);
   void* srv_sel[] = {h->hist_srv, h->work_count_srv, h->cand_n_srv, h->sel_srv, h->work_srv};
   for (void* p : srv_sel) if (p) cudaFree(p);
@@ -263,12 +266,29 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   // failed; the server's single row is settled there entirely.  For the workers, large tensors whose window
   // failed (all of them at the first step) go through the distributed three-level select, whose launches
   // find an empty work list otherwise.
-  // (A server row with a tensor of more than 2^22 elements keeps the distributed select as well: one block
+  // (A server row with a tensor of more than 2^20 elements keeps the distributed select as well: one block
   // would take too long over it.)
-  const bool distributed = fb != h->fb_srv || h->max_n > (1ll << 22);
-  const int inline_max = distributed ? (1 << 16) : 0x7fffffff;
-  LAUNCH(h, S_TOPK_SELECT, k_topk_select_window, pairs, P, cand, rows, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess,
-         tau_out, fb, fb_total, inline_max);
+  const bool distributed = fb != h->fb_srv || h->max_n > (1ll << 20);
+  const int inline_max = distributed ? SAE_TOPK_INLINE_MAX : 0x7fffffff;
+  // Tensors with long candidate regions (the first n_sel_long of the list).  With p = 1 the lists stay short of
+  // their regions and one block of 1024 threads settles each (config 3: 0.619 -> 0.599 ms per step); without the
+  // per-step averaging the unsent entries pile up below the threshold, the lists are several times longer and
+  // a single block is bound by its shared-memory atomics: their chunks go to the distributed select instead,
+  // which spreads them over the device (config 3, p = 20: 0.927 -> 0.896 ms).
+  const bool long_inline = h->topk_nod || !distributed;
+  const int n_long = long_inline ? h->n_sel_long : 0;
+  if (n_long > 0) {
+    LaunchScope ls(h, S_TOPK_SELECT);
+    k_topk_select_window<1024><<<(unsigned)(rows * n_long), 1024, 0, h->stream>>>(
+        P, cand, h->d_sel_list, n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb, fb_total,
+        inline_max, 0x7fffffff, cand_n, work, work_count);
+  }
+  if (P.T > n_long) {
+    LaunchScope ls(h, S_TOPK_SELECT);
+    k_topk_select_window<THREADS><<<(unsigned)(rows * (P.T - n_long)), THREADS, 0, h->stream>>>(
+        P, cand, h->d_sel_list + n_long, P.T - n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb,
+        fb_total, inline_max, long_inline ? 0x7fffffff : SEL_LONG_REGION, cand_n, work, work_count);
+  }
   if (!distributed) return;
   const long long items = (long long)P.ntiles * rows;
   LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, work, work_count);
@@ -297,6 +317,7 @@ CandArgs cand_args(sae_handle* h, bool server) {
   c.off = h->d_cand_off; c.cap = h->d_cand_cap; c.stride = h->cand_stride;
   c.count = server ? h->cand_count_srv : h->cand_count;
   c.T = h->P.T;
+  c.wlog2 = h->d_wlog2;
   return c;
 }
 
@@ -1056,7 +1077,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->hist, topk ? KT * HIST_BINS : 0);
   ALLOC0(h->sel, topk ? KT : 0);
   std::vector<long long> cand_off(T, 0);
-  std::vector<int> cand_cap(T, 0);
+  std::vector<int> cand_cap(T, 0), wlog2(T, SAE_TOPK_WINDOW_LOG2);
   h->cand_stride = 0;
   if (topk) {
     // room for 8 k_j + 1024 keys per (row, tensor): the window normally catches about 2 k_j
@@ -1066,6 +1087,10 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
       unsigned long long cap = 8 * kk + 1024;
       if (cap > (unsigned long long)h->sizes[j]) cap = (unsigned long long)h->sizes[j];
       cand_off[j] = h->cand_stride; cand_cap[j] = (int)cap;
+      // window width: the whole tensor where the region holds it; else 2 % of the old threshold, up to 8 times
+      // wider for small k (whose threshold moves more from step to step and whose region has room to spare)
+      if (cap >= (unsigned long long)h->sizes[j]) wlog2[j] = WINDOW_ALL;
+      else for (unsigned long long w = 2; w <= 8 && w * kk <= 1024; w *= 2) wlog2[j] += 1;
       h->cand_stride += (long long)((cap + 3) / 4 * 4);
     }
   }
@@ -1073,7 +1098,14 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->cand_keys_srv, topk ? (size_t)h->cand_stride : 0);
   ALLOC0(h->cand_count, topk ? KT : 0); ALLOC0(h->cand_count_srv, topk ? T : 0);
   ALLOC0(h->fb, topk ? KT : 0); ALLOC0(h->fb_srv, topk ? T : 0); ALLOC0(h->fb_total, 2);
-  ALLOC0(h->d_cand_off, T); ALLOC0(h->d_cand_cap, T);
+  ALLOC0(h->d_cand_off, T); ALLOC0(h->d_cand_cap, T); ALLOC0(h->d_wlog2, T); ALLOC0(h->d_sel_list, T);
+  std::vector<int> sel_list(T);
+  for (int j = 0; j < T; ++j) sel_list[j] = j;
+  // the order in which the one-launch select takes the tensors: longest candidate regions first, so that their
+  // blocks start first and the short ones fill in behind them
+  std::stable_sort(sel_list.begin(), sel_list.end(), [&](int a, int b) { return cand_cap[a] > cand_cap[b]; });
+  h->n_sel_long = 0;
+  for (int j = 0; j < T; ++j) if (cand_cap[j] > SEL_LONG_REGION) h->n_sel_long += 1;
   ALLOC0(h->work, topk ? (size_t)ntiles * K + (size_t)K * (h->cand_stride / CAND_CHUNK + T) : 0);
   ALLOC0(h->work_count, 1); ALLOC0(h->cand_n, topk ? KT : 0);
 #if SAE_TOPK_PARALLEL_SELECT
@@ -1094,6 +1126,8 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   TRY(cudaMemcpyAsync(h->d_poff, poff.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
   TRY(cudaMemcpyAsync(h->d_cand_off, cand_off.data(), sizeof(long long) * T, cudaMemcpyHostToDevice, h->stream));
   TRY(cudaMemcpyAsync(h->d_cand_cap, cand_cap.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_wlog2, wlog2.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
+  TRY(cudaMemcpyAsync(h->d_sel_list, sel_list.data(), sizeof(int) * T, cudaMemcpyHostToDevice, h->stream));
 #undef ALLOC0
   if (rc == SAE_OK) {
     Plan& P = h->P;

@@ -308,28 +308,35 @@ __device__ __forceinline__ u64 global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait for the completion of the phase with the given parity; false = gave up.  The clock is read once
-// per 256 polls (the first reading starts the interval), so the common case -- done within a few polls -- pays
-// nothing for the bound.
+// One poll: true when the phase with the given parity has completed.  (A poll that finds it incomplete suspends
+// the thread for a hardware-defined time, a few microseconds on B200, or until the phase completes.)
+__device__ __forceinline__ u32 mbar_try(u32 addr, u32 parity) {
+  u32 done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(addr), "r"(parity)
+      : "memory");
+  return done;
+}
+// The path taken when the first poll came back empty-handed, kept out of line so that the kernels' hot loops
+// carry a single poll instruction per wait (inlining the timed loop at every wait cost the three-array worker
+// pass 16 %): polls on and gives up once the clock, read after every failed poll, shows the limit exceeded.
+static __device__ __noinline__ bool mbar_wait_slow(u32 addr, u32 parity, u32 limit_us) {
+  const u64 t0 = global_ns();
+  const u64 limit_ns = (u64)(limit_us ? limit_us : DEFAULT_WAIT_US) * 1000ull;
+  for (;;) {
+    if (mbar_try(addr, parity)) return true;
+    if (global_ns() - t0 > limit_ns) return false;
+  }
+}
+// Bounded wait for the completion of the phase with the given parity; false = gave up.
 __device__ __forceinline__ bool mbar_wait(u64* bar, u32 parity, const WaitCfg& wc) {
   const u32 addr = smem_u32(bar);
-  u64 t0 = 0;
-  for (u32 it = 0;; ++it) {
-    u32 done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(addr), "r"(parity)
-        : "memory");
-    if (done) return true;
-    if ((it & 255u) == 255u) {
-      const u64 now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > (u64)(wc.limit_us ? wc.limit_us : DEFAULT_WAIT_US) * 1000ull) return false;
-    }
-  }
+  if (mbar_try(addr, parity)) return true;
+  return mbar_wait_slow(addr, parity, wc.limit_us);
 }
 // 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on `bar`.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, u32 bytes, u64* bar) {

@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(THREADS) k_server_dense(Plan P, ServerArgs A) 
   const int tid = threadIdx.x;
   const bool emit = (COMP == 2) && A.emit_srv;
   const bool sign_dc = (COMP == 1) && A.emit_srv;        // scaled sign, double-way: the server's L1 partials and words
-  const u32 lo = emit ? window_lo(A.tau_srv_prev[ti.j]) : NO_GUESS;
+  const u32 lo = emit ? window_lo(A.tau_srv_prev[ti.j], A.cand_srv.wlog2[ti.j]) : NO_GUESS;
   WarpStage stg; stg.buf = cstage + ((COMP == 2) ? (tid >> 5) * CAND_STAGE : 0); stg.n = 0;
   LaneAcc acc; lane_acc_init(acc);
   if (COMP != 0 && !SUM) {                               // (SUM: no rows are read, so no worker thresholds either)

@@ -158,7 +158,7 @@ __global__ void __launch_bounds__(THREADS) k_server_candidates(Plan P, const flo
   __shared__ u32 cstage[(THREADS / 32) * CAND_STAGE];
   const TileInfo ti = tile_info(P, blockIdx.x);
   const int tid = threadIdx.x;
-  const u32 lo = window_lo(tau_srv_prev[ti.j]);
+  const u32 lo = window_lo(tau_srv_prev[ti.j], C.wlog2[ti.j]);
   if (lo == NO_GUESS) return;
   WarpStage stg; stg.buf = cstage + (tid >> 5) * CAND_STAGE; stg.n = 0;
   const float* __restrict__ dp = delta + ti.poff + ti.t0;

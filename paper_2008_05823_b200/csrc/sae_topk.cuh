@@ -33,21 +33,29 @@ struct CandArgs {
   long long stride;      // keys per row
   u32* count;            // [rows][T] append cursors (may run past cap: that is the overflow signal)
   int T;
+  const int* wlog2;      // [T] log2 of the window's width in key units below last step's threshold; WINDOW_ALL:
+                         // the tensor's region holds all of it, every non-zero key is a candidate
 };
+
+constexpr int WINDOW_ALL = 32;
 
 constexpr u32 NO_GUESS = 0xffffffffu;
 constexpr int CAND_STAGE = 256;   // keys a warp stages in shared memory before one append to global memory
 
-// Lower edge of the window for a previous threshold key: 2^SAE_TOPK_WINDOW_LOG2 key units below it, i.e.
-// 2^(SAE_TOPK_WINDOW_LOG2 - 23) octaves (the default 18 is about 2 %).  With error feedback the entries
-// that were not sent keep growing until they cross the threshold, so the density just below it is high
-// (of the order of n / threshold): a wide window would overflow the candidate list.
+// Lower edge of the window for a previous threshold key: 2^wlog2 key units below it, i.e. 2^(wlog2 - 23) octaves
+// (SAE_TOPK_WINDOW_LOG2 = 18, about 2 %, for the large tensors).  With error feedback the entries that were not
+// sent keep growing until they cross the threshold, so the density just below it is high (of the order of
+// n / threshold): a wide window would overflow the candidate list of a large tensor.  A small tensor's threshold
+// -- the k-th largest of few values, k = 1 .. a few hundred -- moves by far more than 2 % from step to step, and
+// its region has room to spare (8 k + 1024 keys): its window is up to 8 times wider, and a tensor that fits its
+// region whole collects every non-zero key, with or without a guess.
 #ifndef SAE_TOPK_WINDOW_LOG2
 #define SAE_TOPK_WINDOW_LOG2 18
 #endif
-__device__ __forceinline__ u32 window_lo(u32 tau_prev) {
+__device__ __forceinline__ u32 window_lo(u32 tau_prev, int wlog2) {
+  if (wlog2 >= WINDOW_ALL) return 1u;
   if (tau_prev == 0u) return NO_GUESS;                 // no usable guess (first step, or an all-zero tail)
-  return tau_prev > (1u << SAE_TOPK_WINDOW_LOG2) ? tau_prev - (1u << SAE_TOPK_WINDOW_LOG2) : 1u;
+  return tau_prev > (1u << wlog2) ? tau_prev - (1u << wlog2) : 1u;
 }
 
 // Per-warp staging of candidate keys in shared memory; `n` is warp-uniform.
@@ -114,10 +122,11 @@ constexpr int HIST_BINS = 2048;
 // Walks a histogram of `bins` (1024 or 2048) counters from the top: returns in *bin the bin that holds the
 // rank-th entry and in *rank_in the rank inside it.  Block-wide; hist may be shared or global memory;
 // the counters are cleared.  part/above: THREADS words of shared memory each.
+template <int NT = THREADS>
 __device__ __forceinline__ void walk_from_top(u32* hist, int bins, u32 rank, u32* part, u32* above, u32* out_bin,
                                               u32* out_rank) {
   const int tid = threadIdx.x;
-  const int per = bins / THREADS;         // 8 or 4
+  const int per = bins / NT;              // 8 or 4 (256 threads), 2 or 1 (1024 threads)
   u32 c[8];
   u32 sum = 0;
   for (int q = 0; q < per; ++q) {
@@ -139,7 +148,7 @@ __device__ __forceinline__ void walk_from_top(u32* hist, int bins, u32 rank, u32
   __syncthreads();
   if (tid == 0) {
     u32 run = 0;
-    for (int t = 0; t < THREADS / 32; ++t) { above[t] = run; run += part[t]; }
+    for (int t = 0; t < NT / 32; ++t) { above[t] = run; run += part[t]; }
   }
   __syncthreads();
   u32 run = above[wrp] + inc - sum;
@@ -160,26 +169,10 @@ __device__ __forceinline__ void walk_from_top(u32* hist, int bins, u32 rank, u32
 //   y <  0: data item x = tile * rows + row of a pair whose window failed (keys come from the values);
 //   y >= 0: chunk y (CAND_CHUNK keys) of the candidate list of pair x = row * T + j.
 constexpr int CAND_CHUNK = 4096;
-
-// One thread per (row, tensor): decides whether the candidate window holds the threshold, queues the
-// candidate chunks if so, raises the fallback flag otherwise, and resets the cursor.
-__global__ void __launch_bounds__(THREADS) k_topk_decide(CandArgs C, int rows, const int* __restrict__ n, u32 num, u32 den,
-                                                          const u32* __restrict__ tau_guess, u32* cand_n, u32* fallback,
-                                                          u32* fallback_total, int2* work, u32* work_count) {
-  const int rj = blockIdx.x * THREADS + threadIdx.x;
-  if (rj >= rows * C.T) return;
-  const int j = rj % C.T;
-  const u32 cnt = C.count[rj];
-  const u32 kk = topk_count_of(n[j], num, den);
-  const bool ok = window_lo(tau_guess[rj]) != NO_GUESS && cnt <= (u32)C.cap[j] && cnt >= kk;
-  C.count[rj] = 0u;
-  cand_n[rj] = ok ? cnt : 0u;
-  fallback[rj] = ok ? 0u : 1u;
-  if (!ok) { atomicAdd(fallback_total, 1u); return; }
-  const u32 chunks = (cnt + CAND_CHUNK - 1) / CAND_CHUNK;
-  const u32 base = atomicAdd(work_count, chunks);
-  for (u32 c = 0; c < chunks; ++c) work[base + c] = make_int2(rj, (int)c);
-}
+// what the one-launch select left to the distributed select for a pair (its `fallback` word)
+constexpr u32 FB_NONE = 0u;       // settled
+constexpr u32 FB_VALUES = 1u;     // the window failed on a large tensor: radix select over its values
+constexpr u32 FB_LIST = 2u;       // a long candidate list that holds the threshold: radix select over its chunks
 
 // Queues every (tile, row) data item whose (row, tensor) raised the fallback flag.
 __global__ void __launch_bounds__(THREADS) k_topk_worklist(Plan P, int rows, const u32* __restrict__ fallback, int2* work,
@@ -189,7 +182,7 @@ __global__ void __launch_bounds__(THREADS) k_topk_worklist(Plan P, int rows, con
   if (mine >= nitems) return;
   const int tile = (int)(mine / rows);
   const int k = (int)(mine - (long long)tile * rows);
-  if (fallback[(long long)k * P.T + P.tile_tensor[tile]]) work[atomicAdd(work_count, 1u)] = make_int2((int)mine, -1);
+  if (fallback[(long long)k * P.T + P.tile_tensor[tile]] == FB_VALUES) work[atomicAdd(work_count, 1u)] = make_int2((int)mine, -1);
 }
 
 // The rows whose Top-K thresholds are wanted: stored ([rows][dpad] in buf), or -- when the worker pass did
@@ -202,10 +195,29 @@ struct DeltaSrc {
   int recompute;
 };
 
-__device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* hist) {
-  if (level == 0) atomicAdd(hist + (key >> 20), 1u);
-  else if (level == 1) { if ((key >> 20) == prefix) atomicAdd(hist + ((key >> 10) & 1023u), 1u); }
-  else { if ((key >> 10) == prefix) atomicAdd(hist + (key & 1023u), 1u); }
+// ++hist[bin] for the lanes with `take` set, one atomic per distinct bin of the warp: the keys of a tensor share
+// their leading digits, so plain per-lane atomics would pile up on a few addresses.  Whole warps only.
+__device__ __forceinline__ void hist_add_aggregated(u32* hist, u32 bin, bool take) {
+  if (!__any_sync(0xffffffffu, take)) return;
+  const u32 peers = __match_any_sync(0xffffffffu, take ? bin : 0xffffffffu);
+  if (take && (threadIdx.x & 31) == (u32)(__ffs(peers) - 1)) atomicAdd(hist + bin, (u32)__popc(peers));
+}
+
+// digit of `key` at a level of the 11 + 10 + 10 radix select, and whether the key lies in the prefix bucket
+__device__ __forceinline__ bool radix_digit(u32 key, int level, u32 prefix, u32* digit) {
+  if (level == 0) { *digit = key >> 20; return true; }
+  if (level == 1) { *digit = (key >> 10) & 1023u; return (key >> 20) == prefix; }
+  *digit = key & 1023u;
+  return (key >> 10) == prefix;
+}
+
+// one key per lane into the level's histogram (`valid` masks lanes past the end).  Plain shared-memory atomics:
+// in the distributed select, where a block handles 4096 keys at a time, aggregating equal digits across the
+// warp first costs more than the pile-up it avoids (measured: histogram launches 18 -> 30 us).
+__device__ __forceinline__ void hist_elem(u32 key, int level, u32 prefix, u32* hist, bool valid = true) {
+  u32 digit;
+  const bool in = radix_digit(key, level, prefix, &digit);
+  if (valid && in) atomicAdd(hist + digit, 1u);
 }
 
 // Level L histogram over the work list (a fixed grid of blocks strides over it).  Every item accumulates
@@ -249,8 +261,11 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
           hist_elem(mag_key(v.w), level, prefix, target);
         }
       } else {
-        for (int i = tid; i < ti.cnt; i += THREADS)
-          hist_elem(mag_key(src.recompute ? __fmaf_rn(src.eta, bp[i], eb[i]) : bp[i]), level, prefix, target);
+        for (int i = tid; i - tid < ti.cnt; i += THREADS) {
+          const bool valid = i < ti.cnt;
+          const float v = valid ? (src.recompute ? __fmaf_rn(src.eta, bp[i], eb[i]) : bp[i]) : 0.0f;
+          hist_elem(mag_key(v), level, prefix, target, valid);
+        }
       }
     } else {
       rj = w.x;
@@ -259,7 +274,7 @@ __global__ void __launch_bounds__(THREADS) k_topk_hist(Plan P, CandArgs C, int r
       const int cnt = min((int)(cand_n[rj] - (u32)w.y * CAND_CHUNK), CAND_CHUNK);
       const u32 prefix = level ? st[rj].prefix : 0u;
       u32* target = sh;
-      for (int i = tid; i < cnt; i += THREADS) hist_elem(keys[i], level, prefix, target);
+      for (int i = tid; i - tid < cnt; i += THREADS) hist_elem(i < cnt ? keys[i] : 0u, level, prefix, target, i < cnt);
     }
     __syncthreads();
     u32* gh = hist + (long long)rj * HIST_BINS;
@@ -296,7 +311,8 @@ __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const
 }
 
 // ---------------------------------------------------------------------------------------------------
-// The whole select of one (row, tensor) in one block.
+// The whole select of one (row, tensor) in one block -- except for the tensors with long candidate regions when
+// the distributed select follows anyway: their lists are queued for it chunk by chunk.
 //
 // Window path (the list did not overflow and holds at least k keys, so the k-th largest key of the tensor is
 // the k-th largest key of the list): every key of the list is >= lo.  Pass 1 bins rel = key - lo in steps of
@@ -309,77 +325,162 @@ __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const
 // Failed window: tensors of at most inline_max elements are settled here by the three-level radix select
 // (11 + 10 + 10 bits) over their values, read by this block alone; larger ones raise their fallback flag for
 // the distributed select that follows.
-constexpr int WIN_SHIFT = 8;
 constexpr int WIN_BINS = 2048;            // covers 2^19 key units above lo: twice the window below the old threshold
+constexpr int SEL_U = 4;                  // loads a thread keeps in flight while it walks a list or a tensor
+constexpr int SEL_LONG_REGION = 16384;    // candidate regions above this many keys count as long (see topk_thresholds)
+#ifndef SAE_TOPK_INLINE_MAX
+#define SAE_TOPK_INLINE_MAX 2048
+#endif
 
-__global__ void __launch_bounds__(THREADS) k_topk_select_window(Plan P, CandArgs C, int rows, u32 num, u32 den,
-                                                                 DeltaSrc src, const u32* tau_guess, u32* tau_out,
-                                                                 u32* fallback, u32* fallback_total, int inline_max) {
+// Calls f(key, valid) for every key of a candidate list, the whole block in step (every thread makes the same
+// number of calls, so f may use warp-collective operations).  The list is read with 16-byte loads, SEL_U of them
+// in flight per thread: a block walks its list alone, and what bounds it is the number of round trips to L2.
+template <int NT, class F>
+__device__ __forceinline__ void for_each_key(const u32* __restrict__ keys, u32 cnt, F f) {
+  const uint4* __restrict__ k4 = reinterpret_cast<const uint4*>(keys);    // (regions start on 16-byte boundaries)
+  const u32 n4 = (cnt + 3u) >> 2;
+  for (u32 b = 0; b < n4; b += NT * SEL_U) {
+    uint4 q[SEL_U];
+#pragma unroll
+    for (int u = 0; u < SEL_U; ++u) {
+      const u32 idx = b + u * NT + threadIdx.x;
+      q[u] = idx < n4 ? k4[idx] : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < SEL_U; ++u) {
+      const u32 i = (b + u * NT + threadIdx.x) * 4u;
+      f(q[u].x, i < cnt); f(q[u].y, i + 1u < cnt); f(q[u].z, i + 2u < cnt); f(q[u].w, i + 3u < cnt);
+    }
+  }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(NT) k_topk_select_window(Plan P, CandArgs C, const int* __restrict__ jlist, int nj,
+                                                            u32 num, u32 den, DeltaSrc src, const u32* tau_guess,
+                                                            u32* tau_out, u32* fallback, u32* fallback_total,
+                                                            int inline_max, int chain_min_cap, u32* cand_n, int2* work,
+                                                            u32* work_count) {
   __shared__ u32 sh[HIST_BINS];
-  __shared__ u32 part[THREADS];
-  __shared__ u32 above[THREADS];
+  __shared__ u32 part[NT / 32];
+  __shared__ u32 above[NT / 32];
   __shared__ u32 sh_bin, sh_rank, sh_above;
   const int tid = threadIdx.x;
-  const int rj = blockIdx.x;              // row * T + j
-  const int row = rj / C.T, j = rj - row * C.T;
+  const int row = blockIdx.x / nj, j = jlist[blockIdx.x - row * nj];     // this launch's tensors: jlist[0 .. nj)
+  const int rj = row * C.T + j;
   const int n = P.n[j];
   const u32 kk = topk_count_of(n, num, den);
   const u32 cnt = C.count[rj];
-  const u32 lo = window_lo(tau_guess[rj]);
-  bool ok = lo != NO_GUESS && cnt <= (u32)C.cap[j] && cnt >= kk;
-  for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
+  const int wl = C.wlog2[j];
+  const bool all = wl >= WINDOW_ALL;      // the list holds every non-zero key of the tensor
+  const int shift = all ? 0 : wl - 10;    // bin width of pass 1: 1024 bins span the window below the old threshold
+  const u32 lo = window_lo(tau_guess[rj], wl);
+  const bool ok = lo != NO_GUESS && cnt <= (u32)C.cap[j] && cnt >= kk;
+  for (int b = tid; b < HIST_BINS; b += NT) sh[b] = 0u;
   if (tid == 0) sh_above = 0u;
   __syncthreads();
   if (tid == 0) C.count[rj] = 0u;         // (every thread has read the cursor: the barrier above)
+  if (ok && C.cap[j] > chain_min_cap) {
+    // A long list: one block would be bound by its shared-memory atomics (tens of microseconds for 10^5 keys).
+    // Its chunks go to the work list of the distributed select, which spreads them over the device.
+    if (tid == 0) {
+      cand_n[rj] = cnt;
+      fallback[rj] = FB_LIST;
+      const u32 chunks = (cnt + CAND_CHUNK - 1) / CAND_CHUNK;
+      const u32 base = atomicAdd(work_count, chunks);
+      for (u32 c = 0; c < chunks; ++c) work[base + c] = make_int2(rj, (int)c);
+    }
+    return;
+  }
   if (ok) {
     const u32* __restrict__ keys = C.keys + (long long)row * C.stride + C.off[j];
+    const u32 RANGE = all ? 0u : ((u32)WIN_BINS << shift);
     u32 mine = 0;
-    for (u32 i = tid; i < cnt; i += THREADS) {
-      const u32 rel = keys[i] - lo;
-      if (rel >= ((u32)WIN_BINS << WIN_SHIFT)) ++mine;
-      else atomicAdd(sh + (rel >> WIN_SHIFT), 1u);
-    }
+    if (!all)
+      for_each_key<NT>(keys, cnt, [&](u32 key, bool valid) {
+        const u32 rel = key - lo;
+        if (valid) {
+          if (rel >= RANGE) ++mine;
+          else atomicAdd(sh + (rel >> shift), 1u);
+        }
+      });
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
     if ((tid & 31) == 0 && mine) atomicAdd(&sh_above, mine);
     __syncthreads();
-    const u32 over = sh_above;
-    if (kk <= over) {
-      ok = false;                         // (uniform: every thread reads the same count)
-      __syncthreads();
-      for (int b = tid; b < HIST_BINS; b += THREADS) sh[b] = 0u;
-      __syncthreads();
-    } else {
-      walk_from_top(sh, WIN_BINS, kk - over, part, above, &sh_bin, &sh_rank);     // (clears the bins)
+    const u32 over = all ? cnt : sh_above;   // (uniform: every thread reads the same count)
+    if (kk > over) {
+      walk_from_top<NT>(sh, WIN_BINS, kk - over, part, above, &sh_bin, &sh_rank);     // (clears the bins)
       const u32 bin = sh_bin, rank = sh_rank;
-      for (u32 i = tid; i < cnt; i += THREADS) {
-        const u32 rel = keys[i] - lo;
-        if ((rel >> WIN_SHIFT) == bin) atomicAdd(sh + (rel & ((1u << WIN_SHIFT) - 1u)), 1u);
-      }
+      for_each_key<NT>(keys, cnt, [&](u32 key, bool valid) {
+        const u32 rel = key - lo;
+        if (valid && (rel >> shift) == bin) atomicAdd(sh + (rel & ((1u << shift) - 1u)), 1u);
+      });
       __syncthreads();
-      walk_from_top(sh, 1024, rank, part, above, &sh_bin, &sh_rank);
+      walk_from_top<NT>(sh, shift > 10 ? HIST_BINS : 1024, rank, part, above, &sh_bin, &sh_rank);
       if (tid == 0) {
-        tau_out[rj] = lo + (bin << WIN_SHIFT) + sh_bin;
-        fallback[rj] = 0u;
+        tau_out[rj] = lo + (bin << shift) + sh_bin;
+        fallback[rj] = FB_NONE;
       }
       return;
     }
+    // The threshold rose past the binned range: it is the kk-th largest of the list's keys above the range
+    // (a heavy tail spread over many octaves).  Three radix levels over those keys, still from the list.
+    __syncthreads();
+    for (int b = tid; b < HIST_BINS; b += NT) sh[b] = 0u;
+    __syncthreads();
+    u32 prefix = 0u, rank = kk;
+    for (int level = 0; level < 3; ++level) {
+      for_each_key<NT>(keys, cnt, [&](u32 key, bool valid) {
+        u32 digit;
+        const bool in = radix_digit(key, level, prefix, &digit);
+        hist_add_aggregated(sh, digit, valid && key - lo >= RANGE && in);
+      });
+      __syncthreads();
+      walk_from_top<NT>(sh, level == 0 ? HIST_BINS : 1024, rank, part, above, &sh_bin, &sh_rank);
+      prefix = (level == 0) ? sh_bin : ((prefix << 10) | sh_bin);
+      rank = sh_rank;
+      __syncthreads();                    // (sh_bin / sh_rank are rewritten by the next level)
+    }
+    if (tid == 0) { tau_out[rj] = prefix; fallback[rj] = FB_NONE; }
+    return;
   }
   // ---- the window failed ----
   if (tid == 0) atomicAdd(fallback_total, 1u);
   if (n > inline_max) {
-    if (tid == 0) fallback[rj] = 1u;      // a large tensor: left to the distributed select
+    if (tid == 0) fallback[rj] = FB_VALUES;   // a large tensor: left to the distributed select
     return;
   }
-  if (tid == 0) fallback[rj] = 0u;
+  if (tid == 0) fallback[rj] = FB_NONE;
   const float* __restrict__ bp = (src.recompute ? src.m : src.buf) + (long long)row * P.dpad + P.poff[j];
   const float* __restrict__ eb = src.ebar + P.poff[j];               // read only when recomputing
   u32 prefix = 0u, rank = kk;
   for (int level = 0; level < 3; ++level) {
-    for (int i = tid; i < n; i += THREADS)
-      hist_elem(mag_key(src.recompute ? __fmaf_rn(src.eta, bp[i], eb[i]) : bp[i]), level, prefix, sh);
+    // (tensors start on 128-byte boundaries in the padded layout and their padding is zero: 16-byte loads may run
+    // up to three elements past n, and those are masked)
+    const int n4 = (n + 3) >> 2;
+    for (int b0 = 0; b0 < n4; b0 += NT * SEL_U) {
+      float4 vq[SEL_U], eq[SEL_U];
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) {
+        const int idx = b0 + u * NT + tid;
+        vq[u] = idx < n4 ? ld4(bp + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+        eq[u] = (src.recompute && idx < n4) ? ld4(eb + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) {
+        const int i = 4 * (b0 + u * NT + tid);
+        const float v[4] = {vq[u].x, vq[u].y, vq[u].z, vq[u].w}, e[4] = {eq[u].x, eq[u].y, eq[u].z, eq[u].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const u32 key = mag_key(src.recompute ? __fmaf_rn(src.eta, v[c], e[c]) : v[c]);
+          u32 digit;
+          const bool in = radix_digit(key, level, prefix, &digit);
+          hist_add_aggregated(sh, digit, i + c < n && in);
+        }
+      }
+    }
     __syncthreads();
-    walk_from_top(sh, level == 0 ? HIST_BINS : 1024, rank, part, above, &sh_bin, &sh_rank);
+    walk_from_top<NT>(sh, level == 0 ? HIST_BINS : 1024, rank, part, above, &sh_bin, &sh_rank);
     prefix = (level == 0) ? sh_bin : ((prefix << 10) | sh_bin);
     rank = sh_rank;
     __syncthreads();                      // (sh_bin / sh_rank are rewritten by the next level)

@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(FW_THREADS, 1) k_worker_fused(Plan P, StepPara
         }
         acc_j = it.j;
       }
-      const u32 lo = TOPK ? window_lo(__float_as_uint(S.sc[s][kl0])) : NO_GUESS;
+      const u32 lo = TOPK ? window_lo(__float_as_uint(S.sc[s][kl0]), A.cand.wlog2[it.j]) : NO_GUESS;
       const float* sm = S.m[s];
       const float* sg = S.g[s];
       const float* se = S.e[s];

@@ -76,7 +76,7 @@ __device__ __forceinline__ WtItem wt_lookup(const Plan& P, const WorkerArgs& A, 
   it.k = k; it.j = ti.j; it.cnt = ti.cnt; it.tiles_j = ti.tiles_j; it.n = ti.n;
   if (ESRC == ESRC_LAZY_SIGN) it.sprev = A.scale_prev[(long long)k * P.T + ti.j];
   if (ESRC == ESRC_LAZY_TOPK || TOPK) it.tprev = A.tau_prev[(long long)k * P.T + ti.j];
-  if (TOPK) it.lo = window_lo(it.tprev);
+  if (TOPK) it.lo = window_lo(it.tprev, A.cand.wlog2[ti.j]);
   it.vec = (ti.cnt == TILE) && ((reinterpret_cast<uintptr_t>(A.g + it.gofs) & 15) == 0);
   return it;
 }

@@ -113,8 +113,10 @@ def test_topk_candidate_window_is_used_and_exact():
         compare_state(gpu, orc, so.TOPK, tag=f"window t={t + 1}")
         compare_server_messages(gpu, orc, so.TOPK, 1, tag=f"window t={t + 1}")
     fb = gpu.get_state(sb.STATE_TOPK_FALLBACKS).cpu().numpy()
-    assert K * len(sizes) <= fb[0] < K * len(sizes) * steps // 2, fb      # the first step always falls back
-    assert len(sizes) <= fb[1] < len(sizes) * steps // 2, fb
+    # the first step has no previous threshold to look around: every pair misses, except for tensors small enough
+    # that their candidate region holds them whole (here the 700-element one), which never need a guess
+    assert K * (len(sizes) - 1) <= fb[0] < K * len(sizes) * steps // 2, fb
+    assert len(sizes) - 1 <= fb[1] < len(sizes) * steps // 2, fb
 
 
 def test_topk_ties_and_zeros():
