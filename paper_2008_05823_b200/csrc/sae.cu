@@ -219,10 +219,16 @@ int check_launch(sae_handle* h) {
   return SAE_OK;
 }
 
+// SAE_DEBUG_FAIL_ALLOC=<n> (testing only, read by sae_init): the n-th device allocation of that sae_init
+// (0-based) reports cudaErrorMemoryAllocation without calling cudaMalloc, so that the clean-up path of a failed
+// initialisation can be exercised without exhausting a shared GPU's memory.
+thread_local long g_fail_alloc_at = -1, g_alloc_index = 0;
+
 template <class T>
 cudaError_t dalloc(T** p, size_t count) {
   *p = nullptr;
   if (count == 0) count = 1;
+  if (g_fail_alloc_at >= 0 && g_alloc_index++ == g_fail_alloc_at) return cudaErrorMemoryAllocation;
   return cudaMalloc((void**)p, count * sizeof(T));
 }
 
@@ -270,24 +276,32 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   // would take too long over it.)
   const bool distributed = fb != h->fb_srv || h->max_n > (1ll << 20);
   const int inline_max = distributed ? SAE_TOPK_INLINE_MAX : 0x7fffffff;
-  // Tensors with long candidate regions (the first n_sel_long of the list).  With p = 1 the lists stay short of
-  // their regions and one block of 1024 threads settles each (config 3: 0.619 -> 0.599 ms per step); without the
-  // per-step averaging the unsent entries pile up below the threshold, the lists are several times longer and
-  // a single block is bound by its shared-memory atomics: their chunks go to the distributed select instead,
-  // which spreads them over the device (config 3, p = 20: 0.927 -> 0.896 ms).
-  const bool long_inline = h->topk_nod || !distributed;
+  // Tensors with long candidate regions (the first n_sel_long of the list, longest first).  A single block
+  // that walks a list of 10^5 keys is bound by its shared-memory atomics (60-120 us), the distributed select
+  // spreads the same keys over the device but costs three levels of launches with real work in them.  What
+  // pays, measured on config 3 (ms per step, p = 1 / p = 20; the select chains of the previous form 0.637 / 0.898):
+  //   * the server's one row: its lists are short of their regions (its Delta is the mean of sparse messages);
+  //     a block of 1024 threads per long list settles all of them in 12 us;
+  //   * the workers with p = 1 (the lists stay short of their regions): blocks of 1024 threads, 0.599 / -- (the
+  //     longest regions' chunks to the distributed select instead: 0.614);
+  //   * the workers with stored differences (no averaging every step: the unsent entries pile up below the
+  //     threshold and the lists are several times longer): every long list's chunks go to the distributed select,
+  //     -- / 0.890 (blocks of 1024 threads: 0.927).
+  const bool server_row = fb == h->fb_srv;
+  const bool long_inline = server_row || h->topk_nod || !distributed;
   const int n_long = long_inline ? h->n_sel_long : 0;
+  const int chunk_above = long_inline ? 0x7fffffff : SEL_LONG_REGION;
   if (n_long > 0) {
     LaunchScope ls(h, S_TOPK_SELECT);
     k_topk_select_window<1024><<<(unsigned)(rows * n_long), 1024, 0, h->stream>>>(
         P, cand, h->d_sel_list, n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb, fb_total,
-        inline_max, 0x7fffffff, cand_n, work, work_count);
+        inline_max, chunk_above, cand_n, work, work_count);
   }
   if (P.T > n_long) {
     LaunchScope ls(h, S_TOPK_SELECT);
     k_topk_select_window<THREADS><<<(unsigned)(rows * (P.T - n_long)), THREADS, 0, h->stream>>>(
         P, cand, h->d_sel_list + n_long, P.T - n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb,
-        fb_total, inline_max, long_inline ? 0x7fffffff : SEL_LONG_REGION, cand_n, work, work_count);
+        fb_total, inline_max, chunk_above, cand_n, work, work_count);
   }
   if (!distributed) return;
   const long long items = (long long)P.ntiles * rows;
@@ -994,6 +1008,9 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
 
   DeviceGuard guard(cfg->device);
   if (!guard.ok) { g_init_cuda_error = (int)cudaGetLastError(); return SAE_ERR_CUDA; }
+  g_fail_alloc_at = -1; g_alloc_index = 0;
+  if (const char* ev = getenv("SAE_DEBUG_FAIL_ALLOC")) { const long v = atol(ev); if (v >= 0) g_fail_alloc_at = v; }
+  struct FailAllocOff { ~FailAllocOff() { g_fail_alloc_at = -1; } } fail_alloc_off;   // only this sae_init
 
   sae_handle* h = new (std::nothrow) sae_handle();
   if (!h) return SAE_ERR_NOMEM;

@@ -25,7 +25,10 @@
 namespace sae {
 
 constexpr int FW_WARPS = 16;                       // worker warps (warps 0..15)
-constexpr int FW_AVG_WARPS = 4;                    // averager warps (warps 17..20); warp 16 is the producer
+#ifndef SAE_FW_AVG_WARPS
+#define SAE_FW_AVG_WARPS 4
+#endif
+constexpr int FW_AVG_WARPS = SAE_FW_AVG_WARPS;     // averager warps (warps 17..); warp 16 is the producer
 constexpr int FW_THREADS = (FW_WARPS + 1 + FW_AVG_WARPS) * 32;
 constexpr int FW_MAXTILE = 2048;
 constexpr int FW_MAXBOX = 256;                     // inner extent of a TMA box (the hardware limit)
