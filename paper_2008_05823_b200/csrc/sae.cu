@@ -8,6 +8,7 @@
 
 #include <cuda.h>
 #include <cudaTypedefs.h>
+#include <nvtx3/nvToolsExt.h>      // header-only: ranges cost nothing unless a profiler has injected itself
 #include <algorithm>
 #include <cstdio>
 #include <cstdlib>
@@ -184,15 +185,24 @@ cudaEvent_t take_event(sae_handle* h) {
   return e;
 }
 
+// One per kernel launch: counts it, brackets it with events while per-kernel timing is on, and opens an NVTX
+// range named after the kernel's role ("worker_pass", "server_aggregate", ...) for timeline tools.
 struct LaunchScope {
   sae_handle* h; int slot; cudaEvent_t a, b;
   LaunchScope(sae_handle* h_, int slot_) : h(h_), slot(slot_), a(nullptr), b(nullptr) {
+    nvtxRangePushA(kSlotNames[slot]);
     if (h->profiling) { a = take_event(h); b = take_event(h); cudaEventRecord(a, h->stream); }
   }
   ~LaunchScope() {
     h->launches++;
     if (h->profiling) { cudaEventRecord(b, h->stream); h->pending.push_back({slot, a, b}); }
+    nvtxRangePop();
   }
+};
+
+struct ApiRange {       // an NVTX range around a whole entry point
+  explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+  ~ApiRange() { nvtxRangePop(); }
 };
 
 #define LAUNCH(h, slot, kern, grid, ...)                                   \
@@ -1467,6 +1477,7 @@ int sae_avg_set(sae_handle* h, const float* sum_padded) {
 }
 
 int sae_step_begin(sae_handle* h, const float* grads_local, float lr) {
+  ApiRange nvtx_range("sae_step_begin");
   if (!h || !grads_local || !(lr > 0.0f) || !(lr < 3.0e38f)) return SAE_ERR_INVALID_ARG;
   if (!h->shard || h->mid_step || h->avg_owed || h->attached != h->K_total) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
@@ -1475,6 +1486,7 @@ int sae_step_begin(sae_handle* h, const float* grads_local, float lr) {
 }
 
 int sae_step_end(sae_handle* h) {
+  ApiRange nvtx_range("sae_step_end");
   if (!h || !h->shard || !h->mid_step) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
@@ -1482,6 +1494,7 @@ int sae_step_end(sae_handle* h) {
 }
 
 int sae_step(sae_handle* h, const float* grads, float lr) {
+  ApiRange nvtx_range("sae_step");
   if (!h || !grads || !(lr > 0.0f) || !(lr < 3.0e38f) || h->shard) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
@@ -1489,6 +1502,7 @@ int sae_step(sae_handle* h, const float* grads, float lr) {
 }
 
 int sae_step_host(sae_handle* h, const float* grads_host, float lr) {
+  ApiRange nvtx_range("sae_step_host");
   if (!h || !grads_host || !(lr > 0.0f) || !(lr < 3.0e38f) || h->shard) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
@@ -1499,6 +1513,7 @@ int sae_step_host(sae_handle* h, const float* grads_host, float lr) {
 }
 
 int sae_get_params(sae_handle* h, float* out) {
+  ApiRange nvtx_range("sae_get_params");
   if (!h || !out) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
@@ -1520,6 +1535,7 @@ int sae_get_params_host(sae_handle* h, float* out_host) {
 }
 
 int sae_get_step_ahead(sae_handle* h, int32_t worker, float* out) {
+  ApiRange nvtx_range("sae_get_step_ahead");
   if (!h || !out || worker < 0 || worker >= h->P.K) return SAE_ERR_INVALID_ARG;
   DeviceGuard guard(h->device);
   if (!guard.ok) return SAE_ERR_CUDA;
