@@ -216,7 +216,7 @@ def cpu_baseline(w, avg_period, seed, steps, warmup, wall_budget_s=200.0, sample
     single = {"value": n1 / dt1 * frac, "unit": "steps/s", "cores": 1, "steps": n1, "seconds": dt1,
               "sample": "the same sample of whole tensors on one thread, scaled by the sampled fraction"}
     del orc1
-    est_full_step = 2.0 * (dt_s / n_s) / frac          # (x2: the sample under-estimates, its small tensors sit in cache)
+    est_full_step = 1.25 * (dt_s / n_s) / frac         # (a margin: the sample's small tensors sit in cache)
     # ---- full size, if memory and time allow
     sets = 1 if 4 * K * d > (4 << 30) else 2
     need = 4 * (4 * K * d + sets * K * d + 8 * d)       # oracle state m, e, Delta, C(Delta) + gradient sets
