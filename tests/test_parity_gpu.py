@@ -605,3 +605,39 @@ def test_step_ahead_point_read_after_every_step(K, comp, dc, mode):
         compare_state(gpu, orc, comp, tag="read every step, end")
         compare_server_messages(gpu, orc, comp, dc, tag="read every step, end")
         gpu.close()
+
+
+@pytest.mark.parametrize("K,p", [(8, 1), (8, 0), (2, 3), (16, 1)])
+def test_topk_thresholds_that_jump(K, p):
+    """Learning rates that jump by factors of 4 and 20: the thresholds leave their candidate windows in both
+    directions -- upwards past the range the one-launch select bins finely (found among the list's keys above
+    it), downwards out of the list altogether (the window fails: small tensors settled inside the block, large
+    ones by the distributed select).  Tensors of every class: one that fits its candidate region whole, small and
+    medium ones, and two whose regions are long enough for the wide blocks / the chunked lists.  Thresholds,
+    selection masks and state against the oracle after every step."""
+    import torch
+    sizes = [700, 33, 5000, 40_000, 2_100_000 // K + 4096 * 3 + 5, 2_600_000 // K]
+    d = int(np.sum(sizes))
+    scales = synth.tensor_scales(31, len(sizes), -3.0, -2.0)
+    x0 = synth.x0_numpy(31, d)
+    kw = dict(compressor=so.TOPK, avg_period=p, momentum=0.9, topk_num=1, topk_den=10)
+    orc = so.Oracle(K, sizes, x0, threads=8, **kw)
+    gpu = sb.Sae(K, sizes, torch.from_numpy(x0).cuda(), **kw)
+    lrs = [0.1] * 4 + [0.4] * 2 + [0.02] * 3 + [0.1] * 2 + [2.0, 0.001, 0.1]
+    for t, lr in enumerate(lrs):
+        g = synth.grads_numpy(31, t, K, sizes, scales, 66, 100.0)
+        orc.step(g, lr)
+        gpu.step(torch.from_numpy(g).cuda(), lr)
+        tag = f"jump K={K} p={p} t={t + 1} lr={lr}"
+        gpu.sync()
+        for k in (0, K - 1):
+            assert_same(f"{tag} tau[{k}]", gpu.get_state(sb.STATE_WORKER_TAU, k).cpu().numpy().view(np.uint32).astype(np.uint64),
+                        orc.tau(k))
+        assert_same(f"{tag} tau_srv", gpu.get_state(sb.STATE_SERVER_TAU).cpu().numpy().view(np.uint32).astype(np.uint64),
+                    orc.tau(-1))
+        if t % 3 == 2 or t == len(lrs) - 1:
+            compare_state(gpu, orc, so.TOPK, tag=tag)
+            compare_server_messages(gpu, orc, so.TOPK, 1, tag=tag)
+    fb = gpu.get_state(sb.STATE_TOPK_FALLBACKS).cpu().numpy()
+    assert fb[0] > K * (len(sizes) - 1)          # windows did fail after the first step as well
+    gpu.close()
