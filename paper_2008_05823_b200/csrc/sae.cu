@@ -1116,7 +1116,8 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
       cand_off[j] = h->cand_stride; cand_cap[j] = (int)cap;
       // window width: the whole tensor where the region holds it; else 2 % of the old threshold, up to 8 times
       // wider for small k (whose threshold moves more from step to step and whose region has room to spare)
-      if (cap >= (unsigned long long)h->sizes[j]) wlog2[j] = WINDOW_ALL;
+      if (cap >= (unsigned long long)h->sizes[j] && h->sizes[j] <= 16384) wlog2[j] = WINDOW_ALL;   // (small tensors only:
+                                        // with a large Top-K ratio every region holds its tensor, and listing all of K x d would not pay)
       else for (unsigned long long w = 2; w <= 8 && w * kk <= 1024; w *= 2) wlog2[j] += 1;
       h->cand_stride += (long long)((cap + 3) / 4 * 4);
     }

@@ -88,6 +88,12 @@ def test_topk_keep_everything():
     run_pair(2, [100, 4096, 5000], so.TOPK, 4, p=2, num=1, den=1)
 
 
+def test_topk_large_ratios_on_large_tensors():
+    """Half and a quarter of the entries kept: every candidate region is as large as its tensor."""
+    run_pair(2, [100, 40_000, 300_000], so.TOPK, 4, p=1, num=1, den=2)
+    run_pair(4, [5000, 70_000, 3 * 4096], so.TOPK, 4, p=3, num=1, den=4, lrs=[0.1, 0.3, 0.02])
+
+
 def test_sign_aligned_rows_vector_path():
     """d a multiple of 4 and tensors of whole tiles: every tile takes the 128-bit path."""
     run_pair(4, [4096, 8192, 4096 * 5, 64, 2048], so.SIGN, 6, p=1)
