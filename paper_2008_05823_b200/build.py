@@ -17,7 +17,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC", "-shared"]
 
 TARGETS = {
-    "libsae.so": (["sae.cu", "sae_noalloc.cu"], ["sae_kernels.cuh", "sae_worker_tma.cuh", "sae_worker_fused.cuh", "sae_topk.cuh", "sae_shard_topk.cuh", "sae_device.cuh", os.path.join(INCLUDE, "sae.h")]),
+    "libsae.so": (["sae.cu", "sae_noalloc.cu"], ["sae_kernels.cuh", "sae_worker_tma.cuh", "sae_worker_fused.cuh", "sae_worker_small.cuh", "sae_topk.cuh", "sae_shard_topk.cuh", "sae_device.cuh", os.path.join(INCLUDE, "sae.h")]),
     "libsae_synth.so": (["synth_gen.cu"], []),
 }
 

@@ -4,6 +4,7 @@
 #include "sae_kernels.cuh"
 #include "sae_worker_tma.cuh"
 #include "sae_worker_fused.cuh"
+#include "sae_worker_small.cuh"
 #include "sae_shard_topk.cuh"
 
 #include <cuda.h>
@@ -18,6 +19,10 @@
 #include <vector>
 
 // folded Top-K forms: the workers' threshold select on a second stream beside the server pass and its select
+// small problems: the short-chain worker pass instead of the persistent ones
+#ifndef SAE_SMALL_WORKER
+#define SAE_SMALL_WORKER 1
+#endif
 #ifndef SAE_TOPK_PARALLEL_SELECT
 #define SAE_TOPK_PARALLEL_SELECT 1
 #endif
@@ -72,6 +77,7 @@ struct sae_handle {
                            // e_srv holds Delta, the server records hold its L1 sum; the next server pass
                            // (or flush_server, before anything reads x or e) carries them out
   int inline_fin;          // small problem: the server pass forms the worker scales itself (one launch fewer)
+  int small_worker;        // ... and the worker pass is the short-chain kernel (k_worker_small)
   u32 *hist;
   SelectState* sel;
   // Top-K candidate windows: key lists, per-tensor region offsets / capacities, cursors, fallback flags
@@ -467,6 +473,27 @@ void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
   else launch_worker_wd<ESRC, SIGN, WRITE_D, false, TOPK>(h, sp, wa);
 }
 
+// The short-chain worker pass of small problems: a block per quarter tile, all workers.
+template <int ESRC, bool WRITE_D>
+void launch_small(sae_handle* h, const StepParams& sp, const WorkerArgs& wa, float eta_prev) {
+  SmallArgs a;
+  a.g = wa.g; a.m = wa.m; a.D = wa.D; a.ebar = const_cast<float*>(wa.ebar); a.x = wa.x; a.scale_prev = wa.scale_prev;
+  a.words = wa.words; a.recs = wa.recs; a.status = wa.status; a.eta_prev = eta_prev;
+  const size_t smem = (size_t)h->P.K * WS_ELEMS * sizeof(float);
+  const long long grid = (long long)h->P.ntiles * WS_SUB;
+  static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
+  if (configured_device != h->device) {
+    cudaFuncSetAttribute(k_worker_small<ESRC, WRITE_D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)(WS_MAXK * WS_ELEMS * sizeof(float)));
+    cudaFuncSetAttribute(k_worker_small<ESRC, WRITE_D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)(WS_MAXK * WS_ELEMS * sizeof(float)));
+    configured_device = h->device;
+  }
+  LaunchScope ls(h, S_WORKER);
+  if (sp.wd) k_worker_small<ESRC, WRITE_D, true><<<(unsigned)grid, THREADS, smem, h->stream>>>(h->P, sp, a);
+  else k_worker_small<ESRC, WRITE_D, false><<<(unsigned)grid, THREADS, smem, h->stream>>>(h->P, sp, a);
+}
+
 template <int COMP, int SRV>
 void launch_apply(sae_handle* h, int avg, const ApplyArgs& aa) {
   if (avg == AVG_NONE) LAUNCH(h, S_APPLY, (k_apply<COMP, SRV, AVG_NONE>), h->P.ntiles, h->P, aa);
@@ -643,12 +670,17 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
       fa.g = grads; fa.m = h->m; fa.ebar = ebar_now(h); fa.x = h->x; fa.scale_prev = h->scale[h->last];
       fa.words = h->words; fa.recs = recs_now; fa.status = h->status; fa.eta_prev = h->eta_prev; fa.g_tma_ok = 0;
       fa.ssum = h->tail_pending ? h->ssum : nullptr;
-      launch_fused(h, sp, fa);
+      if (h->small_worker) launch_small<ESRC_PENDING_AVG, false>(h, sp, wa, h->eta_prev);
+      else launch_fused(h, sp, fa);
     } else if (h->esrc == ESRC_UNIFORM) {
-      if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
+      if (h->small_worker) {
+        if (write_d) launch_small<ESRC_UNIFORM, true>(h, sp, wa, 0.0f); else launch_small<ESRC_UNIFORM, false>(h, sp, wa, 0.0f);
+      } else if (write_d) launch_worker<ESRC_UNIFORM, true, true>(h, sp, wa);
       else launch_worker<ESRC_UNIFORM, true, false>(h, sp, wa);
     } else if (h->esrc == ESRC_LOCAL_D) {
       launch_worker<ESRC_LOCAL_D, true, true>(h, sp, wa);
+    } else if (h->small_worker) {
+      launch_small<ESRC_LAZY_SIGN, true>(h, sp, wa, 0.0f);
     } else {
       launch_worker<ESRC_LAZY_SIGN, true, true>(h, sp, wa);
     }
@@ -1098,6 +1130,7 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   ALLOC0(h->recs, sign ? KT : 0); ALLOC0(h->recs_srv, sign ? T : 0);
   // latency-bound sizes (the whole K x d state fits L2 several times over): one launch fewer per step
   h->inline_fin = (sign && !shard && (long long)K * dpad <= (1ll << 24)) ? 1 : 0;
+  h->small_worker = (SAE_SMALL_WORKER && h->inline_fin && K <= WS_MAXK && !h->mu0) ? 1 : 0;
   if (h->inline_fin) {
     ALLOC0(h->recs_srv_alt, T); ALLOC0(h->recs_srv_alt2, T); ALLOC0(h->recs_srv_alt3, T); ALLOC0(h->recs_alt, KT);
   }

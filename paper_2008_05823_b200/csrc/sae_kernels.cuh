@@ -113,6 +113,9 @@ constexpr int SRV_B = 8;    // workers per batch of word loads
 #ifndef SAE_K3_STAGE
 #define SAE_K3_STAGE 1
 #endif
+#ifndef SAE_K3_FIN_EARLY
+#define SAE_K3_FIN_EARLY 1
+#endif
 #ifndef SAE_K3_SUM_DIRECT
 #define SAE_K3_SUM_DIRECT 1
 #endif
@@ -156,6 +159,9 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
   // the parameters with twelve independent 16-byte loads up front.)
   constexpr bool DIRECT = SUM && SAE_K3_SUM_DIRECT;
   constexpr bool STAGE = SAE_K3_STAGE && !FIN && !DIRECT;
+  // the server error (and parameters) fetched by the thread itself ahead of the worker loop: the streaming form,
+  // and the small problems, where a step is a chain of latencies and registers are not what limits the pass
+  constexpr bool EARLY = DIRECT || (FIN && SAE_K3_FIN_EARLY);
   __shared__ alignas(128) float s_e[STAGE ? TILE : 4];
   __shared__ alignas(128) float s_x[(STAGE && LAZY) ? TILE : 4];
   __shared__ alignas(8) u64 s_bar;
@@ -239,13 +245,13 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) sv[q] = ld4_stream(A.ssum + pbase + i + 4 * q);
       }
-      float4 ev[((DC || STAGE) && !DIRECT) ? 1 : SRV_E / 4];
-      float4 xd[(DIRECT && LAZY) ? SRV_E / 4 : 1];
-      if constexpr (DIRECT || (!DC && !STAGE)) {
+      float4 ev[((DC || STAGE) && !EARLY) ? 1 : SRV_E / 4];
+      float4 xd[(EARLY && LAZY) ? SRV_E / 4 : 1];
+      if constexpr (EARLY || (!DC && !STAGE)) {
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) ev[q] = ld4(ep + i + 4 * q);
       }
-      if constexpr (DIRECT && LAZY) {
+      if constexpr (EARLY && LAZY) {
 #pragma unroll
         for (int q = 0; q < SRV_E / 4; ++q) xd[q] = ld4(xp + i + 4 * q);
       }
@@ -299,13 +305,13 @@ __global__ void __launch_bounds__(THREADS) k_server_sign(Plan P, ServerArgs A, i
         }
         float4 e;
         if constexpr (STAGE) e = ld4(s_e + i + 4 * q);
-        else if constexpr (DIRECT) e = ev[q];
+        else if constexpr (EARLY) e = ev[q];
         else if constexpr (DC) e = ld4(ep + i + 4 * q);
         else e = ev[q];
         if constexpr (LAZY) {
           // e holds the previous step's Delta: C(Delta) is its scaled sign (double-way) or Delta itself
           float4 xv;
-          if constexpr (DIRECT) xv = xd[q];
+          if constexpr (EARLY) xv = xd[q];
           else xv = STAGE ? ld4(s_x + i + 4 * q) : ld4(xp + i + 4 * q);
           float4 cs;
           cs.x = DC ? sign_code(e.x, s_old) : e.x; cs.y = DC ? sign_code(e.y, s_old) : e.y;

@@ -61,8 +61,9 @@ def _fresh_handle_is_exact(K, sizes, p):
 
 
 def test_worker_pass_wait_runs_out():
-    """Item 0 of the plain worker pass = (tile 0, worker 0), a full tile fetched by bulk copies."""
-    K, sizes, p = 4, [3 * 4096, 5000], 0
+    """Item 0 of the plain worker pass = (tile 0, worker 0), a full tile fetched by bulk copies (a problem above
+    the small-problem limit: below it the worker pass makes no bulk copies)."""
+    K, sizes, p = 4, [(1 << 22) + 3 * 4096, 5000], 0
     status, elapsed = _run_until_timeout(K, sizes, p, drop=0, steps=1)
     assert status == (0, sb.ERR_TIMEOUT), status
     assert elapsed < 10.0
@@ -72,8 +73,8 @@ def test_worker_pass_wait_runs_out():
 def test_folded_worker_pass_wait_runs_out():
     """One worker, p = 1: the second step runs the folded-averaging pass, whose element ranges are half tiles --
     the dropped index lies beyond the first step's items (one per tile) and beyond the server pass's tiles."""
-    K, sizes, p = 1, [4 * 4096, 5000, 2 * 4096], 1
-    ntiles = 4 + 2 + 2
+    K, sizes, p = 1, [(1 << 24) + 4 * 4096, 5000, 2 * 4096], 1          # (above the small-problem limit)
+    ntiles = (1 << 12) + 4 + 2 + 2
     status, elapsed = _run_until_timeout(K, sizes, p, drop=2 * ntiles - 2, steps=3)
     assert status == (1, sb.ERR_TIMEOUT), status
     assert elapsed < 10.0
