@@ -269,7 +269,7 @@ def config_dict(w, p, args, world):
             "server_compress": "double-way" if w.server_compress else "single-way",
             "topk": f"{w.topk_num}/{w.topk_den}" if w.compressor == configs.TOPK else None,
             "local_steps": args.local_steps,
-            "caller_reads_state_between_steps": False,
+            "caller_reads_state_between_steps": bool(getattr(args, "read_step_ahead", False)),
             "parallelism": "replicas only" if world > 1 else "1 GPU, workers are a batch axis",
             "l2": l2_note(grad_bytes, ring)}
 
@@ -511,6 +511,9 @@ def main():
                          "with one rank it times the same two-phase, table-driven path on one GPU")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-step-ahead", action="store_true", help="skip the arm that reads the step-ahead point every step")
+    ap.add_argument("--read-step-ahead", action="store_true",
+                    help="make the headline itself the loop that fetches the step-ahead point after every step "
+                         "(the default run reports that loop beside the headline, as `with_step_ahead`)")
     ap.add_argument("--no-all-configs", dest="all_configs", action="store_false",
                     help="skip the short runs of every configuration under both schedules (default run only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -540,7 +543,8 @@ def main():
         w.name += f"_blk{args.block_size}"
     p = args.avg_period
     overridden = (args.workers > 0 or args.mode is not None or args.single_way or args.momentum is not None or
-                  args.topk_percent is not None or args.block_size > 0 or args.local_steps != 1 or p != 1)
+                  args.topk_percent is not None or args.block_size > 0 or args.local_steps != 1 or p != 1 or
+                  args.read_step_ahead)
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -693,9 +697,13 @@ def main():
     ring = ring_length(args, grad_bytes, p)
     gen, x0, grads = make_inputs(w, ring)
     head = measure(w, x0, grads, p, args.steps, max(args.warmup, ring + 1 if grad_bytes <= L2_BYTES else 0),
-                   local_steps=args.local_steps)
+                   read_step_ahead=args.read_step_ahead, local_steps=args.local_steps)
     ms_per_step, value, kernels = head["ms_per_step"], head["steps_per_s"], head["kernels"]
     step_bytes, worker_bytes, variant = algorithmic_bytes(w, p)
+    if args.read_step_ahead:                   # this loop's own byte count, and the plain worker pass it runs
+        step_bytes, _ = step_ahead_bytes(w, p)
+        if p == 1:
+            worker_bytes, variant = 12 * K * d + 4 * d, "uniform_error_pass"
     wk_ms = kernels["worker_pass"]["ms_per_launch"]
     achieved, frac, frac_nom = fractions(worker_bytes, wk_ms)
     per = WORKER_PASS_DRAM_BYTES.get(variant)
@@ -712,7 +720,7 @@ def main():
 
     # ---- the loop of Algorithm 1 as the paper runs it: the gradient point is read after every step --------
     with_step_ahead = None
-    if not args.no_step_ahead and args.local_steps == 1:
+    if not args.no_step_ahead and not args.read_step_ahead and args.local_steps == 1:
         sa_steps = max(3, min(args.steps, 30))
         sa = measure(w, x0, grads, p, sa_steps, args.warmup, read_step_ahead=True)
         sa_bytes, sa_formula = step_ahead_bytes(w, p)
