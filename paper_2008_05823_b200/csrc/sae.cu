@@ -477,8 +477,16 @@ void launch_worker(sae_handle* h, const StepParams& sp, const WorkerArgs& wa) {
 template <int ESRC, bool WRITE_D>
 void launch_small(sae_handle* h, const StepParams& sp, const WorkerArgs& wa, float eta_prev) {
   SmallArgs a;
+  memset(&a, 0, sizeof(a));
   a.g = wa.g; a.m = wa.m; a.D = wa.D; a.ebar = const_cast<float*>(wa.ebar); a.x = wa.x; a.scale_prev = wa.scale_prev;
   a.words = wa.words; a.recs = wa.recs; a.status = wa.status; a.eta_prev = eta_prev;
+  if (sp.wd && h->srv_pending) {
+    // weight decay: the previous step's server lines are carried out by this pass before it reads x
+    L1Record* rs[4] = {h->recs_srv, h->recs_srv_alt, h->recs_srv_alt2, h->recs_srv_alt3};
+    a.lsrv = 1; a.dc = h->cfg.server_compress ? 1 : 0; a.e_srv = h->e_srv; a.x_rw = h->x;
+    a.recs_srv_prev = rs[(h->rot + 3) % 4]; a.scale_srv = h->scale_srv;
+    h->srv_pending = 0;
+  }
   const size_t smem = (size_t)h->P.K * WS_ELEMS * sizeof(float);
   const long long grid = (long long)h->P.ntiles * WS_SUB;
   static thread_local int configured_device = -1;     // opt in to > 48 KB of dynamic shared memory once
@@ -651,7 +659,8 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     const bool defer_avg = avg_after && !write_d && h->fused_ok;
     // The server lines of this step can be left to the next step's server pass when nothing in between
     // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
-    const bool lazy_ok = SAE_LAZY_SERVER && !sp.wd;
+    // (small problems with weight decay: the lines wait as well, for the next worker pass, which carries them out)
+    const bool lazy_ok = SAE_LAZY_SERVER && (!sp.wd || (h->small_worker && h->local_steps <= 1));
     // Folded form (p = 1 steady state, large problems): the whole server pass of this step stays open -- the
     // next step's worker pass re-forms every message C(Delta^(k)) in its averager warps anyway and adds them up
     // in k order on the way; a streaming server pass then only reads that sum.

@@ -32,6 +32,14 @@ struct SmallArgs {
   L1Record* recs;            // [K][T]
   u32* status;
   float eta_prev;            // learning rate of the previous step (pending average)
+  // Weight decay makes the worker lines read x, so the server lines of the previous step (e = Delta - C(Delta),
+  // x = x - C(Delta)) cannot wait for the next server pass as they do otherwise; instead of a kernel of their own
+  // they are carried out here, element by element, before x is used (lsrv != 0):
+  int lsrv, dc;
+  float* e_srv;                    // [dpad] in: the pending Delta, out: the server error
+  float* x_rw;                     // [dpad] parameters
+  const L1Record* recs_srv_prev;   // [T] exact L1 sums of the pending Delta (double-way)
+  float* scale_srv;                // [T] out: the server scales formed from them
 };
 
 template <int ESRC, bool WRITE_D, bool WD>
@@ -59,6 +67,12 @@ __global__ void __launch_bounds__(THREADS) k_worker_small(Plan P, StepParams sp,
     }
   }
   if (ESRC != ESRC_UNIFORM && tid < K) s_scale[tid] = A.scale_prev[(long long)tid * P.T + ti.j];
+  __shared__ float s_srv;
+  if (WD && A.lsrv && A.dc && tid == 32) {           // (a thread of another warp than the scale loads)
+    const L1Record r = A.recs_srv_prev[ti.j];
+    s_srv = scale_from_limbs(r.limb[0], r.limb[1], r.limb[2], ti.n);
+    if (t0 == 0) A.scale_srv[ti.j] = s_srv;
+  }
   __syncthreads();
 
   const int e0 = tid * 4;                            // this thread's four elements
@@ -68,6 +82,24 @@ __global__ void __launch_bounds__(THREADS) k_worker_small(Plan P, StepParams sp,
   if (any) {
     if (ESRC != ESRC_LAZY_SIGN) eb = ld4(A.ebar + pbase + e0);
     if (WD) xv = ld4(A.x + pbase + e0);
+    if (WD && A.lsrv) {
+      // the pending server lines of these four elements (the operations of the apply kernel), then x as re-updated
+      const float4 ds = ld4(A.e_srv + pbase + e0);
+      const float ss = A.dc ? s_srv : 0.0f;
+      float4 cs;
+      cs.x = A.dc ? sign_code(ds.x, ss) : ds.x; cs.y = A.dc ? sign_code(ds.y, ss) : ds.y;
+      cs.z = A.dc ? sign_code(ds.z, ss) : ds.z; cs.w = A.dc ? sign_code(ds.w, ss) : ds.w;
+      float4 es;
+      es.x = __fsub_rn(ds.x, cs.x); es.y = __fsub_rn(ds.y, cs.y); es.z = __fsub_rn(ds.z, cs.z); es.w = __fsub_rn(ds.w, cs.w);
+      xv.x = __fsub_rn(xv.x, cs.x); xv.y = __fsub_rn(xv.y, cs.y); xv.z = __fsub_rn(xv.z, cs.z); xv.w = __fsub_rn(xv.w, cs.w);
+      if (!full) {                                   // the padding past the end of the tensor stays zero
+        if (e0 + 1 >= cnt) { es.y = 0.f; xv.y = 0.f; }
+        if (e0 + 2 >= cnt) { es.z = 0.f; xv.z = 0.f; }
+        if (e0 + 3 >= cnt) { es.w = 0.f; xv.w = 0.f; }
+      }
+      st4(A.e_srv + pbase + e0, es);
+      st4(A.x_rw + pbase + e0, xv);
+    }
   }
   if (ESRC == ESRC_PENDING_AVG && any) {
     // the average the previous step left pending, from the K momentum rows as they stand

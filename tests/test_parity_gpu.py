@@ -267,7 +267,7 @@ def test_graph_replay_on_a_side_stream(comp, p):
                 compare_state(gpu, orc, comp, tag=f"graph comp={comp} p={p} t={t + 1}")
                 compare_server_messages(gpu, orc, comp, 1, tag=f"graph comp={comp} p={p} t={t + 1}")
         per_step = np.diff(np.array(launches))
-        assert per_step.min() >= 3          # replayed steps still account for their kernels
+        assert per_step.min() >= 2          # replayed steps still account for their kernels (worker + server pass)
         gpu.close()
 
 
