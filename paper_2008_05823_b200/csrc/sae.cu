@@ -96,8 +96,8 @@ struct sae_handle {
   u32 *hist_srv, *work_count_srv, *cand_n_srv;
   SelectState* sel_srv;
   int2* work_srv;
-  cudaStream_t aux;
-  cudaEvent_t ev_fork, ev_join;
+  cudaStream_t aux, aux2[2];            // aux2: for the second launch of a select (workers' [0], server's [1])
+  cudaEvent_t ev_fork, ev_join, ev_fork2[2], ev_join2[2];
   long long cand_stride;
   u32* status;
   u32* status_host;      // pinned
@@ -229,6 +229,10 @@ struct ApiRange {       // an NVTX range around a whole entry point
     kern<<<(unsigned)(grid), THREADS, kDenseSmem, (h)->stream>>>(__VA_ARGS__);                             \
   } while (0)
 
+// for functions without a status of their own: a failed call is picked up by the step's check_launch below
+// (the runtime keeps the last error)
+#define SAE_CUDA_VOID(h, call) do { (void)(h); (void)(call); } while (0)
+
 int check_launch(sae_handle* h) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { h->last_cuda_error = (int)e; return SAE_ERR_CUDA; }
@@ -260,6 +264,11 @@ void free_all(sae_handle* h) {
   if (h->ev_fork) cudaEventDestroy(h->ev_fork);
   if (h->ev_join) cudaEventDestroy(h->ev_join);
   if (h->aux) cudaStreamDestroy(h->aux);
+  for (int i = 0; i < 2; ++i) {
+    if (h->ev_fork2[i]) cudaEventDestroy(h->ev_fork2[i]);
+    if (h->ev_join2[i]) cudaEventDestroy(h->ev_join2[i]);
+    if (h->aux2[i]) cudaStreamDestroy(h->aux2[i]);
+  }
   void* tabs[] = {(void*)h->d_word_rows, (void*)h->d_scale_rows[0], (void*)h->d_scale_rows[1], (void*)h->d_d_rows,
                   (void*)h->d_entry_rows, (void*)h->d_count_rows, (void*)h->d_tau_rows[0], (void*)h->d_tau_rows[1],
                   (void*)h->msg_entries, (void*)h->msg_count, (void*)h->agg_acc};
@@ -307,21 +316,36 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   const bool long_inline = server_row || h->topk_nod || !distributed;
   const int n_long = long_inline ? h->n_sel_long : 0;
   const int chunk_above = long_inline ? 0x7fffffff : SEL_LONG_REGION;
+#ifndef SAE_SEL_TWO_STREAMS
+#define SAE_SEL_TWO_STREAMS 1
+#endif
+  // The two launches take different lists: side by side where a second stream is at hand (the wide blocks leave
+  // half of every SM's thread slots free, the narrow ones fill them) -- not while kernels are timed one by one.
+  const int si = server_row ? 1 : 0;
+  const bool two = SAE_SEL_TWO_STREAMS && n_long > 0 && P.T > n_long && h->aux2[si] != nullptr && !h->profiling;
+  cudaStream_t short_stream = h->stream;
+  if (two) {
+    SAE_CUDA_VOID(h, cudaEventRecord(h->ev_fork2[si], h->stream));
+    SAE_CUDA_VOID(h, cudaStreamWaitEvent(h->aux2[si], h->ev_fork2[si], 0));
+    short_stream = h->aux2[si];
+  }
   if (n_long > 0) {
     LaunchScope ls(h, S_TOPK_SELECT);
     k_topk_select_window<1024><<<(unsigned)(rows * n_long), 1024, 0, h->stream>>>(
         P, cand, h->d_sel_list, n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb, fb_total,
-        inline_max, chunk_above, cand_n, work, work_count);
+        inline_max, chunk_above, cand_n, work, work_count, rows);
   }
   if (P.T > n_long) {
     LaunchScope ls(h, S_TOPK_SELECT);
-    k_topk_select_window<THREADS><<<(unsigned)(rows * (P.T - n_long)), THREADS, 0, h->stream>>>(
+    k_topk_select_window<THREADS><<<(unsigned)(rows * (P.T - n_long)), THREADS, 0, short_stream>>>(
         P, cand, h->d_sel_list + n_long, P.T - n_long, h->cfg.topk_num, h->cfg.topk_den, src, tau_guess, tau_out, fb,
-        fb_total, inline_max, chunk_above, cand_n, work, work_count);
+        fb_total, inline_max, chunk_above, cand_n, work, work_count, rows);
+  }
+  if (two) {
+    SAE_CUDA_VOID(h, cudaEventRecord(h->ev_join2[si], h->aux2[si]));
+    SAE_CUDA_VOID(h, cudaStreamWaitEvent(h->stream, h->ev_join2[si], 0));
   }
   if (!distributed) return;
-  const long long items = (long long)P.ntiles * rows;
-  LAUNCH(h, S_TOPK_SELECT, k_topk_worklist, (items + THREADS - 1) / THREADS, P, rows, fb, work, work_count);
   const long long hist_grid = 8LL * h->persistent_blocks;
   for (int level = 0; level < 3; ++level) {
     LAUNCH(h, S_TOPK_HIST, k_topk_hist, hist_grid, P, cand, rows, level, src, cand_n, sel, hist, work, work_count);
@@ -1185,6 +1209,11 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
     TRY(cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking));
     TRY(cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
     TRY(cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+    for (int i = 0; i < 2; ++i) {
+      TRY(cudaStreamCreateWithFlags(&h->aux2[i], cudaStreamNonBlocking));
+      TRY(cudaEventCreateWithFlags(&h->ev_fork2[i], cudaEventDisableTiming));
+      TRY(cudaEventCreateWithFlags(&h->ev_join2[i], cudaEventDisableTiming));
+    }
   }
 #endif
   ALLOC0(h->status, 1);

@@ -18,9 +18,9 @@
 // threshold is resolved by two histogram passes over it in shared memory -- the keys of a list lie in a narrow
 // window above `lo`, so they are binned by their distance from `lo` and spread evenly over the bins -- and a
 // pair whose window failed is resolved by the same block with the three-level radix select over its values
-// when the tensor is small.  Only large tensors whose window failed go to the work list of the distributed
-// three-level select (k_topk_worklist, then k_topk_hist / k_topk_select per level), whose launches find the
-// list empty otherwise.
+// when the tensor is small.  Only large tensors whose window failed queue their tiles on the work list of the
+// distributed three-level select (k_topk_hist / k_topk_select per level), whose launches find the list empty
+// otherwise.
 #pragma once
 #include "sae_device.cuh"
 
@@ -174,17 +174,6 @@ constexpr u32 FB_NONE = 0u;       // settled
 constexpr u32 FB_VALUES = 1u;     // the window failed on a large tensor: radix select over its values
 constexpr u32 FB_LIST = 2u;       // a long candidate list that holds the threshold: radix select over its chunks
 
-// Queues every (tile, row) data item whose (row, tensor) raised the fallback flag.
-__global__ void __launch_bounds__(THREADS) k_topk_worklist(Plan P, int rows, const u32* __restrict__ fallback, int2* work,
-                                                            u32* work_count) {
-  const long long nitems = (long long)P.ntiles * rows;
-  const long long mine = (long long)blockIdx.x * THREADS + threadIdx.x;
-  if (mine >= nitems) return;
-  const int tile = (int)(mine / rows);
-  const int k = (int)(mine - (long long)tile * rows);
-  if (fallback[(long long)k * P.T + P.tile_tensor[tile]] == FB_VALUES) work[atomicAdd(work_count, 1u)] = make_int2((int)mine, -1);
-}
-
 // The rows whose Top-K thresholds are wanted: stored ([rows][dpad] in buf), or -- when the worker pass did
 // not store the model differences -- recomputed as fma(eta, m^(k), ebar), the operation that formed them.
 struct DeltaSrc {
@@ -323,8 +312,8 @@ __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const
 // the pair is treated like a failed window.
 //
 // Failed window: tensors of at most inline_max elements are settled here by the three-level radix select
-// (11 + 10 + 10 bits) over their values, read by this block alone; larger ones raise their fallback flag for
-// the distributed select that follows.
+// (11 + 10 + 10 bits) over their values, read by this block alone; larger ones raise their fallback flag and queue
+// their tiles for the distributed select that follows.
 constexpr int WIN_BINS = 2048;            // covers 2^19 key units above lo: twice the window below the old threshold
 constexpr int SEL_U = 4;                  // loads a thread keeps in flight while it walks a list or a tensor
 constexpr int SEL_LONG_REGION = 16384;    // candidate regions above this many keys count as long (see topk_thresholds)
@@ -359,7 +348,7 @@ __global__ void __launch_bounds__(NT) k_topk_select_window(Plan P, CandArgs C, c
                                                             u32 num, u32 den, DeltaSrc src, const u32* tau_guess,
                                                             u32* tau_out, u32* fallback, u32* fallback_total,
                                                             int inline_max, int chain_min_cap, u32* cand_n, int2* work,
-                                                            u32* work_count) {
+                                                            u32* work_count, int rows) {
   __shared__ u32 sh[HIST_BINS];
   __shared__ u32 part[NT / 32];
   __shared__ u32 above[NT / 32];
@@ -446,8 +435,16 @@ __global__ void __launch_bounds__(NT) k_topk_select_window(Plan P, CandArgs C, c
   }
   // ---- the window failed ----
   if (tid == 0) atomicAdd(fallback_total, 1u);
-  if (n > inline_max) {
-    if (tid == 0) fallback[rj] = FB_VALUES;   // a large tensor: left to the distributed select
+  if (n > inline_max) {                       // a large tensor: its tiles to the distributed select
+    const int tiles = (n + TILE - 1) / TILE;
+    if (tid == 0) {
+      fallback[rj] = FB_VALUES;
+      sh_bin = atomicAdd(work_count, (u32)tiles);
+    }
+    __syncthreads();
+    const u32 base = sh_bin;
+    const int first = P.first_tile[j];
+    for (int t = tid; t < tiles; t += NT) work[base + t] = make_int2((first + t) * rows + row, -1);
     return;
   }
   if (tid == 0) fallback[rj] = FB_NONE;
