@@ -312,6 +312,9 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   //   * the workers with stored differences (no averaging every step: the unsent entries pile up below the
   //     threshold and the lists are several times longer): every long list's chunks go to the distributed select,
   //     -- / 0.890 (blocks of 1024 threads: 0.927).
+  // "Long" is a region of more than 65 536 keys (tensors above 0.8 M elements at 1 %): with the two launches side
+  // by side the narrow blocks take the mid-sized lists at no cost to the critical path (16 384 as the limit:
+  // 0.597 / 0.885; 65 536: 0.594 / 0.877; 131 072: 0.597 / 0.881).
   const bool server_row = fb == h->fb_srv;
   const bool long_inline = server_row || h->topk_nod || !distributed;
   const int n_long = long_inline ? h->n_sel_long : 0;

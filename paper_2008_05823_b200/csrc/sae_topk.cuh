@@ -316,7 +316,7 @@ __global__ void __launch_bounds__(THREADS) k_topk_select(int T, int level, const
 // their tiles for the distributed select that follows.
 constexpr int WIN_BINS = 2048;            // covers 2^19 key units above lo: twice the window below the old threshold
 constexpr int SEL_U = 4;                  // loads a thread keeps in flight while it walks a list or a tensor
-constexpr int SEL_LONG_REGION = 16384;    // candidate regions above this many keys count as long (see topk_thresholds)
+constexpr int SEL_LONG_REGION = 65536;    // candidate regions above this many keys count as long (see topk_thresholds)
 #ifndef SAE_TOPK_INLINE_MAX
 #define SAE_TOPK_INLINE_MAX 2048
 #endif
