@@ -683,7 +683,8 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     const bool write_d = h->mu0 || !((h->esrc == ESRC_UNIFORM || pending_in) && avg_after);
     if (write_d && !h->D) return SAE_ERR_INVALID_ARG;
     // p = 1: the average is not formed here but at the head of the next worker pass
-    const bool defer_avg = avg_after && !write_d && h->fused_ok;
+    // (the persistent folded pass takes power-of-two worker counts; the small-problem worker pass any)
+    const bool defer_avg = avg_after && !write_d && (h->fused_ok || (h->small_worker && c.avg_period == 1));
     // The server lines of this step can be left to the next step's server pass when nothing in between
     // needs x or e: no weight decay (the worker pass reads x), no averaging in the apply kernel.
     // (small problems with weight decay: the lines wait as well, for the next worker pass, which carries them out)
@@ -1704,7 +1705,7 @@ int sae_load_state(sae_handle* h, const void* in, size_t bytes) {
       hd.weight_decay != c.weight_decay || hd.worker_begin != h->k0 || hd.num_workers_total != h->K_total ||
       std::max(hd.local_steps, 1) != h->local_steps)
     return SAE_ERR_INVALID_ARG;                         // a checkpoint of a different configuration
-  if (hd.esrc == ESRC_PENDING_AVG && !h->fused_ok) return SAE_ERR_INVALID_ARG;
+  if (hd.esrc == ESRC_PENDING_AVG && !h->fused_ok && !(h->small_worker && c.avg_period == 1)) return SAE_ERR_INVALID_ARG;
   const char* q = (const char*)in + 256;
   for (const auto& s : ckpt_sections(h)) {
     SAE_CUDA(h, cudaMemcpyAsync(s.ptr, q, s.bytes, cudaMemcpyDeviceToDevice, h->stream));

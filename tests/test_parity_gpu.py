@@ -51,6 +51,29 @@ def test_sign_variants(dc, mode, mu, lam):
     run_pair(3, RAGGED, so.SIGN, 6, p=2, dc=dc, mode=mode, mu=mu, lam=lam, seed=1)
 
 
+@pytest.mark.parametrize("dc", [0, 1])
+@pytest.mark.parametrize("p", [0, 1, 3])
+def test_sign_weight_decay_small_problem_without_getters_in_between(dc, p):
+    """Weight decay makes the worker lines read x, so the server lines of a step cannot wait for the next server
+    pass; on small problems the next worker pass carries them out itself.  State compared every fourth step only,
+    so that most steps find the previous one's lines still pending; a steady p = 1 step is then two launches."""
+    import torch
+    K, sizes, seed = 3, RAGGED, 5
+    run_pair(K, sizes, so.SIGN, 13, seed=seed, p=p, dc=dc, lam=5e-4, lrs=[0.1, 0.1, 0.05], every=4)
+    if p == 1:
+        d = int(np.sum(sizes))
+        scales = synth.tensor_scales(seed, len(sizes), -4.0, -1.0)
+        gpu = sb.Sae(K, sizes, torch.from_numpy(synth.x0_numpy(seed, d)).cuda(), compressor=so.SIGN, server_compress=dc,
+                     avg_period=1, weight_decay=5e-4)
+        g = torch.from_numpy(synth.grads_numpy(seed, 0, K, sizes, scales)).cuda()
+        counts = []
+        for t in range(6):
+            gpu.step(g, 0.1)
+            counts.append(gpu.kernel_launches)
+        assert np.diff(np.array(counts))[-3:].tolist() == [2, 2, 2]
+        gpu.close()
+
+
 @pytest.mark.parametrize("K", [1, 3, 4])
 @pytest.mark.parametrize("p", [0, 1, 3])
 @pytest.mark.parametrize("num,den", [(1, 100), (1, 10)])
