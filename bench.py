@@ -261,7 +261,7 @@ def config_dict(w, p, args, world):
     """The `config` object of the JSON line: the same for the native and the reference arm."""
     from paper_2008_05823_b200 import configs
     grad_bytes = 4 * w.num_workers * w.d
-    ring = ring_length(args, grad_bytes, p)
+    ring = ring_length(args, grad_bytes, p, w.compressor == configs.TOPK)
     return {"workload": w.name, "num_workers": w.num_workers, "d": w.d, "num_tensors": w.num_tensors,
             "compressor": {0: "identity", 1: "scaled_sign", 2: "topk"}[w.compressor],
             "avg_period": p, "momentum": w.momentum, "lr": w.lr, "weight_decay": w.weight_decay,
@@ -274,18 +274,25 @@ def config_dict(w, p, args, world):
             "l2": l2_note(grad_bytes, ring)}
 
 
-def ring_length(args, grad_bytes, period=1):
+def ring_length(args, grad_bytes, period=1, topk=False):
     """Gradient sets kept in HBM and cycled, at most 40 GB of them.  Large sets: four, or two.  Sets smaller than
     L2: enough of them that the ring as a whole is twice L2 (a set is evicted before its turn comes again),
     rounded up to a multiple of the step pattern's period -- lcm(4, p): scale buffers alternate, record
     buffers rotate by four, every p-th step averages -- so that a given set always meets the same kind of step
-    and the library's cache of step graphs (keyed on the gradient pointer) stays small."""
+    and the library's cache of step graphs (keyed on the gradient pointer) stays small.
+    Top-K: as many sets as 40 GB hold, up to 48.  A short ring makes the gradients periodic, and with them the
+    momentum and the Top-K thresholds, which then jump from step to step by more than stochastic gradients make
+    them (the thresholds of about thirty (worker, tensor) pairs leave their candidate windows on every step of a
+    ring of 2 or 4 sets, none with a fresh set every step): work that a training run would not see."""
     import math
     if args.ring:
         return args.ring
+    pattern = math.lcm(4, max(1, period))
+    if grad_bytes > L2_BYTES and topk:
+        n = int(min(48, (40 << 30) // grad_bytes))
+        return n // pattern * pattern if n >= pattern else max(2, n // 2 * 2)
     if grad_bytes > L2_BYTES:
         return 4 if 4 * grad_bytes <= (40 << 30) else 2     # (powers of two divide the step pattern's period)
-    pattern = math.lcm(4, max(1, period))
     need = -(-2 * L2_BYTES // grad_bytes)
     return int(-(-need // pattern) * pattern)
 
@@ -682,7 +689,7 @@ def main():
         for idx in range(configs.NUM_WORKLOADS - 1):
             wl = configs.workload(idx)
             gb = 4 * wl.num_workers * wl.d
-            _, xs, gs = make_inputs(wl, ring_length(args, gb, wl.avg_period_paper))
+            _, xs, gs = make_inputs(wl, ring_length(args, gb, wl.avg_period_paper, wl.compressor == configs.TOPK))
             n_steps = {0: 400, 1: 400, 2: 100, 3: 100}[idx]
             for period in (1, wl.avg_period_paper):
                 # warm-up: every (gradient set, step kind) pair once, so that its step graph exists before the timed region
@@ -694,9 +701,10 @@ def main():
     # ---- headline: device-resident throughput, state not read between steps ------------------------------
     K, d = w.num_workers, w.d
     grad_bytes = 4 * K * d
-    ring = ring_length(args, grad_bytes, p)
+    ring = ring_length(args, grad_bytes, p, w.compressor == configs.TOPK)
     gen, x0, grads = make_inputs(w, ring)
-    head = measure(w, x0, grads, p, args.steps, max(args.warmup, ring + 1 if grad_bytes <= L2_BYTES else 0),
+    # (warm-up: every gradient set at least once, so that its step graph exists before the timed region)
+    head = measure(w, x0, grads, p, args.steps, max(args.warmup, ring + 1),
                    read_step_ahead=args.read_step_ahead, local_steps=args.local_steps)
     ms_per_step, value, kernels = head["ms_per_step"], head["steps_per_s"], head["kernels"]
     step_bytes, worker_bytes, variant = algorithmic_bytes(w, p)
