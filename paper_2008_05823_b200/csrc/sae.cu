@@ -86,6 +86,7 @@ struct sae_handle {
   int* d_cand_cap;
   int* d_sel_list;       // [T] the order in which the one-launch select takes the tensors
   int n_sel_long;        // how many of them (the first ones) have long candidate regions
+  int n_sel_long_srv;    // the same for the server's row, which counts shorter regions as long (see topk_thresholds)
   int* d_wlog2;          // [T] width of each tensor's candidate window (log2 of key units; WINDOW_ALL: whole tensor)
   int2* work;            // work list of the radix select: data items and candidate chunks
   u32* work_count;
@@ -317,7 +318,12 @@ void topk_thresholds(sae_handle* h, const DeltaSrc& src, int rows, const CandArg
   // 0.597 / 0.885; 65 536: 0.594 / 0.877; 131 072: 0.597 / 0.881).
   const bool server_row = fb == h->fb_srv;
   const bool long_inline = server_row || h->topk_nod || !distributed;
-  const int n_long = long_inline ? h->n_sel_long : 0;
+#ifndef SAE_SRV_LONG_REGION
+#define SAE_SRV_LONG_REGION 16384
+#endif
+  // (the server's select sits at the end of the step's longest chain, behind the server pass: there the mid-sized
+  // lists are worth wide blocks of their own -- 12 us beside 12 instead of 12 beside 24)
+  const int n_long = long_inline ? (server_row ? h->n_sel_long_srv : h->n_sel_long) : 0;
   const int chunk_above = long_inline ? 0x7fffffff : SEL_LONG_REGION;
 #ifndef SAE_SEL_TWO_STREAMS
 #define SAE_SEL_TWO_STREAMS 1
@@ -1204,6 +1210,8 @@ int init_impl(const sae_config* cfg, int k0, int K_loc, bool shard, const float*
   std::stable_sort(sel_list.begin(), sel_list.end(), [&](int a, int b) { return cand_cap[a] > cand_cap[b]; });
   h->n_sel_long = 0;
   for (int j = 0; j < T; ++j) if (cand_cap[j] > SEL_LONG_REGION) h->n_sel_long += 1;
+  h->n_sel_long_srv = 0;
+  for (int j = 0; j < T; ++j) if (cand_cap[j] > SAE_SRV_LONG_REGION) h->n_sel_long_srv += 1;
   ALLOC0(h->work, topk ? (size_t)ntiles * K + (size_t)K * (h->cand_stride / CAND_CHUNK + T) : 0);
   ALLOC0(h->work_count, 1); ALLOC0(h->cand_n, topk ? KT : 0);
 #if SAE_TOPK_PARALLEL_SELECT
