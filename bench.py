@@ -43,6 +43,8 @@ WORKER_PASS_DRAM_BYTES = {
     "sign_general": (19.64, 0.0, "ncu capture of the plain worker pass, config-2 shapes at 4 workers"),
     "sign_p1_folded": (12.0, 15.63, "ncu capture of k_worker_fused<32> on config 4 itself (one-pass metrics), "
                                     "43.752 GB per launch"),
+    "sign_p1_folded16": (12.0, 12.51, "ncu capture of k_worker_fused<16> on config 2 itself (one-pass metrics), "
+                                      "5.227 GB per launch"),
     "topk_p1": (12.0, 3.81, "ncu capture of the Top-K worker pass, config-3 shapes at 4 workers"),
     "topk_general": (19.83, 0.0, "ncu capture of the Top-K worker pass with stored differences, config-3 shapes at 4 workers"),
     "topk_p1_folded": (12.0, 12.18, "ncu capture of k_worker_fused<8, Top-K> on config 3"),
@@ -350,11 +352,12 @@ def algorithmic_bytes(w, avg_period):
         # Top-K: g R, m RW | ebar R (Delta is not stored: the server pass recomputes it from m)
         # Top-K with 8 or 16 workers and no weight decay, folded form: ebar R and W, and the worker-axis sum W
         folded = topk and w.num_workers in (8, 16) and w.weight_decay == 0.0
-        # scaled sign with 32 workers, no weight decay, above the small-problem limit: the worker pass also writes
+        # scaled sign from 16 workers on, no weight decay, above the small-problem limit: the worker pass also writes
         # the ordered sum of the previous step's messages (the folded server pass)
-        sign_folded = (not topk) and w.num_workers >= 32 and w.weight_decay == 0.0 and Wd > (1 << 24)
+        sign_folded = (not topk) and w.num_workers >= 16 and w.weight_decay == 0.0 and Wd > (1 << 24)
         worker = (12 * Wd + (12 if folded else 4) * d) if topk else 12 * Wd + (12 if sign_folded else 8) * d
-        variant = ("topk_p1_folded" if folded else "topk_p1") if topk else ("sign_p1_folded" if sign_folded else "sign_p1")
+        sign_variant = ("sign_p1_folded" if w.num_workers >= 32 else "sign_p1_folded16") if sign_folded else "sign_p1"
+        variant = ("topk_p1_folded" if folded else "topk_p1") if topk else sign_variant
     elif w.momentum == 0.0:
         step = 12 * Wd + 16 * d              # g R, e RW | x RW, e_srv RW  (mu = 0: no momentum rows)
         worker = 12 * Wd                     # g R, Delta(e) RW

@@ -28,7 +28,7 @@
 #endif
 // scaled sign, p = 1: from this many workers on, the server pass of a step is folded into the next worker pass
 #ifndef SAE_SIGN_FOLD_MIN_K
-#define SAE_SIGN_FOLD_MIN_K 32
+#define SAE_SIGN_FOLD_MIN_K 16
 #endif
 
 using namespace sae;
@@ -698,9 +698,10 @@ int do_step_direct(sae_handle* h, const float* grads, float lr) {
     // Folded form (p = 1 steady state, large problems): the whole server pass of this step stays open -- the
     // next step's worker pass re-forms every message C(Delta^(k)) in its averager warps anyway and adds them up
     // in k order on the way; a streaming server pass then only reads that sum.
-    // (Worth it from 32 workers on: the unpacking server pass costs K additions per parameter, the streaming
-    // one and the extra vector the worker pass writes do not depend on K -- config 4: 7.82 -> 7.62 ms per step,
-    // config 2 with 16 workers: 0.931 ms either way.)
+    // (Worth the more the more workers: the unpacking server pass costs K additions per parameter, the streaming
+    // one and the extra vector the worker pass writes do not depend on K -- config 4, 32 workers: 7.82 -> 7.62 ms
+    // per step; config 2, 16 workers: 0.945 -> 0.939, the worker pass 0.821 -> 0.842 and the server pass
+    // 0.122 -> 0.098; below 16 workers the unpacking pass is the cheaper one.)
     // The same open form, at any K, for a caller that reads the state between steps: the getter closes the step
     // in one pass over the momentum rows (flush_tail), which leaves the plain uniform error behind.
     const bool fold_sign = defer_avg && lazy_ok && !h->inline_fin && h->local_steps <= 1 &&
