@@ -61,4 +61,5 @@ def test_single_process_helpers():
     assert bench.whole_job_value(10, 1000.0, 1) == 10.0
     step, worker, variant = bench.algorithmic_bytes(__import__("paper_2008_05823_b200.configs", fromlist=["x"]).workload(2), 1)
     Wd, d = 16 * 25557032, 25557032
-    assert step == 12 * Wd + 24 * d and worker == 12 * Wd + 8 * d and variant == "sign_p1"
+    # (16 workers: the worker pass also writes the sum of the previous step's messages)
+    assert step == 12 * Wd + 24 * d and worker == 12 * Wd + 12 * d and variant == "sign_p1_folded16"
